@@ -1,0 +1,199 @@
+"""Plain fp64 CPU oracle of the L4Q quantization-aware LoRA linear layer.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, obviously-correct
+statement of what the CUDA library computes.  It shares no code with the CUDA
+path, imports nothing from it, and must never be called by it.
+
+Every function follows one passage of the paper (arXiv 2402.04902) in the
+paper's order and notation; there is no blocking, fusion or reordering.
+Matrix products use numpy's fp64 matmul as a library step.
+
+Layout (row-major, tokens flattened; the paper writes column vectors,
+``Y = W X``, this file writes the transposed, equivalent ``Y = X W^T``):
+
+    X  [M, i]   activations            dY [M, o]   upstream gradient
+    W0 [o, i]   frozen weight          A  [r, i], B [o, r]  LoRA factors
+    s, b [o, i/g]  scale / offset of each group of g consecutive elements
+                   of a weight row (groups run along d_in)
+
+Readings taken where the paper is silent (each is also listed in the design
+notes of the repository):
+  * the paper's constant "alpha" in Eq. 7 is ``gamma = alpha / rank`` here;
+  * round() is round-half-to-even;
+  * the integer grid is [Q_N, Q_P] = [-2^(n-1), 2^(n-1)-1] as in Eq. 3 when
+    ``signed_grid`` is set, else the shifted twin [0, 2^n - 1];
+  * the in-range test of the STE uses the *unrounded* w and is inclusive,
+    exactly as printed in App. A.1 / Eq. 13-14;
+  * dX = dY W_q is the textbook linear backward (the paper never prints it);
+  * the packed export format (bit order, fp16 parameters) is this library's.
+
+Pinned by tests/test_oracle_pins.py and tests/test_oracle_bruteforce.py
+against: B = 0 => merge == W0; grid membership; zero clipping under the
+Asymm / L4Q_init initialisations (Table 4, "Initial" E_clip = 0.0); the LoRA
+limits of Eq. 1-2; finite differences of the STE surrogate; a hand-worked
+example; scalar brute force on tiny layers; pack/unpack round trips.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+
+@dataclass(frozen=True)
+class L4QSpec:
+    """Hyper-parameters of one L4Q linear layer (Sec. 2.1, 2.2, 3.2)."""
+
+    rank: int
+    alpha: float
+    bits: int
+    group_size: int
+    signed_grid: bool = False
+    grad_scale: float = 1.0
+
+    @property
+    def gamma(self) -> float:
+        return float(self.alpha) / float(self.rank)
+
+
+def grid_bounds(spec: L4QSpec) -> tuple[int, int]:
+    """(Q_N, Q_P) of Eq. 3: signed [-2^(n-1), 2^(n-1)-1], or shifted to start at 0."""
+    n = spec.bits
+    if spec.signed_grid:
+        return -(1 << (n - 1)), (1 << (n - 1)) - 1
+    return 0, (1 << n) - 1
+
+
+def _f64(x) -> np.ndarray:
+    return np.asarray(x, dtype=np.float64)
+
+
+def _expand_groups(p: np.ndarray, group_size: int) -> np.ndarray:
+    """[o, G] per-group parameter -> [o, G*g], one value per weight element."""
+    return np.repeat(p, group_size, axis=1)
+
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Round fp64 values to the nearest bfloat16 (8 significant bits, ties to
+    even) and return them as fp64.  Normal range only (no subnormal/overflow
+    handling: layer values are O(1e-3 .. 1e3))."""
+    x = _f64(x)
+    m, e = np.frexp(x)                    # x = m * 2^e, 0.5 <= |m| < 1
+    return np.ldexp(np.rint(m * 256.0) / 256.0, e)
+
+
+def merge(spec: L4QSpec, W0, A, B) -> np.ndarray:
+    """Eq. 7: W_comb = W0 + gamma * B A."""
+    return _f64(W0) + spec.gamma * (_f64(B) @ _f64(A))
+
+
+def prequant(spec: L4QSpec, W_comb, s, b) -> np.ndarray:
+    """w = (W_comb - b) / s, the unrounded grid coordinate (App. A.2, definition of w)."""
+    g = spec.group_size
+    return (_f64(W_comb) - _expand_groups(_f64(b), g)) / _expand_groups(_f64(s), g)
+
+
+def quant_codes(spec: L4QSpec, w) -> np.ndarray:
+    """Eq. 8: w~ = round(clamp(w, Q_N, Q_P)), integer-valued fp64."""
+    qn, qp = grid_bounds(spec)
+    return np.rint(np.minimum(np.maximum(_f64(w), qn), qp))
+
+
+def dequant(spec: L4QSpec, w_tilde, s, b) -> np.ndarray:
+    """Eq. 9: W_q = w~ * s + b."""
+    g = spec.group_size
+    return _f64(w_tilde) * _expand_groups(_f64(s), g) + _expand_groups(_f64(b), g)
+
+
+def fake_quant_weight(spec: L4QSpec, W0, A, B, s, b):
+    """Eq. 7-9 in order.  Returns (w, w~, W_q)."""
+    w = prequant(spec, merge(spec, W0, A, B), s, b)
+    wt = quant_codes(spec, w)
+    return w, wt, dequant(spec, wt, s, b)
+
+
+def forward(spec: L4QSpec, X, W0, A, B, s, b, bf16_reference: bool = False) -> np.ndarray:
+    """Eq. 10: Y = X W_q^T.
+
+    ``bf16_reference``: W_q is rounded to bf16 before the product and Y after
+    it (what a bf16-operand, wide-accumulate GEMM sees); all sums stay fp64.
+    """
+    _, _, Wq = fake_quant_weight(spec, W0, A, B, s, b)
+    if bf16_reference:
+        Wq = round_to_bf16(Wq)
+    Y = _f64(X) @ Wq.T
+    return round_to_bf16(Y) if bf16_reference else Y
+
+
+def backward(spec: L4QSpec, X, dY, W0, A, B, s, b, bf16_reference: bool = False) -> dict:
+    """Backward of the layer; nothing is taken from the forward pass (App. E.2:
+    the quantized weight is recomputed).
+
+      dX = dY W_q                                   (textbook; implied by Eq. 10)
+      G  = dL/dW_q = dY^T X                         (Eq. 11)
+      m  = [Q_N <= w <= Q_P]                        (App. A.1, STE of round.clamp)
+      ds = sum_group G * {Q_N | w~ - w | Q_P}       (Eq. 5 and App. A.1, three cases)
+      db = sum_group G * (1 - m)                    (Eq. 6 and App. A.1)
+      dA = gamma * B^T (G * m)                      (Eq. 13 / App. A.2)
+      dB = gamma * (G * m) A^T                      (Eq. 14 / App. A.2)
+    """
+    X, dY, A, B = _f64(X), _f64(dY), _f64(A), _f64(B)
+    g = spec.group_size
+    qn, qp = grid_bounds(spec)
+    w, wt, Wq = fake_quant_weight(spec, W0, A, B, s, b)
+
+    Wq_mm = round_to_bf16(Wq) if bf16_reference else Wq
+    dX = dY @ Wq_mm
+    if bf16_reference:
+        dX = round_to_bf16(dX)
+
+    G = dY.T @ X                                            # Eq. 11, [o, i]
+    in_range = (w >= qn) & (w <= qp)
+    m = in_range.astype(np.float64)
+
+    dWq_ds = np.where(in_range, wt - w, np.where(w < qn, float(qn), float(qp)))
+    dWq_db = 1.0 - m
+    o, i = G.shape
+    ds = spec.grad_scale * (G * dWq_ds).reshape(o, i // g, g).sum(axis=2)
+    db = spec.grad_scale * (G * dWq_db).reshape(o, i // g, g).sum(axis=2)
+
+    Gm = G * m
+    dA = spec.gamma * (B.T @ Gm)
+    dB = spec.gamma * (Gm @ A.T)
+    return {"dX": dX, "dA": dA, "dB": dB, "ds": ds, "db": db}
+
+
+def pack_int(spec: L4QSpec, W0, A, B, s, b):
+    """Export of the fully quantized weight (Sec. 3.2: only w~, s, b are kept).
+
+    The paper fixes no storage format; this library's is:
+      u = w~ - Q_N  in [0, 2^n - 1]                 (unsigned code)
+      row bitstream: code j occupies bits [j*n, (j+1)*n), least significant bit
+      first, cut into little-endian 32-bit words -> codes[o, i*n/32] uint32
+      s16 = fp16(s);  b16 = fp16(fp32(b + s*Q_N))   (offset of the unsigned code;
+      formed in fp32, the precision s and b are trained in, then narrowed)
+    so that W_q ~= u * s16 + b16.  Returns (codes uint32, s16 float16, b16 float16).
+    """
+    n = spec.bits
+    qn, _ = grid_bounds(spec)
+    _, wt, _ = fake_quant_weight(spec, W0, A, B, s, b)
+    u = (wt - qn).astype(np.int64)
+    o, i = u.shape
+    if (i * n) % 32 != 0:
+        raise ValueError("d_in * bits must be a multiple of 32")
+    bits = ((u[:, :, None] >> np.arange(n, dtype=np.int64)) & 1).astype(np.uint8)   # [o, i, n], LSB first
+    stream = bits.reshape(o, i * n)
+    words = np.packbits(stream, axis=1, bitorder="little").view("<u4")
+    s16 = _f64(s).astype(np.float16)
+    b16 = (_f64(b) + _f64(s) * qn).astype(np.float32).astype(np.float16)
+    return np.ascontiguousarray(words), s16, b16
+
+
+def unpack_int(spec: L4QSpec, codes: np.ndarray, d_in: int) -> np.ndarray:
+    """Inverse of the bitstream of :func:`pack_int`: uint32 words -> unsigned codes [o, d_in]."""
+    n = spec.bits
+    codes = np.ascontiguousarray(codes.astype("<u4"))
+    o = codes.shape[0]
+    stream = np.unpackbits(codes.view(np.uint8), axis=1, bitorder="little")[:, : d_in * n]
+    bits = stream.reshape(o, d_in, n).astype(np.int64)
+    return (bits << np.arange(n, dtype=np.int64)).sum(axis=2)
