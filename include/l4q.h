@@ -1,0 +1,140 @@
+/*
+ * l4q.h -- C ABI of the B200 (sm_100a) L4Q linear-layer library.
+ *
+ * The layer (arXiv 2402.04902, Sec. 3.2) merges a frozen weight with a LoRA
+ * update, fake-quantizes the merge group-wise with a learnable scale and
+ * offset, and multiplies:
+ *
+ *     gamma  = alpha / rank
+ *     W_comb = W0 + gamma * B A                                   (Eq. 7)
+ *     w      = (W_comb - b) / s           per group of `group_size`
+ *                                         consecutive elements of a row
+ *     w~     = round(clamp(w, Q_N, Q_P))                          (Eq. 8)
+ *     W_q    = w~ * s + b                                         (Eq. 9)
+ *     Y      = X W_q^T                                            (Eq. 10)
+ *
+ * Layout: every tensor is dense row-major.  tokens = flattened batch x seq.
+ *     X [tokens, d_in]   Y, dY [tokens, d_out]   dX [tokens, d_in]
+ *     W0 [d_out, d_in]   A [rank, d_in]   B [d_out, rank]
+ *     s, b, ds, db [d_out, d_in / group_size]
+ * X, Y, dY, dX and W0 have the dtype `io_dtype` (bf16 or fp32); A, B, s, b
+ * and every parameter gradient are fp32.
+ *
+ * Integer grid: by default the codes are unsigned, [Q_N, Q_P] = [0, 2^bits-1];
+ * L4Q_FLAG_SIGNED_GRID selects the grid printed in Eq. 3,
+ * [-2^(bits-1), 2^(bits-1)-1].  round() is round-half-to-even.
+ *
+ * Conventions shared by every entry point:
+ *   - all tensor pointers are DEVICE pointers owned by the caller, 16-byte
+ *     aligned; the library allocates no memory and keeps nothing between
+ *     calls (the forward saves nothing for the backward: the backward
+ *     recomputes the quantized weight, App. E.2);
+ *   - `workspace` is caller-owned device scratch of at least
+ *     l4q_workspace_bytes() bytes, 256-byte aligned; its contents are
+ *     undefined before and after a call;
+ *   - calls are asynchronous on `cuda_stream` (a cudaStream_t, NULL = default
+ *     stream); outputs are overwritten, never accumulated into;
+ *   - errors are return codes only: no exception, no abort, no device trap.
+ *     A device-side wait that runs out of patience records L4Q_ERR_TIMEOUT in
+ *     a device status word which l4q_check() reads.
+ */
+#ifndef L4Q_H_
+#define L4Q_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  L4Q_OK = 0,
+  L4Q_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, misaligned pointer      */
+  L4Q_ERR_UNSUPPORTED = 2,   /* shape / bit-width / rank outside what the kernels cover */
+  L4Q_ERR_WORKSPACE = 3,     /* workspace missing or smaller than l4q_workspace_bytes()  */
+  L4Q_ERR_CUDA = 4,          /* a CUDA runtime or driver call failed                     */
+  L4Q_ERR_TIMEOUT = 5        /* a bounded device-side wait expired (results invalid)     */
+} l4q_status;
+
+enum { L4Q_BF16 = 0, L4Q_F32 = 1 };                 /* io_dtype */
+enum { L4Q_OP_FWD = 0, L4Q_OP_BWD = 1, L4Q_OP_PACK = 2 };
+enum {
+  L4Q_FLAG_SIGNED_GRID = 1u   /* codes in [-2^(bits-1), 2^(bits-1)-1] as in Eq. 3 */
+};
+
+/* Problem statement of one layer (Sec. 2.1, 2.2, 3.2).  Plain data, passed by pointer (host memory). */
+typedef struct l4q_desc {
+  int64_t  tokens;      /* rows of X / Y                                                   */
+  int64_t  d_in;        /* i: columns of W0; multiple of group_size                        */
+  int64_t  d_out;       /* o: rows of W0                                                   */
+  int32_t  rank;        /* r of the LoRA factors                                           */
+  float    alpha;       /* LoRA constant; the merge uses gamma = alpha / rank              */
+  int32_t  bits;        /* n: 2..8 for fwd/bwd, 3 or 4 for l4q_pack_int                    */
+  int32_t  group_size;  /* g: quantization group along d_in; multiple of 8                 */
+  int32_t  io_dtype;    /* L4Q_BF16 or L4Q_F32                                             */
+  uint32_t flags;       /* L4Q_FLAG_*                                                      */
+  float    grad_scale;  /* multiplies ds and db; 1.0f reproduces the paper                 */
+} l4q_desc;
+
+/* Bytes of device scratch the given op (L4Q_OP_*) needs for this problem; 0 if desc is invalid. */
+size_t l4q_workspace_bytes(const l4q_desc* desc, int op);
+
+/*
+ * Forward, Eq. 7-10: Y = X Q(W0 + gamma B A)^T.
+ * In: X, W0 (io_dtype), A, B, s, b (fp32).  Out: Y (io_dtype), overwritten.
+ * bf16 mode: W_q is rounded to bf16 and the product accumulates in fp32 on the
+ * tensor cores; fp32 mode is a plain-ALU validation path.
+ */
+l4q_status l4q_linear_fwd(const l4q_desc* desc, const void* X, const void* W0,
+                          const float* A, const float* B, const float* s, const float* b,
+                          void* Y, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward.  Recomputes W_q from (W0, A, B, s, b); takes nothing from the forward.
+ *   dX = dY W_q                                   (linear backward implied by Eq. 10)
+ *   G  = dY^T X                                   (Eq. 11; never written to memory as a whole)
+ *   m  = [Q_N <= w <= Q_P]                        (App. A.1, inclusive, on the unrounded w)
+ *   ds = grad_scale * sum_group G * {Q_N if w<Q_N | w~ - w if m | Q_P if w>Q_P}   (Eq. 5, App. A.1)
+ *   db = grad_scale * sum_group G * (1 - m)                                       (Eq. 6, App. A.1)
+ *   dA = gamma * B^T (G*m)                        (Eq. 13, App. A.2)
+ *   dB = gamma * (G*m) A^T                        (Eq. 14, App. A.2)
+ * Any of dX, dA, dB, ds, db may be NULL to skip it (dA, dB, ds, db are produced
+ * together: pass all four or none).  Outputs are overwritten.
+ */
+l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, const void* W0,
+                          const float* A, const float* B, const float* s, const float* b,
+                          void* dX, float* dA, float* dB, float* ds, float* db,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Export of the fully quantized layer (Sec. 3.2: inference keeps only w~, s, b).
+ * The paper fixes no storage format; this library's is:
+ *   u = w~ - Q_N in [0, 2^bits - 1]; code j of a row occupies bits
+ *   [j*bits, (j+1)*bits) of the row's bitstream, least significant bit first,
+ *   stored as little-endian 32-bit words: codes [d_out, d_in*bits/32] (uint32);
+ *   s_fp16 = fp16(s), b_fp16 = fp16(b + s*Q_N) as IEEE binary16 bit patterns
+ *   [d_out, d_in/group_size], so that W_q ~= u * s_fp16 + b_fp16.
+ * Codes are taken with the fp32 s and b (they equal the forward's codes).
+ * bits must be 3 or 4 and d_in*bits a multiple of 32.  Needs no workspace.
+ */
+l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, const float* B,
+                        const float* s, const float* b,
+                        uint32_t* codes, uint16_t* s_fp16, uint16_t* b_fp16,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns and clears the device status word
+ * (L4Q_OK, or L4Q_ERR_TIMEOUT if a kernel gave up on a bounded wait), or
+ * L4Q_ERR_CUDA if the stream reported an error. */
+l4q_status l4q_check(void* cuda_stream);
+
+/* Number of kernels launched by this library in this process since load (for launch accounting). */
+uint64_t l4q_launch_count(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char* l4q_status_string(l4q_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* L4Q_H_ */

@@ -1,0 +1,185 @@
+"""ctypes binding of ``libl4q.so`` (C ABI declared in ``include/l4q.h``).
+
+Argument marshalling only: every function here checks dtypes/shapes, takes
+``data_ptr()`` of torch CUDA tensors and calls the C entry point of the same
+name.  No layer arithmetic happens in Python and there is no fallback: if the
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from .synth import LayerConfig
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libl4q.so")
+
+L4Q_OK = 0
+L4Q_BF16, L4Q_F32 = 0, 1
+L4Q_OP_FWD, L4Q_OP_BWD, L4Q_OP_PACK = 0, 1, 2
+L4Q_FLAG_SIGNED_GRID = 1
+
+EXPORTED_SYMBOLS = (
+    "l4q_workspace_bytes", "l4q_linear_fwd", "l4q_linear_bwd", "l4q_pack_int",
+    "l4q_check", "l4q_launch_count", "l4q_status_string",
+)
+
+
+class L4QDesc(ctypes.Structure):
+    """Mirror of ``struct l4q_desc``."""
+
+    _fields_ = [
+        ("tokens", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64),
+        ("rank", ctypes.c_int32), ("alpha", ctypes.c_float),
+        ("bits", ctypes.c_int32), ("group_size", ctypes.c_int32),
+        ("io_dtype", ctypes.c_int32), ("flags", ctypes.c_uint32), ("grad_scale", ctypes.c_float),
+    ]
+
+
+class L4QError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (l4q_status {status})")
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libl4q.so`` (once). Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2402_04902_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, fp, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t
+        dp = ctypes.POINTER(L4QDesc)
+        L.l4q_workspace_bytes.restype = sz
+        L.l4q_workspace_bytes.argtypes = [dp, ctypes.c_int]
+        L.l4q_linear_fwd.restype = ctypes.c_int
+        L.l4q_linear_fwd.argtypes = [dp, vp, vp, fp, fp, fp, fp, vp, vp, sz, vp]
+        L.l4q_linear_bwd.restype = ctypes.c_int
+        L.l4q_linear_bwd.argtypes = [dp, vp, vp, vp, fp, fp, fp, fp, vp, fp, fp, fp, fp, vp, sz, vp]
+        L.l4q_pack_int.restype = ctypes.c_int
+        L.l4q_pack_int.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp, vp, vp, sz, vp]
+        L.l4q_check.restype = ctypes.c_int
+        L.l4q_check.argtypes = [vp]
+        L.l4q_launch_count.restype = ctypes.c_uint64
+        L.l4q_launch_count.argtypes = []
+        L.l4q_status_string.restype = ctypes.c_char_p
+        L.l4q_status_string.argtypes = [ctypes.c_int]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().l4q_status_string(int(status)).decode()
+
+
+def make_desc(cfg: LayerConfig, grad_scale: float = 1.0, tokens: Optional[int] = None) -> L4QDesc:
+    return L4QDesc(tokens=int(tokens if tokens is not None else cfg.tokens), d_in=cfg.d_in, d_out=cfg.d_out,
+                   rank=cfg.rank, alpha=float(cfg.alpha), bits=cfg.bits, group_size=cfg.group_size,
+                   io_dtype=L4Q_BF16 if cfg.io_dtype == "bf16" else L4Q_F32,
+                   flags=L4Q_FLAG_SIGNED_GRID if cfg.signed_grid else 0, grad_scale=float(grad_scale))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("L4Q tensors must be contiguous CUDA tensors")
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+
+
+def _raise(status: int, where: str) -> None:
+    if status != L4Q_OK:
+        raise L4QError(status, where)
+
+
+def l4q_workspace_bytes(desc: L4QDesc, op: int) -> int:
+    return int(lib().l4q_workspace_bytes(ctypes.byref(desc), int(op)))
+
+
+def alloc_workspace(desc: L4QDesc, op: int, device="cuda") -> torch.Tensor:
+    """Device scratch for one op (torch is used for device memory only)."""
+    n = max(l4q_workspace_bytes(desc, op), 256)
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def l4q_linear_fwd(desc: L4QDesc, X, W0, A, B, s, b, Y, workspace, stream=None) -> None:
+    st = lib().l4q_linear_fwd(ctypes.byref(desc), _ptr(X), _ptr(W0), _ptr(A), _ptr(B), _ptr(s), _ptr(b), _ptr(Y),
+                              _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream))
+    _raise(st, "l4q_linear_fwd")
+
+
+def l4q_linear_bwd(desc: L4QDesc, X, dY, W0, A, B, s, b, dX, dA, dB, ds, db, workspace, stream=None) -> None:
+    st = lib().l4q_linear_bwd(ctypes.byref(desc), _ptr(X), _ptr(dY), _ptr(W0), _ptr(A), _ptr(B), _ptr(s), _ptr(b),
+                              _ptr(dX), _ptr(dA), _ptr(dB), _ptr(ds), _ptr(db),
+                              _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream))
+    _raise(st, "l4q_linear_bwd")
+
+
+def l4q_pack_int(desc: L4QDesc, W0, A, B, s, b, codes, s_fp16, b_fp16, workspace=None, stream=None) -> None:
+    st = lib().l4q_pack_int(ctypes.byref(desc), _ptr(W0), _ptr(A), _ptr(B), _ptr(s), _ptr(b), _ptr(codes),
+                            _ptr(s_fp16), _ptr(b_fp16), _ptr(workspace),
+                            workspace.numel() if workspace is not None else 0, _stream(stream))
+    _raise(st, "l4q_pack_int")
+
+
+def l4q_check(stream=None) -> None:
+    """Synchronise the stream and raise if a kernel recorded an error."""
+    _raise(lib().l4q_check(_stream(stream)), "l4q_check")
+
+
+def l4q_launch_count() -> int:
+    return int(lib().l4q_launch_count())
+
+
+# ---------------------------------------------------------------------------
+# Convenience: move one synthetic layer (numpy, from synth.make_layer_inputs)
+# to the device in the dtypes the library expects.  Data movement only.
+# ---------------------------------------------------------------------------
+
+def to_device(cfg: LayerConfig, arrays: dict, device="cuda") -> dict:
+    io = torch.bfloat16 if cfg.io_dtype == "bf16" else torch.float32
+    out = {}
+    for k, v in arrays.items():
+        t = torch.from_numpy(v)
+        if k in ("X", "dY", "W0"):
+            t = t.to(io)           # exact: the values are representable in the io dtype
+        out[k] = t.to(device).contiguous()
+    return out
+
+
+def alloc_outputs(cfg: LayerConfig, device="cuda", tokens: Optional[int] = None) -> dict:
+    io = torch.bfloat16 if cfg.io_dtype == "bf16" else torch.float32
+    M = tokens if tokens is not None else cfg.tokens
+    G = cfg.d_in // cfg.group_size
+    f32 = torch.float32
+    return {
+        "Y": torch.empty(M, cfg.d_out, dtype=io, device=device),
+        "dX": torch.empty(M, cfg.d_in, dtype=io, device=device),
+        "dA": torch.empty(cfg.rank, cfg.d_in, dtype=f32, device=device),
+        "dB": torch.empty(cfg.d_out, cfg.rank, dtype=f32, device=device),
+        "ds": torch.empty(cfg.d_out, G, dtype=f32, device=device),
+        "db": torch.empty(cfg.d_out, G, dtype=f32, device=device),
+    }
+
+
+def alloc_pack_outputs(cfg: LayerConfig, device="cuda") -> dict:
+    G = cfg.d_in // cfg.group_size
+    return {
+        "codes": torch.empty(cfg.d_out, cfg.d_in * cfg.bits // 32, dtype=torch.int32, device=device),
+        "s16": torch.empty(cfg.d_out, G, dtype=torch.float16, device=device),
+        "b16": torch.empty(cfg.d_out, G, dtype=torch.float16, device=device),
+    }

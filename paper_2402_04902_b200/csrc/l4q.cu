@@ -1,0 +1,249 @@
+// C ABI of the L4Q library (see include/l4q.h): argument validation, workspace
+// layout and kernel launches.  One translation unit; the kernels live in the
+// headers included below.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+
+#include "l4q_common.cuh"
+#include "l4q_quant.cuh"
+#include "l4q_val.cuh"
+#include "l4q_gemm.cuh"
+
+using namespace l4q;
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+
+inline void count_launch(int n = 1) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks of the problem statement common to all ops.  Fills the kernel parameters.
+l4q_status make_params(const l4q_desc* d, Params* p) {
+  if (!d) return L4Q_ERR_INVALID_ARG;
+  if (d->tokens <= 0 || d->d_in <= 0 || d->d_out <= 0 || d->rank <= 0 || d->group_size <= 0)
+    return L4Q_ERR_INVALID_ARG;
+  if (d->io_dtype != L4Q_BF16 && d->io_dtype != L4Q_F32) return L4Q_ERR_INVALID_ARG;
+  if (!(d->alpha == d->alpha) || !(d->grad_scale == d->grad_scale)) return L4Q_ERR_INVALID_ARG;
+  if (d->tokens > (1 << 30) || d->d_in > (1 << 30) || d->d_out > (1 << 30)) return L4Q_ERR_UNSUPPORTED;
+  if (d->bits < 2 || d->bits > 8) return L4Q_ERR_UNSUPPORTED;
+  if (d->d_in % d->group_size != 0) return L4Q_ERR_UNSUPPORTED;
+  if (d->group_size % 8 != 0 || d->d_in % 8 != 0) return L4Q_ERR_UNSUPPORTED;
+  if (d->rank > 256) return L4Q_ERR_UNSUPPORTED;
+  if (d->io_dtype == L4Q_BF16 && d->d_out % 8 != 0) return L4Q_ERR_UNSUPPORTED;
+  p->tokens = (int)d->tokens; p->d_in = (int)d->d_in; p->d_out = (int)d->d_out;
+  p->rank = d->rank; p->bits = d->bits; p->group = d->group_size;
+  p->ngroups = (int)(d->d_in / d->group_size);
+  p->gamma = d->alpha / (float)d->rank;
+  if (d->flags & L4Q_FLAG_SIGNED_GRID) {
+    p->qn = -(float)(1 << (d->bits - 1)); p->qp = (float)((1 << (d->bits - 1)) - 1);
+  } else {
+    p->qn = 0.f; p->qp = (float)((1 << d->bits) - 1);
+  }
+  p->grad_scale = d->grad_scale;
+  return L4Q_OK;
+}
+
+size_t wq_scratch_bytes(const l4q_desc* d) {
+  const size_t esz = d->io_dtype == L4Q_BF16 ? 2 : 4;
+  return align_up((size_t)d->d_out * (size_t)d->d_in * esz, 256);
+}
+
+inline l4q_status launch_status() { return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA; }
+
+// Merge + fake-quantize the whole weight into `wq` (io dtype) -- the recompute step of fwd and bwd.
+template <bool IO_BF16>
+l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const float* B, const float* s,
+                          const float* b, void* wq, cudaStream_t st) {
+  const size_t smem = weight_tile_smem_bytes(p.rank);
+  auto kern = k_weight_tile<IO_BF16, WT_MODE_DEQUANT>;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return L4Q_ERR_CUDA;
+  dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
+  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, wq, nullptr, nullptr, nullptr);
+  count_launch();
+  return launch_status();
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t l4q_workspace_bytes(const l4q_desc* desc, int op) {
+  Params p;
+  if (make_params(desc, &p) != L4Q_OK) return 0;
+  switch (op) {
+    case L4Q_OP_FWD:
+    case L4Q_OP_BWD:
+      return wq_scratch_bytes(desc) + 256;
+    case L4Q_OP_PACK:
+    default:
+      return 0;
+  }
+}
+
+l4q_status l4q_linear_fwd(const l4q_desc* desc, const void* X, const void* W0, const float* A, const float* B,
+                          const float* s, const float* b, void* Y, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+  Params p;
+  l4q_status st = make_params(desc, &p);
+  if (st != L4Q_OK) return st;
+  if (!X || !W0 || !A || !B || !s || !b || !Y) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W0) || !aligned16(A) || !aligned16(B) || !aligned16(Y)) return L4Q_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < l4q_workspace_bytes(desc, L4Q_OP_FWD) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return L4Q_ERR_WORKSPACE;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  void* wq = workspace;
+  if (desc->io_dtype == L4Q_F32) {
+    st = launch_dequant<false>(p, W0, A, B, s, b, wq, stream);
+    if (st != L4Q_OK) return st;
+    GemmView g;
+    g.A = reinterpret_cast<const float*>(X); g.a_m = p.d_in; g.a_k = 1;
+    g.B = reinterpret_cast<const float*>(wq); g.b_k = 1; g.b_n = p.d_in;
+    g.M = p.tokens; g.N = p.d_out; g.K = p.d_in;
+    dim3 grid(ceil_div(g.N, VT), ceil_div(g.M, VT));
+    k_val_gemm<<<grid, V_THREADS, 0, stream>>>(g, reinterpret_cast<float*>(Y));
+    count_launch();
+    return launch_status();
+  }
+  st = launch_dequant<true>(p, W0, A, B, s, b, wq, stream);
+  if (st != L4Q_OK) return st;
+  int n = 0;
+  st = gemm_forward_bf16(p, X, wq, Y, stream, &n);
+  count_launch(n);
+  return st;
+}
+
+l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, const void* W0, const float* A,
+                          const float* B, const float* s, const float* b, void* dX, float* dA, float* dB,
+                          float* ds, float* db, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  Params p;
+  l4q_status st = make_params(desc, &p);
+  if (st != L4Q_OK) return st;
+  if (!X || !dY || !W0 || !A || !B || !s || !b) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(dY) || !aligned16(W0) || !aligned16(A) || !aligned16(B) || !aligned16(dX))
+    return L4Q_ERR_INVALID_ARG;
+  const int n_param_out = (dA != nullptr) + (dB != nullptr) + (ds != nullptr) + (db != nullptr);
+  if (n_param_out != 0 && n_param_out != 4) return L4Q_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < l4q_workspace_bytes(desc, L4Q_OP_BWD) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return L4Q_ERR_WORKSPACE;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  void* wq = workspace;
+  const bool f32 = desc->io_dtype == L4Q_F32;
+
+  if (n_param_out == 4) {
+    const size_t gsz = (size_t)p.d_out * p.ngroups * sizeof(float);
+    if (cudaMemsetAsync(dA, 0, (size_t)p.rank * p.d_in * sizeof(float), stream) != cudaSuccess ||
+        cudaMemsetAsync(dB, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess ||
+        cudaMemsetAsync(ds, 0, gsz, stream) != cudaSuccess || cudaMemsetAsync(db, 0, gsz, stream) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+  }
+  if (dX) {
+    st = f32 ? launch_dequant<false>(p, W0, A, B, s, b, wq, stream)
+             : launch_dequant<true>(p, W0, A, B, s, b, wq, stream);
+    if (st != L4Q_OK) return st;
+  }
+  if (f32) {
+    if (dX) {
+      GemmView g;
+      g.A = reinterpret_cast<const float*>(dY); g.a_m = p.d_out; g.a_k = 1;
+      g.B = reinterpret_cast<const float*>(wq); g.b_k = p.d_in; g.b_n = 1;
+      g.M = p.tokens; g.N = p.d_in; g.K = p.d_out;
+      dim3 grid(ceil_div(g.N, VT), ceil_div(g.M, VT));
+      k_val_gemm<<<grid, V_THREADS, 0, stream>>>(g, reinterpret_cast<float*>(dX));
+      count_launch();
+      if ((st = launch_status()) != L4Q_OK) return st;
+    }
+    if (n_param_out == 4) {
+      dim3 grid(ceil_div(p.d_in, VT), ceil_div(p.d_out, VT));
+      k_val_wgrad<<<grid, V_THREADS, 0, stream>>>(p, reinterpret_cast<const float*>(X),
+                                                  reinterpret_cast<const float*>(dY),
+                                                  reinterpret_cast<const float*>(W0), A, B, s, b, dA, dB, ds, db);
+      count_launch();
+      if ((st = launch_status()) != L4Q_OK) return st;
+    }
+    return L4Q_OK;
+  }
+  if (dX) {
+    int n = 0;
+    st = gemm_dgrad_bf16(p, dY, wq, dX, stream, &n);
+    count_launch(n);
+    if (st != L4Q_OK) return st;
+  }
+  if (n_param_out == 4) {
+    int n = 0;
+    st = gemm_wgrad_bf16(p, X, dY, W0, A, B, s, b, dA, dB, ds, db, stream, &n);
+    count_launch(n);
+    if (st != L4Q_OK) return st;
+  }
+  return L4Q_OK;
+}
+
+l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, const float* B, const float* s,
+                        const float* b, uint32_t* codes, uint16_t* s_fp16, uint16_t* b_fp16, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream) {
+  (void)workspace; (void)workspace_bytes;
+  Params p;
+  l4q_status st = make_params(desc, &p);
+  if (st != L4Q_OK) return st;
+  if (!W0 || !A || !B || !s || !b || !codes || !s_fp16 || !b_fp16) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(W0) || !aligned16(A) || !aligned16(codes)) return L4Q_ERR_INVALID_ARG;
+  if (p.bits != 3 && p.bits != 4) return L4Q_ERR_UNSUPPORTED;
+  if (((int64_t)p.d_in * p.bits) % 32 != 0) return L4Q_ERR_UNSUPPORTED;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const size_t smem = weight_tile_smem_bytes(p.rank);
+  dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
+  __half* s16 = reinterpret_cast<__half*>(s_fp16);
+  __half* b16 = reinterpret_cast<__half*>(b_fp16);
+  if (desc->io_dtype == L4Q_BF16) {
+    auto kern = k_weight_tile<true, WT_MODE_PACK>;
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+    kern<<<grid, WT_THREADS, smem, stream>>>(p, W0, A, B, s, b, nullptr, codes, s16, b16);
+  } else {
+    auto kern = k_weight_tile<false, WT_MODE_PACK>;
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+    kern<<<grid, WT_THREADS, smem, stream>>>(p, W0, A, B, s, b, nullptr, codes, s16, b16);
+  }
+  count_launch();
+  return launch_status();
+}
+
+l4q_status l4q_check(void* cuda_stream) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return L4Q_ERR_CUDA;
+  unsigned int word = 0;
+  if (cudaMemcpyFromSymbol(&word, g_l4q_status, sizeof(word)) != cudaSuccess) return L4Q_ERR_CUDA;
+  if (word != 0) {
+    const unsigned int zero = 0;
+    if (cudaMemcpyToSymbol(g_l4q_status, &zero, sizeof(zero)) != cudaSuccess) return L4Q_ERR_CUDA;
+    return (l4q_status)word;
+  }
+  return L4Q_OK;
+}
+
+uint64_t l4q_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* l4q_status_string(l4q_status status) {
+  switch (status) {
+    case L4Q_OK: return "ok";
+    case L4Q_ERR_INVALID_ARG: return "invalid argument";
+    case L4Q_ERR_UNSUPPORTED: return "unsupported shape, bit-width or rank";
+    case L4Q_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case L4Q_ERR_CUDA: return "CUDA call failed";
+    case L4Q_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,55 @@
+// Shared device/host helpers of the L4Q library: problem parameters, the
+// element-wise quantizer arithmetic (Eq. 7-9) and small utilities.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/l4q.h"
+
+namespace l4q {
+
+// Problem parameters in the form the kernels consume.
+struct Params {
+  int tokens, d_in, d_out, rank, bits, group, ngroups;
+  float gamma;        // alpha / rank            (Eq. 7)
+  float qn, qp;       // integer grid bounds     (Eq. 3)
+  float grad_scale;
+};
+
+// Device status word: 0 = ok, otherwise an l4q_status recorded by a kernel
+// that gave up on a bounded wait.  Read and cleared by l4q_check().
+__device__ unsigned int g_l4q_status;
+
+// Grid coordinate w, code w~ and dequantized value W_q of one merged weight.
+//   w  = (W_comb - b) * (1/s)      (App. A.2, definition of w; reciprocal taken once per group)
+//   w~ = rint(clamp(w, Q_N, Q_P))  (Eq. 8; rint = round-half-to-even)
+//   Wq = w~ * s + b                (Eq. 9)
+struct QuantElem {
+  float w, code, wq;
+};
+
+__device__ __forceinline__ QuantElem quantize_elem(float w_comb, float s, float rs, float b, float qn, float qp) {
+  QuantElem q;
+  q.w = (w_comb - b) * rs;
+  q.code = rintf(fminf(fmaxf(q.w, qn), qp));
+  q.wq = fmaf(q.code, s, b);
+  return q;
+}
+
+// W_comb = W0 + gamma * acc, acc = sum_k B[o,k] A[k,j]      (Eq. 7)
+__device__ __forceinline__ float merge_elem(float w0, float acc, float gamma) { return fmaf(gamma, acc, w0); }
+
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+}  // namespace l4q

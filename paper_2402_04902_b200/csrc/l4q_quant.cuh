@@ -1,0 +1,149 @@
+// Weight-tile kernel: merge (Eq. 7) + fake-quantize (Eq. 8-9) one 64 x 256 tile
+// of the weight per thread block, then either
+//   * write the dequantized W_q (bf16 or fp32) for the GEMM kernels, or
+//   * bit-pack the unsigned codes and narrow s, b to fp16 (export, Sec. 3.2).
+// HBM-bound by design: W0 is read with 128-bit loads, one 8-element vector per
+// thread per row, and every output line is written fully coalesced.  The rank-r
+// merge runs on the FP32 pipe with an 8-row x 8-column register block per
+// thread so that one shared-memory read of A feeds 8 rows.
+#pragma once
+
+#include "l4q_common.cuh"
+
+namespace l4q {
+
+constexpr int WT_ROWS = 64;      // rows of W per block
+constexpr int WT_COLS = 256;     // columns of W per block
+constexpr int WT_THREADS = 256;  // 8 warps; warp w owns rows [8w, 8w+8), lane l columns [8l, 8l+8)
+
+enum { WT_MODE_DEQUANT = 0, WT_MODE_PACK = 1 };
+
+inline size_t weight_tile_smem_bytes(int rank) {
+  return (size_t)rank * (WT_COLS + WT_ROWS) * sizeof(float);
+}
+
+template <bool IO_BF16>
+__device__ __forceinline__ void load_w0_vec8(const void* W0, size_t elem_off, float (&v)[8]) {
+  if constexpr (IO_BF16) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W0) + elem_off);
+    v[0] = bf16_lo(raw.x); v[1] = bf16_hi(raw.x); v[2] = bf16_lo(raw.y); v[3] = bf16_hi(raw.y);
+    v[4] = bf16_lo(raw.z); v[5] = bf16_hi(raw.z); v[6] = bf16_lo(raw.w); v[7] = bf16_hi(raw.w);
+  } else {
+    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(W0) + elem_off);
+    const float4 a = p[0], b = p[1];
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+}
+
+template <bool IO_BF16, int MODE>
+__global__ void __launch_bounds__(WT_THREADS)
+k_weight_tile(Params p, const void* __restrict__ W0, const float* __restrict__ A, const float* __restrict__ B,
+              const float* __restrict__ s, const float* __restrict__ b,
+              void* __restrict__ wq_out,                       // MODE_DEQUANT: [d_out, d_in] io dtype
+              uint32_t* __restrict__ codes, __half* __restrict__ s16, __half* __restrict__ b16) {  // MODE_PACK
+  extern __shared__ __align__(16) float smem_f[];
+  const int r = p.rank;
+  float4* A_lo = reinterpret_cast<float4*>(smem_f);            // [r][32]: columns 8l .. 8l+3 of lane l
+  float4* A_hi = A_lo + (size_t)r * 32;                        // [r][32]: columns 8l+4 .. 8l+7
+  float* Bt = reinterpret_cast<float*>(A_hi + (size_t)r * 32); // [r][64]: B[row0 + row][k] at Bt[k*64 + row]
+
+  const int col0 = blockIdx.x * WT_COLS;
+  const int row0 = blockIdx.y * WT_ROWS;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int idx = tid; idx < r * 64; idx += WT_THREADS) {
+    const int k = idx >> 6, v = idx & 63;
+    const int c = col0 + v * 4;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < p.d_in) a = *reinterpret_cast<const float4*>(A + (size_t)k * p.d_in + c);
+    ((v & 1) ? A_hi : A_lo)[k * 32 + (v >> 1)] = a;
+  }
+  for (int idx = tid; idx < r * WT_ROWS; idx += WT_THREADS) {
+    const int row = idx / r, k = idx - row * r;
+    const int o = row0 + row;
+    Bt[k * WT_ROWS + row] = (o < p.d_out) ? B[(size_t)o * r + k] : 0.f;
+  }
+  __syncthreads();
+
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+
+  for (int k = 0; k < r; ++k) {
+    const float4 a0 = A_lo[k * 32 + lane], a1 = A_hi[k * 32 + lane];
+    const float4 b0 = *reinterpret_cast<const float4*>(Bt + k * WT_ROWS + warp * 8);
+    const float4 b1 = *reinterpret_cast<const float4*>(Bt + k * WT_ROWS + warp * 8 + 4);
+    const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(bv[i], av[j], acc[i][j]);
+  }
+
+  const int col = col0 + lane * 8;
+  const bool col_ok = col < p.d_in;
+  const int grp = col_ok ? col / p.group : 0;
+  const int row_words = (int)(((int64_t)p.d_in * p.bits) >> 5);
+
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int o = row0 + warp * 8 + i;
+    if (o >= p.d_out) break;                      // uniform across the warp
+    float code[8];
+    float sv = 1.f, bvv = 0.f;
+    if (col_ok) {
+      float w0[8];
+      load_w0_vec8<IO_BF16>(W0, (size_t)o * p.d_in + col, w0);
+      sv = s[(size_t)o * p.ngroups + grp];
+      bvv = b[(size_t)o * p.ngroups + grp];
+      const float rs = 1.0f / sv;
+      float wq[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const QuantElem q = quantize_elem(merge_elem(w0[j], acc[i][j], p.gamma), sv, rs, bvv, p.qn, p.qp);
+        code[j] = q.code;
+        wq[j] = q.wq;
+      }
+      if constexpr (MODE == WT_MODE_DEQUANT) {
+        if constexpr (IO_BF16) {
+          uint4 out;
+          out.x = pack_bf16x2(wq[0], wq[1]); out.y = pack_bf16x2(wq[2], wq[3]);
+          out.z = pack_bf16x2(wq[4], wq[5]); out.w = pack_bf16x2(wq[6], wq[7]);
+          *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(wq_out) + (size_t)o * p.d_in + col) = out;
+        } else {
+          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(wq_out) + (size_t)o * p.d_in + col);
+          dst[0] = make_float4(wq[0], wq[1], wq[2], wq[3]);
+          dst[1] = make_float4(wq[4], wq[5], wq[6], wq[7]);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) code[j] = p.qn;
+    }
+    if constexpr (MODE == WT_MODE_PACK) {
+      // unsigned codes u = w~ - Q_N, 8 of them per thread, LSB-first
+      uint32_t piece = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) piece |= (uint32_t)(int)(code[j] - p.qn) << (j * p.bits);
+      uint32_t* row_codes = codes + (size_t)o * row_words;
+      if (p.bits == 4) {
+        if (col_ok) row_codes[col >> 3] = piece;                       // 32 lanes -> 128 contiguous bytes
+      } else {                                                         // bits == 3: 4 lanes x 24 bits -> 3 words
+        const uint32_t next = __shfl_down_sync(0xffffffffu, piece, 1);
+        const int t = lane & 3;
+        const uint32_t word = (piece >> (8 * t)) | (next << (24 - 8 * t));
+        const int widx = ((col >> 3) >> 2) * 3 + t;
+        if (t < 3 && widx < row_words) row_codes[widx] = word;        // 24 lanes -> 96 contiguous bytes
+      }
+      if (col_ok && (col % p.group) == 0) {
+        s16[(size_t)o * p.ngroups + grp] = __float2half_rn(sv);
+        b16[(size_t)o * p.ngroups + grp] = __float2half_rn(fmaf(sv, p.qn, bvv));
+      }
+    }
+  }
+}
+
+}  // namespace l4q
