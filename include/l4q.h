@@ -94,7 +94,10 @@ l4q_status l4q_linear_fwd(const l4q_desc* desc, const void* X, const void* W0,
  * Backward.  Recomputes W_q from (W0, A, B, s, b); takes nothing from the forward.
  *   dX = dY W_q                                   (linear backward implied by Eq. 10)
  *   G  = dY^T X                                   (Eq. 11; never written to memory as a whole)
- *   m  = [Q_N <= w <= Q_P]                        (App. A.1, inclusive, on the unrounded w)
+ *   m  = [Q_N <= w <= Q_P]                        (App. A.1, inclusive, on the unrounded w; each
+ *                                                  bound is widened by 2^-10 of a quantization step,
+ *                                                  so an element that a min/max initialisation puts
+ *                                                  exactly on a bound counts as in range, cf. Table 4)
  *   ds = grad_scale * sum_group G * {Q_N if w<Q_N | w~ - w if m | Q_P if w>Q_P}   (Eq. 5, App. A.1)
  *   db = grad_scale * sum_group G * (1 - m)                                       (Eq. 6, App. A.1)
  *   dA = gamma * B^T (G*m)                        (Eq. 13, App. A.2)

@@ -23,7 +23,12 @@ notes of the repository):
   * the integer grid is [Q_N, Q_P] = [-2^(n-1), 2^(n-1)-1] as in Eq. 3 when
     ``signed_grid`` is set, else the shifted twin [0, 2^n - 1];
   * the in-range test of the STE uses the *unrounded* w and is inclusive,
-    exactly as printed in App. A.1 / Eq. 13-14;
+    as printed in App. A.1 / Eq. 13-14, widened by a guard band of
+    ``mask_guard`` = 2^-10 of a quantization step on either side: a min/max
+    initialisation puts the extreme element of every group exactly on a bound
+    (w = Q_P up to the rounding of s), and Table 4 reports zero clipping for
+    that initialisation, so an element on the bound must count as inside no
+    matter which way the last bit of s was rounded;
   * dX = dY W_q is the textbook linear backward (the paper never prints it);
   * the packed export format (bit order, fp16 parameters) is this library's.
 
@@ -50,6 +55,7 @@ class L4QSpec:
     group_size: int
     signed_grid: bool = False
     grad_scale: float = 1.0
+    mask_guard: float = 2.0 ** -10    # guard band of the in-range test, in quantization steps
 
     @property
     def gamma(self) -> float:
@@ -131,7 +137,7 @@ def backward(spec: L4QSpec, X, dY, W0, A, B, s, b, bf16_reference: bool = False)
 
       dX = dY W_q                                   (textbook; implied by Eq. 10)
       G  = dL/dW_q = dY^T X                         (Eq. 11)
-      m  = [Q_N <= w <= Q_P]                        (App. A.1, STE of round.clamp)
+      m  = [Q_N - guard <= w <= Q_P + guard]        (App. A.1, STE of round.clamp; guard: see header)
       ds = sum_group G * {Q_N | w~ - w | Q_P}       (Eq. 5 and App. A.1, three cases)
       db = sum_group G * (1 - m)                    (Eq. 6 and App. A.1)
       dA = gamma * B^T (G * m)                      (Eq. 13 / App. A.2)
@@ -148,10 +154,10 @@ def backward(spec: L4QSpec, X, dY, W0, A, B, s, b, bf16_reference: bool = False)
         dX = round_to_bf16(dX)
 
     G = dY.T @ X                                            # Eq. 11, [o, i]
-    in_range = (w >= qn) & (w <= qp)
+    in_range = (w >= qn - spec.mask_guard) & (w <= qp + spec.mask_guard)
     m = in_range.astype(np.float64)
 
-    dWq_ds = np.where(in_range, wt - w, np.where(w < qn, float(qn), float(qp)))
+    dWq_ds = np.where(in_range, wt - w, np.where(w < qn, float(qn), float(qp)))   # out of range: the violated bound
     dWq_db = 1.0 - m
     o, i = G.shape
     ds = spec.grad_scale * (G * dWq_ds).reshape(o, i // g, g).sum(axis=2)

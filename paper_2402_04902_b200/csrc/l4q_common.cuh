@@ -39,6 +39,16 @@ __device__ __forceinline__ QuantElem quantize_elem(float w_comb, float s, float 
   return q;
 }
 
+// In-range test of the straight-through estimator (App. A.1): Q_N <= w <= Q_P on
+// the unrounded w, inclusive, widened by 2^-10 of a quantization step so that an
+// element a min/max initialisation puts exactly on a bound counts as inside
+// whichever way the last bit of s was rounded (Table 4: zero clipping at init).
+constexpr float kMaskGuard = 0.0009765625f;
+
+__device__ __forceinline__ bool ste_in_range(float w, float qn, float qp) {
+  return (w >= qn - kMaskGuard) && (w <= qp + kMaskGuard);
+}
+
 // W_comb = W0 + gamma * acc, acc = sum_k B[o,k] A[k,j]      (Eq. 7)
 __device__ __forceinline__ float merge_elem(float w0, float acc, float gamma) { return fmaf(gamma, acc, w0); }
 

@@ -114,7 +114,7 @@ k_val_wgrad(Params p, const float* __restrict__ X, const float* __restrict__ dY,
         const QuantElem q = quantize_elem(merge_elem(W0[(size_t)o * p.d_in + j], m_acc, p.gamma), sv, 1.0f / sv, bv,
                                           p.qn, p.qp);
         const float G = Gs[row][jj];
-        const bool in_range = (q.w >= p.qn) && (q.w <= p.qp);
+        const bool in_range = ste_in_range(q.w, p.qn, p.qp);
         if (in_range) {
           ds_acc = fmaf(G, q.code - q.w, ds_acc);
           gm = G;

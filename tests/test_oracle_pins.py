@@ -403,3 +403,30 @@ def test_round_to_bf16():
     rng = np.random.default_rng(15)
     y = rng.normal(size=1000)
     assert np.all(np.abs(orc.round_to_bf16(y) - y) <= np.abs(y) * 2.0 ** -8)
+
+
+def test_mask_guard_band_and_fp32_minmax_init_never_clips():
+    """An element within 2^-10 of a quantization step outside a bound still counts
+    as in range; with a min/max initialisation whose s was rounded to fp32 (so that
+    the group maximum sits at Q_P(1 +- 2^-24)) nothing is clipped: db == 0 exactly,
+    as Table 4 reports for the Asymm initialisation (E_clip = 0.0)."""
+    spec = L4QSpec(rank=1, alpha=1.0, bits=2, group_size=4)          # unsigned grid [0, 3]
+    s = np.array([[1.0]]); b = np.array([[0.0]])
+    W0 = np.array([[-2.0 ** -12, 3.0 + 2.0 ** -12, -2.0 ** -9, 3.0 + 2.0 ** -9]])
+    A = np.array([[1.0, 1.0, 1.0, 1.0]]); B = np.array([[0.0]])
+    X = np.eye(4); dY = np.array([[1.0], [10.0], [100.0], [1000.0]])
+    g = orc.backward(spec, X, dY, W0, A, B, s, b)
+    assert g["dB"][0, 0] == 1.0 + 10.0                                # first two inside the guard band
+    assert g["db"][0, 0] == 100.0 + 1000.0
+    rng = np.random.default_rng(21)
+    o, i, gsz = 16, 64, 16
+    spec = L4QSpec(rank=2, alpha=4.0, bits=4, group_size=gsz)
+    W0 = rng.normal(0, 0.02, (o, i)).astype(np.float32)
+    Wg = W0.reshape(o, i // gsz, gsz)
+    s32 = ((Wg.max(2) - Wg.min(2)) / np.float32(15)).astype(np.float32)
+    b32 = Wg.min(2)
+    A = rng.normal(size=(2, i)); B = np.zeros((o, 2))
+    w = orc.prequant(spec, orc.merge(spec, W0, A, B), s32, b32)
+    assert (w > 15).any()                                             # rounding of s does push some maxima past Q_P
+    g = orc.backward(spec, rng.normal(size=(4, i)), rng.normal(size=(4, o)), W0, A, B, s32, b32)
+    assert np.all(g["db"] == 0.0)
