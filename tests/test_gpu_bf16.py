@@ -1,0 +1,84 @@
+"""GPU parity of the bf16 tensor-core path (tcgen05 GEMMs + fused weight-gradient
+epilogue) against the fp64 oracle, element by element, on sizes the oracle
+finishes in seconds: exact tiles, ragged tails in every dimension, every
+supported rank, both grids, 3- and 4-bit."""
+import numpy as np
+import pytest
+
+from oracle import l4q_oracle as orc
+from paper_2402_04902_b200 import synth
+
+import gpu_harness as gh
+import parity_utils as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def check_layer(cfg, arrays, out, grad_scale=1.0):
+    spec = pu.spec_of(cfg, grad_scale)
+    a = pu.widen(arrays)
+    Y = orc.forward(spec, a["X"], a["W0"], a["A"], a["B"], a["s"], a["b"], bf16_reference=True)
+    g = orc.backward(spec, a["X"], a["dY"], a["W0"], a["A"], a["B"], a["s"], a["b"], bf16_reference=True)
+    errs = {"Y": pu.max_rel_err(out["Y"], Y), "dX": pu.max_rel_err(out["dX"], g["dX"])}
+    for k in ("dA", "dB", "ds", "db"):
+        errs[k] = pu.rel_l2(out[k], g[k])
+    print(cfg.name, {k: f"{v:.2e}" for k, v in errs.items()})
+    assert errs["Y"] <= pu.TOL_OUT["bf16"], errs
+    assert errs["dX"] <= pu.TOL_OUT["bf16"], errs
+    for k in ("dA", "dB", "ds", "db"):
+        assert errs[k] <= pu.TOL_GRAD["bf16"], errs
+    return errs
+
+
+def test_bf16_exact_tiles():
+    cfg = synth.LayerConfig("bf16_2x2_tiles", tokens=256, d_in=512, d_out=512, rank=16, alpha=32.0, bits=4,
+                            group_size=128)
+    arrays = synth.make_layer_inputs(cfg, seed=0)
+    check_layer(cfg, arrays, gh.run_layer(cfg, arrays))
+
+
+@pytest.mark.parametrize("rank,bits,group,signed", [
+    (16, 4, 64, False), (8, 4, 32, True), (32, 3, 64, False), (64, 3, 64, False), (16, 4, 104, True)])
+def test_bf16_ragged_tails(rank, bits, group, signed):
+    # tokens, d_in and d_out all leave partial tiles (128 / 256 / 64); d_in = 832 = 13 x 64 = 8 x 104
+    cfg = synth.LayerConfig(f"bf16_ragged_r{rank}", tokens=300, d_in=832, d_out=392, rank=rank, alpha=32.0,
+                            bits=bits, group_size=group, signed_grid=signed)
+    arrays = synth.make_layer_inputs(cfg, seed=7)
+    check_layer(cfg, arrays, gh.run_layer(cfg, arrays, grad_scale=0.25), grad_scale=0.25)
+
+
+def test_bf16_many_tiles_more_than_sms():
+    # 3 x 56 = 168 forward tiles > 148 SMs: exercises the persistent loop, both accumulator stages and phase flips
+    cfg = synth.LayerConfig("bf16_persistent", tokens=384, d_in=320, d_out=14336, rank=16, alpha=32.0, bits=4,
+                            group_size=64)
+    arrays = synth.make_layer_inputs(cfg, seed=11)
+    check_layer(cfg, arrays, gh.run_layer(cfg, arrays))
+
+
+def test_bf16_backward_is_linear_in_dY_and_additive_over_token_shards():
+    cfg = synth.LayerConfig("bf16_props", tokens=512, d_in=512, d_out=384, rank=16, alpha=32.0, bits=4,
+                            group_size=128)
+    arrays = synth.make_layer_inputs(cfg, seed=13)
+    full = gh.run_layer(cfg, arrays, do_fwd=False)
+    first = {k: (v[:256] if k in ("X", "dY") else v) for k, v in arrays.items()}
+    second = {k: (v[256:] if k in ("X", "dY") else v) for k, v in arrays.items()}
+    o1 = gh.run_layer(cfg, first, do_fwd=False)
+    o2 = gh.run_layer(cfg, second, do_fwd=False)
+    for k in ("dA", "dB", "ds", "db"):
+        assert pu.rel_l2(o1[k] + o2[k], full[k]) <= 1e-3, k
+    assert np.array_equal(np.vstack([o1["dX"], o2["dX"]]), full["dX"])
+    doubled = dict(arrays); doubled["dY"] = arrays["dY"] * np.float32(2.0)      # exact in bf16
+    o3 = gh.run_layer(cfg, doubled, do_fwd=False)
+    for k in ("dA", "dB", "ds", "db"):
+        assert pu.rel_l2(o3[k], 2.0 * full[k]) <= 1e-3, k
+    assert np.array_equal(o3["dX"], 2.0 * full["dX"])
+
+
+def test_bf16_zero_B_no_clipping():
+    cfg = synth.LayerConfig("bf16_zero_B", tokens=256, d_in=512, d_out=256, rank=16, alpha=32.0, bits=4,
+                            group_size=128)
+    arrays = synth.make_layer_inputs(cfg, seed=17, zero_B=True)
+    out = gh.run_layer(cfg, arrays)
+    check_layer(cfg, arrays, out)
+    assert np.all(out["db"] == 0.0)          # min/max init, B = 0: nothing outside the range (Table 4)
+    assert np.abs(out["dA"]).max() == 0.0    # dA = gamma B^T (G m) with B = 0
