@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the L4Q linear layer hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+for every L4Q linear of the workload, l4q_linear_fwd, l4q_linear_bwd (dX, dA,
+dB, ds, db) and l4q_pack_int.  The default workload is the LLaMA-7B-shaped MLP
+(up projection 4096 -> 11008 and down projection 11008 -> 4096, 8192 tokens,
+rank 16, 4-bit, group 128), the layer the throughput target is quoted on.
+
+Prints ONE JSON line (rank 0).  `value` is algorithmic TFLOP/s of the whole job
+(6*M*o*i + 8*o*i*r flops per linear and step) with inputs resident in HBM;
+`e2e` is the same metric with the step's activations (X, dY) copied from pinned
+host memory and the parameter gradients copied back inside the timed region.
+
+N > 1 (launched by torch.distributed.run, one rank per GPU): data parallel over
+tokens -- every rank runs the same layers on its own token batch (weak scaling)
+and the parameter gradients are all-reduced (sum) over NCCL each step.
+
+`--impl reference` times the fp64 CPU oracle (oracle/), as it stands, on the
+host cores on a bounded slice of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2402_04902_b200 import synth  # noqa: E402
+
+METRIC = "l4q_linear_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+
+
+def workloads() -> dict:
+    return {
+        "llama7b_mlp": [synth.CONFIG3A, synth.CONFIG3B],
+        "llama7b_attn_proj": [synth.CONFIG2],
+        "llama7b_mlp_3bit_r64": [synth.CONFIG4A, synth.CONFIG4B],
+        "mistral7b_block": synth.mistral_block_layers(),
+    }
+
+
+def layer_flops(cfg, tokens=None, d_out=None) -> float:
+    """Algorithmic flops of fwd + bwd of one linear: three M*o*i products, merge twice, dA and dB."""
+    M = cfg.tokens if tokens is None else tokens
+    o = cfg.d_out if d_out is None else d_out
+    return 6.0 * M * o * cfg.d_in + 8.0 * o * cfg.d_in * cfg.rank
+
+
+def peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"bf16_tflops": float(p["bf16_tflops"]), "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", 0)),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# --------------------------------------------------------------------------
+
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self) -> dict:
+        return {"sm_mhz": (statistics.median(self.samples) if self.samples else None),
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------
+# the oracle as CPU baseline / reference arm (bounded slice of one layer)
+# --------------------------------------------------------------------------
+
+def oracle_slice_step(cfg, arrays64, spec, rows: int):
+    from oracle import l4q_oracle as orc
+    a = arrays64
+    sl = slice(0, rows)
+    Y = orc.forward(spec, a["X"], a["W0"][sl], a["A"], a["B"][sl], a["s"][sl], a["b"][sl])
+    g = orc.backward(spec, a["X"], a["dY"][:, sl], a["W0"][sl], a["A"], a["B"][sl], a["s"][sl], a["b"][sl])
+    pk = orc.pack_int(spec, a["W0"][sl], a["A"], a["B"][sl], a["s"][sl], a["b"][sl])
+    return Y, g, pk
+
+
+def oracle_sample(cfg, tokens: int, rows: int, seed: int = 0):
+    from oracle import l4q_oracle as orc
+    small = cfg.with_(tokens=tokens)
+    arrays = synth.make_layer_inputs(small, seed=seed)
+    arrays64 = {k: np.asarray(v, dtype=np.float64) for k, v in arrays.items()}
+    spec = orc.L4QSpec(rank=cfg.rank, alpha=cfg.alpha, bits=cfg.bits, group_size=cfg.group_size,
+                       signed_grid=cfg.signed_grid)
+    return arrays64, spec
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 0) for d in threadpool_info() if d.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return int(os.cpu_count() or 1)
+
+
+def time_oracle(cfg, tokens: int, rows: int, steps: int, warmup: int):
+    arrays64, spec = oracle_sample(cfg, tokens, rows)
+    for _ in range(warmup):
+        oracle_slice_step(cfg, arrays64, spec, rows)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_slice_step(cfg, arrays64, spec, rows)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    flops = layer_flops(cfg, tokens=tokens, d_out=rows)
+    return dt, flops
+
+
+def run_reference(args, layers, wl_name):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = layers[0]
+    tokens, rows = 512, max(cfg.d_out // 4 // 8 * 8, 8)
+    dt, flops = time_oracle(cfg, tokens, rows, args.steps, args.warmup)
+    value = flops / dt / 1e12
+    sample = f"{cfg.name}: {tokens} of {cfg.tokens} tokens x first {rows} of {cfg.d_out} output rows, fwd+bwd+pack, fp64"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl_name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------
+
+def run_ours(args, layers, wl_name):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2402_04902_b200 import binding as l4q
+    from paper_2402_04902_b200 import build as l4q_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        l4q_build.build()
+    if world > 1:
+        dist.barrier()
+    l4q.lib()
+
+    # ---- synthetic layers: weights shared by all ranks, activations per rank (data parallel) ----
+    L = []
+    h2d = d2h = 0
+    for li, cfg in enumerate(layers):
+        arrays = synth.make_layer_inputs(cfg, seed=0, layer_id=li, need_acts=False)
+        acts = synth.make_layer_acts(cfg, seed=1000 + rank, layer_id=li)
+        host = {"X": torch.from_numpy(acts["X"]).to(torch.bfloat16).pin_memory(),
+                "dY": torch.from_numpy(acts["dY"]).to(torch.bfloat16).pin_memory()}
+        del acts
+        d = l4q.to_device(cfg, arrays, device=dev)
+        d["X"] = host["X"].to(dev)
+        d["dY"] = host["dY"].to(dev)
+        desc = l4q.make_desc(cfg)
+        outs = l4q.alloc_outputs(cfg, device=dev)
+        pk = l4q.alloc_pack_outputs(cfg, device=dev)
+        ws = l4q.alloc_workspace(desc, l4q.L4Q_OP_BWD, device=dev)
+        grads_host = {k: torch.empty_like(outs[k], device="cpu").pin_memory() for k in ("dA", "dB", "ds", "db")}
+        L.append(dict(cfg=cfg, desc=desc, d=d, outs=outs, pk=pk, ws=ws, host=host, grads_host=grads_host))
+        h2d += host["X"].numel() * 2 + host["dY"].numel() * 2
+        d2h += sum(t.numel() * 4 for t in grads_host.values())
+
+    def step(e2e: bool):
+        for l in L:
+            d, o, pk = l["d"], l["outs"], l["pk"]
+            if e2e:
+                d["X"].copy_(l["host"]["X"], non_blocking=True)
+                d["dY"].copy_(l["host"]["dY"], non_blocking=True)
+            l4q.l4q_linear_fwd(l["desc"], d["X"], d["W0"], d["A"], d["B"], d["s"], d["b"], o["Y"], l["ws"])
+            l4q.l4q_linear_bwd(l["desc"], d["X"], d["dY"], d["W0"], d["A"], d["B"], d["s"], d["b"],
+                               o["dX"], o["dA"], o["dB"], o["ds"], o["db"], l["ws"])
+            l4q.l4q_pack_int(l["desc"], d["W0"], d["A"], d["B"], d["s"], d["b"], pk["codes"], pk["s16"], pk["b16"])
+            if world > 1:
+                for k in ("dA", "dB", "ds", "db"):
+                    dist.all_reduce(o[k])
+            if e2e:
+                for k in ("dA", "dB", "ds", "db"):
+                    l["grads_host"][k].copy_(o[k], non_blocking=True)
+
+    def timed(e2e: bool, steps: int, warmup: int):
+        for _ in range(warmup):
+            step(e2e)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(steps):
+            step(e2e)
+        ev1.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    flops_step_rank = sum(layer_flops(l["cfg"]) for l in L)
+    tokens_step_rank = L[0]["cfg"].tokens
+
+    # ---- device-resident timing, with per-kernel events and clock samples ----
+    launches0 = l4q.l4q_launch_count()
+    l4q.l4q_profile_enable(True)
+    for _ in range(args.warmup):
+        step(False)
+    torch.cuda.synchronize()
+    l4q.l4q_profile_enable(False)
+    l4q.l4q_profile_enable(True)
+    launches0 = l4q.l4q_launch_count()
+    with ClockSampler(local_rank) as clk:
+        ms_total = timed(False, args.steps, 0)
+    launches = l4q.l4q_launch_count() - launches0
+    prof = l4q.l4q_profile_read()
+    l4q.l4q_profile_enable(False)
+    l4q.l4q_check()
+    ms_step = ms_total / args.steps
+    value = world * flops_step_rank / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end: host -> device copies of X, dY and device -> host of the gradients, every step ----
+    ms_e2e = timed(True, args.steps, max(1, min(args.warmup, 2))) / args.steps
+    e2e_value = world * flops_step_rank / (ms_e2e * 1e-3) / 1e12
+    l4q.l4q_check()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (live CUDA-event times from the timed region) ----
+    pk_ = peaks()
+    gemm_flops = {"gemm_fwd": 0.0, "gemm_dgrad": 0.0, "gemm_wgrad": 0.0}
+    pack_bytes = deq_bytes = 0.0
+    for l in L:
+        c = l["cfg"]
+        mm = 2.0 * c.tokens * c.d_out * c.d_in
+        gemm_flops["gemm_fwd"] += mm
+        gemm_flops["gemm_dgrad"] += mm
+        gemm_flops["gemm_wgrad"] += mm + 6.0 * c.d_out * c.d_in * c.rank
+        G = c.d_in // c.group_size
+        small = 4.0 * c.rank * (c.d_in + c.d_out)
+        pack_bytes += c.d_out * c.d_in * (2 + c.bits / 8) + c.d_out * G * 12 + small
+        deq_bytes += 2 * (c.d_out * c.d_in * 4 + c.d_out * G * 8 + small)      # two launches per step (fwd, bwd)
+    kernels = {}
+    for name, (n, ms) in prof.items():
+        if n:
+            kernels[name] = {"launches": n, "total_ms": ms, "avg_ms": ms / n}
+    total_kernel_ms = sum(k["total_ms"] for k in kernels.values()) or 1.0
+    for name, k in kernels.items():
+        k["share"] = k["total_ms"] / total_kernel_ms
+        steps_timed = args.steps
+        if name in gemm_flops:
+            k["tflops"] = gemm_flops[name] * steps_timed / (k["total_ms"] * 1e-3) / 1e12
+        elif name == "pack":
+            k["gbs"] = pack_bytes * steps_timed / (k["total_ms"] * 1e-3) / 1e9
+        elif name == "dequant":
+            k["gbs"] = deq_bytes * steps_timed / (k["total_ms"] * 1e-3) / 1e9
+    dominant = max(kernels, key=lambda n: kernels[n]["total_ms"]) if kernels else None
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        tj = json.load(open(tpath))
+        traffic = tj.get(wl_name, {}).get(dominant)
+    roofline = None
+    if dominant in gemm_flops:
+        ach = kernels[dominant]["tflops"]
+        roofline = {"kernel": dominant, "bound": "tensor", "achieved": ach, "peak": pk_["bf16_tflops"],
+                    "unit": "TFLOP/s", "frac": ach / pk_["bf16_tflops"], "traffic": traffic,
+                    "peak_source": pk_["source"] + " burst cuBLAS bf16",
+                    "frac_of_sustained": (ach / pk_["bf16_tflops_sustained"]) if pk_["bf16_tflops_sustained"] else None}
+    elif dominant is not None:
+        ach = kernels[dominant].get("gbs", 0.0)
+        roofline = {"kernel": dominant, "bound": "hbm", "achieved": ach, "peak": pk_["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / pk_["hbm_gbs"], "traffic": traffic, "peak_source": pk_["source"] + " copy"}
+
+    # ---- CPU baseline: the oracle, as it stands, on a bounded slice of the first layer ----
+    cfg0 = L[0]["cfg"]
+    tokens_s, rows_s = 512, max(cfg0.d_out // 4 // 8 * 8, 8)
+    dt, fl = time_oracle(cfg0, tokens_s, rows_s, steps=2, warmup=1)
+    cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+           "sample": f"{cfg0.name}: {tokens_s} of {cfg0.tokens} tokens x first {rows_s} of {cfg0.d_out} output rows, "
+                     f"fwd+bwd+pack, fp64, {dt:.2f} s per pass"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": wl_name,
+                   "layers": [f"{l['cfg'].d_in}->{l['cfg'].d_out}" for l in L],
+                   "tokens_per_gpu": tokens_step_rank, "rank": L[0]["cfg"].rank, "bits": L[0]["cfg"].bits,
+                   "group_size": L[0]["cfg"].group_size, "parallelism": f"dp{world}",
+                   "l2": "inputs larger than L2 (no flush)"},
+        "tokens_per_s": world * tokens_step_rank / (ms_step * 1e-3),
+        "frac_of_bf16_peak": value / world / pk_["bf16_tflops"],
+        "clocks": clk.summary(),
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "kernels": kernels,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="llama7b_mlp", choices=sorted(workloads()))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    layers = workloads()[args.workload]
+    if args.impl == "reference":
+        run_reference(args, layers, args.workload)
+    else:
+        run_ours(args, layers, args.workload)
+
+
+if __name__ == "__main__":
+    main()

@@ -134,6 +134,28 @@ l4q_status l4q_check(void* cuda_stream);
 /* Number of kernels launched by this library in this process since load (for launch accounting). */
 uint64_t l4q_launch_count(void);
 
+/*
+ * Optional per-kernel timing.  While enabled, every kernel this library launches
+ * is bracketed by a pair of CUDA events on its stream (a fixed pool of 8192
+ * pairs, created on the first enable; launches beyond the pool between two reads
+ * are not timed).  l4q_profile_read() waits for the recorded events, adds them
+ * to the running totals and returns, for one kernel (L4Q_KERNEL_*), the number
+ * of timed launches and their total device time in milliseconds since enabling.
+ */
+enum {
+  L4Q_KERNEL_DEQUANT = 0,     /* merge + fake-quantize -> W_q scratch (Eq. 7-9)             */
+  L4Q_KERNEL_PACK = 1,        /* merge + quantize + bit-pack (export)                       */
+  L4Q_KERNEL_GEMM_FWD = 2,    /* Y = X W_q^T (Eq. 10)                                       */
+  L4Q_KERNEL_GEMM_DGRAD = 3,  /* dX = dY W_q                                                */
+  L4Q_KERNEL_GEMM_WGRAD = 4,  /* dY^T X tiles reduced into ds, db, dA, dB (Eq. 11, 5-6, 13-14) */
+  L4Q_KERNEL_VAL_GEMM = 5,    /* fp32 validation GEMM                                       */
+  L4Q_KERNEL_VAL_WGRAD = 6,   /* fp32 validation weight-gradient reduction                  */
+  L4Q_KERNEL_COUNT = 7
+};
+l4q_status l4q_profile_enable(int enable);
+l4q_status l4q_profile_read(int kernel, uint64_t* launches, double* total_ms);
+const char* l4q_kernel_name(int kernel);
+
 /* Static, NUL-terminated description of a status code. */
 const char* l4q_status_string(l4q_status status);
 

@@ -111,27 +111,34 @@ def dequant(spec: L4QSpec, w_tilde, s, b) -> np.ndarray:
     return _f64(w_tilde) * _expand_groups(_f64(s), g) + _expand_groups(_f64(b), g)
 
 
-def fake_quant_weight(spec: L4QSpec, W0, A, B, s, b):
-    """Eq. 7-9 in order.  Returns (w, w~, W_q)."""
+def fake_quant_weight(spec: L4QSpec, W0, A, B, s, b, codes=None):
+    """Eq. 7-9 in order.  Returns (w, w~, W_q).
+
+    ``codes``: optional integer array taken as w~ instead of Eq. 8.  Where w sits
+    on (or within rounding error of) a tie k + 1/2, both neighbours are correct
+    results of round(); a caller that has checked another implementation's codes
+    to be such neighbours passes them here so that everything downstream of the
+    rounding decision is compared on the same decision.
+    """
     w = prequant(spec, merge(spec, W0, A, B), s, b)
-    wt = quant_codes(spec, w)
+    wt = quant_codes(spec, w) if codes is None else _f64(codes)
     return w, wt, dequant(spec, wt, s, b)
 
 
-def forward(spec: L4QSpec, X, W0, A, B, s, b, bf16_reference: bool = False) -> np.ndarray:
+def forward(spec: L4QSpec, X, W0, A, B, s, b, bf16_reference: bool = False, codes=None) -> np.ndarray:
     """Eq. 10: Y = X W_q^T.
 
     ``bf16_reference``: W_q is rounded to bf16 before the product and Y after
     it (what a bf16-operand, wide-accumulate GEMM sees); all sums stay fp64.
     """
-    _, _, Wq = fake_quant_weight(spec, W0, A, B, s, b)
+    _, _, Wq = fake_quant_weight(spec, W0, A, B, s, b, codes)
     if bf16_reference:
         Wq = round_to_bf16(Wq)
     Y = _f64(X) @ Wq.T
     return round_to_bf16(Y) if bf16_reference else Y
 
 
-def backward(spec: L4QSpec, X, dY, W0, A, B, s, b, bf16_reference: bool = False) -> dict:
+def backward(spec: L4QSpec, X, dY, W0, A, B, s, b, bf16_reference: bool = False, codes=None) -> dict:
     """Backward of the layer; nothing is taken from the forward pass (App. E.2:
     the quantized weight is recomputed).
 
@@ -146,7 +153,7 @@ def backward(spec: L4QSpec, X, dY, W0, A, B, s, b, bf16_reference: bool = False)
     X, dY, A, B = _f64(X), _f64(dY), _f64(A), _f64(B)
     g = spec.group_size
     qn, qp = grid_bounds(spec)
-    w, wt, Wq = fake_quant_weight(spec, W0, A, B, s, b)
+    w, wt, Wq = fake_quant_weight(spec, W0, A, B, s, b, codes)
 
     Wq_mm = round_to_bf16(Wq) if bf16_reference else Wq
     dX = dY @ Wq_mm

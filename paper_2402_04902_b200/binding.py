@@ -26,7 +26,11 @@ L4Q_FLAG_SIGNED_GRID = 1
 EXPORTED_SYMBOLS = (
     "l4q_workspace_bytes", "l4q_linear_fwd", "l4q_linear_bwd", "l4q_pack_int",
     "l4q_check", "l4q_launch_count", "l4q_status_string",
+    "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
 )
+
+KERNEL_IDS = {"dequant": 0, "pack": 1, "gemm_fwd": 2, "gemm_dgrad": 3, "gemm_wgrad": 4, "val_gemm": 5,
+              "val_wgrad": 6}
 
 
 class L4QDesc(ctypes.Structure):
@@ -74,6 +78,12 @@ def lib() -> ctypes.CDLL:
         L.l4q_launch_count.argtypes = []
         L.l4q_status_string.restype = ctypes.c_char_p
         L.l4q_status_string.argtypes = [ctypes.c_int]
+        L.l4q_profile_enable.restype = ctypes.c_int
+        L.l4q_profile_enable.argtypes = [ctypes.c_int]
+        L.l4q_profile_read.restype = ctypes.c_int
+        L.l4q_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_double)]
+        L.l4q_kernel_name.restype = ctypes.c_char_p
+        L.l4q_kernel_name.argtypes = [ctypes.c_int]
         _lib = L
     return _lib
 
@@ -143,6 +153,24 @@ def l4q_check(stream=None) -> None:
 
 def l4q_launch_count() -> int:
     return int(lib().l4q_launch_count())
+
+
+def l4q_profile_enable(enable: bool) -> None:
+    _raise(lib().l4q_profile_enable(1 if enable else 0), "l4q_profile_enable")
+
+
+def l4q_profile_read() -> dict:
+    """{kernel name: (timed launches, total device ms)} since profiling was enabled."""
+    out = {}
+    for name, kid in KERNEL_IDS.items():
+        n, ms = ctypes.c_uint64(0), ctypes.c_double(0.0)
+        _raise(lib().l4q_profile_read(kid, ctypes.byref(n), ctypes.byref(ms)), "l4q_profile_read")
+        out[name] = (int(n.value), float(ms.value))
+    return out
+
+
+def l4q_kernel_name(kernel: int) -> str:
+    return lib().l4q_kernel_name(int(kernel)).decode()
 
 
 # ---------------------------------------------------------------------------

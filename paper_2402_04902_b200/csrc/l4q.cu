@@ -4,6 +4,8 @@
 #include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "l4q_common.cuh"
 #include "l4q_quant.cuh"
@@ -16,10 +18,49 @@ namespace {
 
 std::atomic<uint64_t> g_launches{0};
 
-inline void count_launch(int n = 1) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+// ---- optional per-kernel timing (l4q_profile_*) ------------------------------
+struct ProfSlot { cudaEvent_t begin, end; int kernel; };
+std::mutex g_prof_mu;
+bool g_prof_on = false;
+std::vector<ProfSlot> g_prof_pool;
+size_t g_prof_used = 0;
+double g_prof_ms[L4Q_KERNEL_COUNT];
+uint64_t g_prof_n[L4Q_KERNEL_COUNT];
+constexpr size_t kProfPool = 8192;
+
+// Brackets one kernel launch: counts it and, when profiling is on, records a pair of events around it.
+class KernelScope {
+ public:
+  KernelScope(int kernel, cudaStream_t st) : st_(st) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    if (g_prof_on && g_prof_used < g_prof_pool.size()) {
+      slot_ = (long)g_prof_used++;
+      g_prof_pool[slot_].kernel = kernel;
+      cudaEventRecord(g_prof_pool[slot_].begin, st_);
+    }
+  }
+  ~KernelScope() {
+    if (slot_ >= 0) cudaEventRecord(g_prof_pool[slot_].end, st_);
+  }
+ private:
+  cudaStream_t st_;
+  long slot_ = -1;
+};
+
+void prof_drain_locked() {
+  for (size_t i = 0; i < g_prof_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(g_prof_pool[i].end) == cudaSuccess &&
+        cudaEventElapsedTime(&ms, g_prof_pool[i].begin, g_prof_pool[i].end) == cudaSuccess) {
+      g_prof_ms[g_prof_pool[i].kernel] += ms;
+      g_prof_n[g_prof_pool[i].kernel] += 1;
+    }
+  }
+  g_prof_used = 0;
+}
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Checks of the problem statement common to all ops.  Fills the kernel parameters.
@@ -48,6 +89,9 @@ l4q_status make_params(const l4q_desc* d, Params* p) {
   return L4Q_OK;
 }
 
+// The bf16 weight-gradient epilogue is instantiated for these ranks only.
+bool wgrad_rank_supported(int rank) { return rank == 8 || rank == 16 || rank == 32 || rank == 64; }
+
 size_t wq_scratch_bytes(const l4q_desc* d) {
   const size_t esz = d->io_dtype == L4Q_BF16 ? 2 : 4;
   return align_up((size_t)d->d_out * (size_t)d->d_in * esz, 256);
@@ -65,8 +109,22 @@ l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return L4Q_ERR_CUDA;
   dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
+  KernelScope ks(L4Q_KERNEL_DEQUANT, st);
   kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, wq, nullptr, nullptr, nullptr);
-  count_launch();
+  return launch_status();
+}
+
+template <bool IO_BF16>
+l4q_status launch_pack(const Params& p, const void* W0, const float* A, const float* B, const float* s,
+                       const float* b, uint32_t* codes, __half* s16, __half* b16, cudaStream_t st) {
+  const size_t smem = weight_tile_smem_bytes(p.rank);
+  auto kern = k_weight_tile<IO_BF16, WT_MODE_PACK>;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return L4Q_ERR_CUDA;
+  dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
+  KernelScope ks(L4Q_KERNEL_PACK, st);
+  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, nullptr, codes, s16, b16);
   return launch_status();
 }
 
@@ -108,16 +166,14 @@ l4q_status l4q_linear_fwd(const l4q_desc* desc, const void* X, const void* W0, c
     g.B = reinterpret_cast<const float*>(wq); g.b_k = 1; g.b_n = p.d_in;
     g.M = p.tokens; g.N = p.d_out; g.K = p.d_in;
     dim3 grid(ceil_div(g.N, VT), ceil_div(g.M, VT));
+    KernelScope ks(L4Q_KERNEL_VAL_GEMM, stream);
     k_val_gemm<<<grid, V_THREADS, 0, stream>>>(g, reinterpret_cast<float*>(Y));
-    count_launch();
     return launch_status();
   }
   st = launch_dequant<true>(p, W0, A, B, s, b, wq, stream);
   if (st != L4Q_OK) return st;
-  int n = 0;
-  st = gemm_forward_bf16(p, X, wq, Y, stream, &n);
-  count_launch(n);
-  return st;
+  KernelScope ks(L4Q_KERNEL_GEMM_FWD, stream);
+  return gemm_forward_bf16(p, X, wq, Y, stream);
 }
 
 l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, const void* W0, const float* A,
@@ -131,14 +187,16 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
     return L4Q_ERR_INVALID_ARG;
   const int n_param_out = (dA != nullptr) + (dB != nullptr) + (ds != nullptr) + (db != nullptr);
   if (n_param_out != 0 && n_param_out != 4) return L4Q_ERR_INVALID_ARG;
+  const bool f32 = desc->io_dtype == L4Q_F32;
+  if (!f32 && n_param_out == 4 && !wgrad_rank_supported(p.rank)) return L4Q_ERR_UNSUPPORTED;
   if (!workspace || workspace_bytes < l4q_workspace_bytes(desc, L4Q_OP_BWD) ||
       (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return L4Q_ERR_WORKSPACE;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   void* wq = workspace;
-  const bool f32 = desc->io_dtype == L4Q_F32;
 
   if (n_param_out == 4) {
+    // the reductions below accumulate with fp32 atomics: start from zero
     const size_t gsz = (size_t)p.d_out * p.ngroups * sizeof(float);
     if (cudaMemsetAsync(dA, 0, (size_t)p.rank * p.d_in * sizeof(float), stream) != cudaSuccess ||
         cudaMemsetAsync(dB, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess ||
@@ -157,30 +215,28 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
       g.B = reinterpret_cast<const float*>(wq); g.b_k = p.d_in; g.b_n = 1;
       g.M = p.tokens; g.N = p.d_in; g.K = p.d_out;
       dim3 grid(ceil_div(g.N, VT), ceil_div(g.M, VT));
+      KernelScope ks(L4Q_KERNEL_VAL_GEMM, stream);
       k_val_gemm<<<grid, V_THREADS, 0, stream>>>(g, reinterpret_cast<float*>(dX));
-      count_launch();
       if ((st = launch_status()) != L4Q_OK) return st;
     }
     if (n_param_out == 4) {
       dim3 grid(ceil_div(p.d_in, VT), ceil_div(p.d_out, VT));
+      KernelScope ks(L4Q_KERNEL_VAL_WGRAD, stream);
       k_val_wgrad<<<grid, V_THREADS, 0, stream>>>(p, reinterpret_cast<const float*>(X),
                                                   reinterpret_cast<const float*>(dY),
                                                   reinterpret_cast<const float*>(W0), A, B, s, b, dA, dB, ds, db);
-      count_launch();
       if ((st = launch_status()) != L4Q_OK) return st;
     }
     return L4Q_OK;
   }
   if (dX) {
-    int n = 0;
-    st = gemm_dgrad_bf16(p, dY, wq, dX, stream, &n);
-    count_launch(n);
+    KernelScope ks(L4Q_KERNEL_GEMM_DGRAD, stream);
+    st = gemm_dgrad_bf16(p, dY, wq, dX, stream);
     if (st != L4Q_OK) return st;
   }
   if (n_param_out == 4) {
-    int n = 0;
-    st = gemm_wgrad_bf16(p, X, dY, W0, A, B, s, b, dA, dB, ds, db, stream, &n);
-    count_launch(n);
+    KernelScope ks(L4Q_KERNEL_GEMM_WGRAD, stream);
+    st = gemm_wgrad_bf16(p, X, dY, W0, A, B, s, b, dA, dB, ds, db, stream);
     if (st != L4Q_OK) return st;
   }
   return L4Q_OK;
@@ -198,25 +254,10 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
   if (p.bits != 3 && p.bits != 4) return L4Q_ERR_UNSUPPORTED;
   if (((int64_t)p.d_in * p.bits) % 32 != 0) return L4Q_ERR_UNSUPPORTED;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-  const size_t smem = weight_tile_smem_bytes(p.rank);
-  dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
   __half* s16 = reinterpret_cast<__half*>(s_fp16);
   __half* b16 = reinterpret_cast<__half*>(b_fp16);
-  if (desc->io_dtype == L4Q_BF16) {
-    auto kern = k_weight_tile<true, WT_MODE_PACK>;
-    if (smem > 48 * 1024 &&
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return L4Q_ERR_CUDA;
-    kern<<<grid, WT_THREADS, smem, stream>>>(p, W0, A, B, s, b, nullptr, codes, s16, b16);
-  } else {
-    auto kern = k_weight_tile<false, WT_MODE_PACK>;
-    if (smem > 48 * 1024 &&
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return L4Q_ERR_CUDA;
-    kern<<<grid, WT_THREADS, smem, stream>>>(p, W0, A, B, s, b, nullptr, codes, s16, b16);
-  }
-  count_launch();
-  return launch_status();
+  return desc->io_dtype == L4Q_BF16 ? launch_pack<true>(p, W0, A, B, s, b, codes, s16, b16, stream)
+                                    : launch_pack<false>(p, W0, A, B, s, b, codes, s16, b16, stream);
 }
 
 l4q_status l4q_check(void* cuda_stream) {
@@ -233,6 +274,48 @@ l4q_status l4q_check(void* cuda_stream) {
 }
 
 uint64_t l4q_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+l4q_status l4q_profile_enable(int enable) {
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  if (enable && g_prof_pool.empty()) {
+    g_prof_pool.resize(kProfPool);
+    for (auto& sl : g_prof_pool) {
+      if (cudaEventCreate(&sl.begin) != cudaSuccess || cudaEventCreate(&sl.end) != cudaSuccess) {
+        g_prof_pool.clear();
+        return L4Q_ERR_CUDA;
+      }
+    }
+  }
+  if (enable && !g_prof_on) {
+    g_prof_used = 0;
+    for (int k = 0; k < L4Q_KERNEL_COUNT; ++k) { g_prof_ms[k] = 0.0; g_prof_n[k] = 0; }
+  }
+  if (!enable && g_prof_on) prof_drain_locked();
+  g_prof_on = enable != 0;
+  return L4Q_OK;
+}
+
+l4q_status l4q_profile_read(int kernel, uint64_t* launches, double* total_ms) {
+  if (kernel < 0 || kernel >= L4Q_KERNEL_COUNT || !launches || !total_ms) return L4Q_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  prof_drain_locked();
+  *launches = g_prof_n[kernel];
+  *total_ms = g_prof_ms[kernel];
+  return L4Q_OK;
+}
+
+const char* l4q_kernel_name(int kernel) {
+  switch (kernel) {
+    case L4Q_KERNEL_DEQUANT: return "k_weight_tile<dequant>";
+    case L4Q_KERNEL_PACK: return "k_weight_tile<pack>";
+    case L4Q_KERNEL_GEMM_FWD: return "k_gemm_bf16<fwd>";
+    case L4Q_KERNEL_GEMM_DGRAD: return "k_gemm_bf16<dgrad>";
+    case L4Q_KERNEL_GEMM_WGRAD: return "k_gemm_bf16<wgrad>";
+    case L4Q_KERNEL_VAL_GEMM: return "k_val_gemm";
+    case L4Q_KERNEL_VAL_WGRAD: return "k_val_wgrad";
+    default: return "unknown kernel";
+  }
+}
 
 const char* l4q_status_string(l4q_status status) {
   switch (status) {

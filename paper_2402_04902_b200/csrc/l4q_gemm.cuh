@@ -476,36 +476,31 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
 }
 
 // Y[tokens, d_out] = X[tokens, d_in] Wq[d_out, d_in]^T
-inline l4q_status gemm_forward_bf16(const Params& p, const void* X, const void* Wq, void* Y, cudaStream_t st, int* n) {
-  *n = 0;
+inline l4q_status gemm_forward_bf16(const Params& p, const void* X, const void* Wq, void* Y, cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, X, p.tokens, p.d_in, BM) || !make_tmap_bf16(&tb, Wq, p.d_out, p.d_in, BN))
     return L4Q_ERR_CUDA;
   GemmArgs g{};
   g.M = p.tokens; g.N = p.d_out; g.K = p.d_in;
   g.C = reinterpret_cast<__nv_bfloat16*>(Y);
-  *n = 1;
   return launch_gemm<false, false, EPI_STORE, 0, 4>(ta, tb, g, st);
 }
 
 // dX[tokens, d_in] = dY[tokens, d_out] Wq[d_out, d_in]
-inline l4q_status gemm_dgrad_bf16(const Params& p, const void* dY, const void* Wq, void* dX, cudaStream_t st, int* n) {
-  *n = 0;
+inline l4q_status gemm_dgrad_bf16(const Params& p, const void* dY, const void* Wq, void* dX, cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BM) || !make_tmap_bf16(&tb, Wq, p.d_out, p.d_in, BK))
     return L4Q_ERR_CUDA;
   GemmArgs g{};
   g.M = p.tokens; g.N = p.d_in; g.K = p.d_out;
   g.C = reinterpret_cast<__nv_bfloat16*>(dX);
-  *n = 1;
   return launch_gemm<false, true, EPI_STORE, 0, 4>(ta, tb, g, st);
 }
 
 // G[d_out, d_in] = dY^T X reduced on chip into dA, dB, ds, db (which must be zero on entry).
 inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY, const void* W0, const float* A,
                                   const float* B, const float* s, const float* b, float* dA, float* dB, float* ds,
-                                  float* db, cudaStream_t st, int* n) {
-  *n = 0;
+                                  float* db, cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BK) || !make_tmap_bf16(&tb, X, p.tokens, p.d_in, BK))
     return L4Q_ERR_CUDA;
@@ -515,13 +510,12 @@ inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY
   g.W0 = reinterpret_cast<const __nv_bfloat16*>(W0);
   g.A = A; g.B = B; g.s = s; g.b = b;
   g.dA = dA; g.dB = dB; g.ds = ds; g.db = db;
-  *n = 1;
   switch (p.rank) {
     case 8: return launch_gemm<true, true, EPI_WGRAD, 8, 3>(ta, tb, g, st);
     case 16: return launch_gemm<true, true, EPI_WGRAD, 16, 3>(ta, tb, g, st);
     case 32: return launch_gemm<true, true, EPI_WGRAD, 32, 3>(ta, tb, g, st);
     case 64: return launch_gemm<true, true, EPI_WGRAD, 64, 3>(ta, tb, g, st);
-    default: *n = 0; return L4Q_ERR_UNSUPPORTED;
+    default: return L4Q_ERR_UNSUPPORTED;
   }
 }
 

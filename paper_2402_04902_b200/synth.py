@@ -139,6 +139,14 @@ def group_minmax_init(W0: np.ndarray, bits: int, group_size: int, signed_grid: b
     return s, b
 
 
+def make_layer_acts(cfg: LayerConfig, seed: int = 0, layer_id: int = 0) -> dict:
+    """X and dY of one layer only (same streams as :func:`make_layer_inputs`)."""
+    o, i, M = cfg.d_out, cfg.d_in, cfg.tokens
+    base = 16 * layer_id
+    return {"X": _narrow(normal(seed, base + _S_X, M * i), cfg.io_dtype).reshape(M, i),
+            "dY": _narrow(normal(seed, base + _S_DY, M * o), cfg.io_dtype).reshape(M, o)}
+
+
 def make_layer_inputs(cfg: LayerConfig, seed: int = 0, layer_id: int = 0,
                       zero_B: bool = False, need_acts: bool = True) -> dict:
     """All tensors of one layer, as float32 numpy arrays holding values that
@@ -160,8 +168,7 @@ def make_layer_inputs(cfg: LayerConfig, seed: int = 0, layer_id: int = 0,
     s, b = group_minmax_init(W0, cfg.bits, cfg.group_size, cfg.signed_grid)
     out = {"W0": W0, "A": A, "B": B, "s": s, "b": b}
     if need_acts:
-        out["X"] = _narrow(normal(seed, base + _S_X, M * i), cfg.io_dtype).reshape(M, i)
-        out["dY"] = _narrow(normal(seed, base + _S_DY, M * o), cfg.io_dtype).reshape(M, o)
+        out.update(make_layer_acts(cfg, seed, layer_id))
     return out
 
 
