@@ -126,6 +126,40 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
                         uint32_t* codes, uint16_t* s_fp16, uint16_t* b_fp16,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * Forward pass for callers that cannot hand the library any scratch memory.
+ * (The paper has no counterpart; this entry point exists for integration only.)
+ *
+ * Same inputs, output and arithmetic as l4q_linear_fwd, but without the
+ * workspace arguments: the dequantized weight goes into a fixed array of
+ * L4Q_STATIC_SCRATCH_BYTES that is part of the library's device image.  It is
+ * meant for code that runs where device allocation is off limits: a plug-in or
+ * custom op inside a runtime whose own allocator has already claimed the
+ * device's free memory, a latency-critical loop that must not hit the implicit
+ * device-wide synchronisation of cudaMalloc/cudaFree, or a process that is
+ * held to a fixed memory budget decided at start-up.  The call performs no
+ * cudaMalloc, cudaFree or other allocating call.
+ *
+ *   - Limit: d_out * d_in * sizeof(io_dtype), rounded up to 256 bytes, must not
+ *     exceed L4Q_STATIC_SCRATCH_BYTES (32 MiB: a 4096 x 4096 bf16 weight).
+ *     Larger problems return L4Q_ERR_WORKSPACE and launch nothing; use
+ *     l4q_linear_fwd with a caller-owned workspace for those.
+ *   - Cost: every GPU on which this library is loaded keeps the 32 MiB reserved
+ *     until the process exits, whether or not this function is ever called.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and remembers it; make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last
+ *     call left in it.  Nothing in it needs to start at zero (each call
+ *     rewrites the whole region it later reads), but two calls whose kernels
+ *     can overlap on the GPU (different streams, or different host threads
+ *     without ordering) race on it: order them on one stream or with events.
+ */
+#define L4Q_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+l4q_status l4q_linear_fwd_static(const l4q_desc* desc, const void* X, const void* W0,
+                                 const float* A, const float* B, const float* s, const float* b,
+                                 void* Y, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the device status word
  * (L4Q_OK, or L4Q_ERR_TIMEOUT if a kernel gave up on a bounded wait), or
  * L4Q_ERR_CUDA if the stream reported an error. */

@@ -27,7 +27,10 @@ EXPORTED_SYMBOLS = (
     "l4q_workspace_bytes", "l4q_linear_fwd", "l4q_linear_bwd", "l4q_pack_int",
     "l4q_check", "l4q_launch_count", "l4q_status_string",
     "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
+    "l4q_linear_fwd_static",
 )
+
+L4Q_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 KERNEL_IDS = {"dequant": 0, "pack": 1, "gemm_fwd": 2, "gemm_dgrad": 3, "gemm_wgrad": 4, "val_gemm": 5,
               "val_wgrad": 6}
@@ -68,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.l4q_workspace_bytes.argtypes = [dp, ctypes.c_int]
         L.l4q_linear_fwd.restype = ctypes.c_int
         L.l4q_linear_fwd.argtypes = [dp, vp, vp, fp, fp, fp, fp, vp, vp, sz, vp]
+        L.l4q_linear_fwd_static.restype = ctypes.c_int
+        L.l4q_linear_fwd_static.argtypes = [dp, vp, vp, fp, fp, fp, fp, vp, vp]
         L.l4q_linear_bwd.restype = ctypes.c_int
         L.l4q_linear_bwd.argtypes = [dp, vp, vp, vp, fp, fp, fp, fp, vp, fp, fp, fp, fp, vp, sz, vp]
         L.l4q_pack_int.restype = ctypes.c_int
@@ -130,6 +135,15 @@ def l4q_linear_fwd(desc: L4QDesc, X, W0, A, B, s, b, Y, workspace, stream=None) 
     st = lib().l4q_linear_fwd(ctypes.byref(desc), _ptr(X), _ptr(W0), _ptr(A), _ptr(B), _ptr(s), _ptr(b), _ptr(Y),
                               _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream))
     _raise(st, "l4q_linear_fwd")
+
+
+def l4q_linear_fwd_static(desc: L4QDesc, X, W0, A, B, s, b, Y, stream=None) -> None:
+    """Forward without a workspace: for callers that may not allocate device memory
+    (the scratch is a fixed 32 MiB array inside the library; see include/l4q.h for
+    the size limit and the sharing rules)."""
+    st = lib().l4q_linear_fwd_static(ctypes.byref(desc), _ptr(X), _ptr(W0), _ptr(A), _ptr(B), _ptr(s), _ptr(b),
+                                     _ptr(Y), _stream(stream))
+    _raise(st, "l4q_linear_fwd_static")
 
 
 def l4q_linear_bwd(desc: L4QDesc, X, dY, W0, A, B, s, b, dX, dA, dB, ds, db, workspace, stream=None) -> None:

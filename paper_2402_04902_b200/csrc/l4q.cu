@@ -260,6 +260,68 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
                                     : launch_pack<false>(p, W0, A, B, s, b, codes, s16, b16, stream);
 }
 
+// ---- forward without caller-provided scratch --------------------------------------------------
+// Scratch for the dequantized weight of l4q_linear_fwd_static.  Lives in the library image: every
+// device that loads the library reserves these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_fwd_static_scratch[L4Q_STATIC_SCRATCH_BYTES];
+
+// Never launched; naming the array in device code keeps the symbol in the device image.
+__global__ void k_static_scratch_anchor(unsigned char* out) {
+  if (out) *out = g_fwd_static_scratch[0];
+}
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices];   // device address of g_fwd_static_scratch, per device; null until set up
+
+// In host code `g_fwd_static_scratch` is only a handle for the runtime, not an address a kernel can
+// use.  The device address is looked up once per device, with that device current.
+l4q_status static_scratch_for_current_device(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return L4Q_ERR_CUDA;
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_fwd_static_scratch) != cudaSuccess || !ptr) return L4Q_ERR_CUDA;
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return L4Q_OK;
+}
+}  // namespace
+
+l4q_status l4q_linear_fwd_static(const l4q_desc* desc, const void* X, const void* W0, const float* A, const float* B,
+                                 const float* s, const float* b, void* Y, void* cuda_stream) {
+  Params p;
+  l4q_status st = make_params(desc, &p);
+  if (st != L4Q_OK) return st;
+  if (!X || !W0 || !A || !B || !s || !b || !Y) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W0) || !aligned16(A) || !aligned16(B) || !aligned16(Y)) return L4Q_ERR_INVALID_ARG;
+  if (wq_scratch_bytes(desc) > (size_t)L4Q_STATIC_SCRATCH_BYTES) return L4Q_ERR_WORKSPACE;   // weight too large
+  void* wq = nullptr;
+  if ((st = static_scratch_for_current_device(&wq)) != L4Q_OK) return st;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  // The whole d_out x d_in region that the GEMM reads is rewritten by the dequantize kernel first,
+  // so nothing left in the array by an earlier call is ever read.
+  if (desc->io_dtype == L4Q_F32) {
+    st = launch_dequant<false>(p, W0, A, B, s, b, wq, stream);
+    if (st != L4Q_OK) return st;
+    GemmView g;
+    g.A = reinterpret_cast<const float*>(X); g.a_m = p.d_in; g.a_k = 1;
+    g.B = reinterpret_cast<const float*>(wq); g.b_k = 1; g.b_n = p.d_in;
+    g.M = p.tokens; g.N = p.d_out; g.K = p.d_in;
+    dim3 grid(ceil_div(g.N, VT), ceil_div(g.M, VT));
+    KernelScope ks(L4Q_KERNEL_VAL_GEMM, stream);
+    k_val_gemm<<<grid, V_THREADS, 0, stream>>>(g, reinterpret_cast<float*>(Y));
+    return launch_status();
+  }
+  st = launch_dequant<true>(p, W0, A, B, s, b, wq, stream);
+  if (st != L4Q_OK) return st;
+  KernelScope ks(L4Q_KERNEL_GEMM_FWD, stream);
+  return gemm_forward_bf16(p, X, wq, Y, stream);
+}
+
 l4q_status l4q_check(void* cuda_stream) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (cudaStreamSynchronize(stream) != cudaSuccess) return L4Q_ERR_CUDA;
