@@ -63,9 +63,8 @@ struct __align__(8) GemmBarriers {
   volatile uint32_t abort;
 };
 
-inline size_t gemm_smem_bytes(int stages, int epi) {
-  return 1024 /*alignment slack*/ + (size_t)stages * STAGE_BYTES + (epi == EPI_WGRAD ? STG_BYTES : 0) +
-         sizeof(GemmBarriers);
+inline size_t gemm_smem_bytes(int stages, int epi_bytes) {
+  return 1024 /*alignment slack*/ + (size_t)stages * STAGE_BYTES + (size_t)epi_bytes + sizeof(GemmBarriers);
 }
 
 // Bounded mbarrier wait.  Returns immediately once the CTA's abort flag is set.
@@ -98,15 +97,73 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
   tn = in_band / rows;
 }
 
+// Shared memory of the wgrad epilogue (after the pipeline stages):
+//   stg [2 groups][128 rows][33]  Gm chunk, transposed access for the dA column sums
+//   Bs  [128 rows][RANK]          the tile's rows of B (zero beyond d_out)
+//   As  [2 groups][RANK][32]      the current 32-column chunk of A, one copy per epilogue group
+__host__ __device__ constexpr int wgrad_epi_smem_bytes(int rank) {
+  return STG_BYTES + 128 * rank * 4 + EPI_GROUPS * rank * 32 * 4;
+}
+
+// Loads this thread's share of A[:, jc : jc+32] (RANK x 32 floats = RANK*8 float4 over 128 threads).
+template <int RANK>
+__device__ __forceinline__ void load_a_chunk(const GemmArgs& g, int jc, int t, float4 (&regs)[(RANK * 8 + 127) / 128]) {
+#pragma unroll
+  for (int u = 0; u < (RANK * 8 + 127) / 128; ++u) {
+    const int f = t + u * 128;
+    const int k = f >> 3, v = f & 7;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (f < RANK * 8 && jc + v * 4 < g.p.d_in) a = __ldg(reinterpret_cast<const float4*>(g.A + (size_t)k * g.p.d_in + jc + v * 4));
+    regs[u] = a;
+  }
+}
+template <int RANK>
+__device__ __forceinline__ void store_a_chunk(float* As_g, int t, const float4 (&regs)[(RANK * 8 + 127) / 128]) {
+#pragma unroll
+  for (int u = 0; u < (RANK * 8 + 127) / 128; ++u) {
+    const int f = t + u * 128;
+    if (f < RANK * 8) reinterpret_cast<float4*>(As_g)[f] = regs[u];      // As_g[k][v*4..] with f = k*8 + v
+  }
+}
+
+// One 128 x 256 tile of G = dY^T X, read from tensor memory and reduced into ds, db, dA, dB.
+// Thread = one weight row (TMEM lane) of one epilogue group; the group owns 4 chunks of 32 columns.
+// Everything that does not depend on the accumulator (B rows, the first A chunk) is fetched before
+// waiting for the MMAs; W0, s, b and the next A chunk are fetched ahead of the arithmetic that
+// precedes their use, so that the loads' latency hides behind the FMA loops.
 template <int RANK>
 __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, int n0, uint32_t tmem_acc, int quarter,
-                                                    int lane, int eg, float* stg, uint64_t* tmem_empty_bar) {
+                                                    int lane, int eg, float* epi_smem, GemmBarriers* bars,
+                                                    uint64_t* tmem_full_bar, uint32_t full_parity,
+                                                    uint64_t* tmem_empty_bar) {
   const Params& p = g.p;
-  const int row_in_tile = quarter * 32 + lane;
-  const int o = m0 + row_in_tile;
+  float* stg_g = epi_smem + (size_t)eg * 128 * STG_LD;
+  float* Bs = epi_smem + EPI_GROUPS * 128 * STG_LD;
+  float* As_g = Bs + 128 * RANK + (size_t)eg * RANK * 32;
+  const int t = quarter * 32 + lane;                   // row in tile = thread index within the group
+  const int t256 = eg * 128 + t;
+  const int o = m0 + t;
   const bool row_ok = o < p.d_out;
-  const int t_in_group = row_in_tile;                 // 0..127 within the epilogue group
+  constexpr int CHUNKS_PER_GROUP = (BN / 32) / EPI_GROUPS;
+  constexpr int A_REGS = (RANK * 8 + 127) / 128;
 
+  // ---- before the accumulator is ready ----
+  ptx::named_bar_sync(3, EPI_THREADS);                 // both groups are done with the previous tile's Bs
+#pragma unroll
+  for (int u = 0; u < (32 * RANK + EPI_THREADS - 1) / EPI_THREADS; ++u) {
+    const int f = t256 + u * EPI_THREADS;              // float4 index into Bs
+    if (f < 32 * RANK) {
+      const int row = f / (RANK / 4), kq = f % (RANK / 4);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (m0 + row < p.d_out) v = __ldg(reinterpret_cast<const float4*>(g.B + (size_t)(m0 + row) * RANK + kq * 4));
+      reinterpret_cast<float4*>(Bs)[f] = v;
+    }
+  }
+  {
+    float4 a0[A_REGS];
+    load_a_chunk<RANK>(g, n0 + eg * CHUNKS_PER_GROUP * 32, t, a0);
+    store_a_chunk<RANK>(As_g, t, a0);
+  }
   float brow[RANK];
 #pragma unroll
   for (int k = 0; k < RANK; k += 4) {
@@ -117,18 +174,39 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
   float dBacc[RANK];
 #pragma unroll
   for (int k = 0; k < RANK; ++k) dBacc[k] = 0.f;
+  ptx::named_bar_sync(3, EPI_THREADS);                 // Bs and the first A chunk are visible
+
+  bounded_wait(tmem_full_bar, full_parity, bars);
+  ptx::tc_fence_after_sync();
 
   float ds_acc = 0.f, db_acc = 0.f;
   int cur_grp = -1;
-  constexpr int CHUNKS_PER_GROUP = (BN / 32) / EPI_GROUPS;
 
+#pragma unroll 1
   for (int cc = 0; cc < CHUNKS_PER_GROUP; ++cc) {
     const int c = eg * CHUNKS_PER_GROUP + cc;
-    const int jc = n0 + c * 32;                       // first column of the chunk
+    const int jc = n0 + c * 32;                        // first column of the chunk
+
+    // loads issued ahead of their use
+    uint4 wraw[4];
+    float sv[4], bv[4];
+    int grp[4];
+#pragma unroll
+    for (int sub = 0; sub < 4; ++sub) {
+      const int j = jc + sub * 8;
+      const bool ok = row_ok && j < p.d_in;
+      grp[sub] = ok ? j / p.group : -1;
+      wraw[sub] = ok ? __ldg(reinterpret_cast<const uint4*>(g.W0 + (size_t)o * p.d_in + j)) : make_uint4(0, 0, 0, 0);
+      sv[sub] = ok ? __ldg(g.s + (size_t)o * p.ngroups + grp[sub]) : 1.f;
+      bv[sub] = ok ? __ldg(g.b + (size_t)o * p.ngroups + grp[sub]) : 0.f;
+    }
+    float4 a_next[A_REGS];
+    if (cc + 1 < CHUNKS_PER_GROUP) load_a_chunk<RANK>(g, jc + 32, t, a_next);
+
     uint32_t raw[32];
     ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), raw);
     ptx::tmem_ld_wait();
-    if (cc == CHUNKS_PER_GROUP - 1) {                 // accumulator stage fully read by this thread
+    if (cc == CHUNKS_PER_GROUP - 1) {                  // accumulator stage fully read by this thread
       ptx::tc_fence_before_sync();
       ptx::mbar_arrive(tmem_empty_bar);
     }
@@ -142,11 +220,10 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
     for (int e = 0; e < 32; ++e) acc[e] = 0.f;
 #pragma unroll
     for (int k = 0; k < RANK; ++k) {
-      const float* arow = g.A + (size_t)k * p.d_in + jc;
+      const float4* arow = reinterpret_cast<const float4*>(As_g + k * 32);
 #pragma unroll
       for (int v = 0; v < 8; ++v) {
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (jc + v * 4 < p.d_in) a = __ldg(reinterpret_cast<const float4*>(arow + v * 4));
+        const float4 a = arow[v];
         acc[v * 4 + 0] = fmaf(brow[k], a.x, acc[v * 4 + 0]);
         acc[v * 4 + 1] = fmaf(brow[k], a.y, acc[v * 4 + 1]);
         acc[v * 4 + 2] = fmaf(brow[k], a.z, acc[v * 4 + 2]);
@@ -157,26 +234,22 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
     // quantizer state, STE gate, ds / db partial sums                           (Eq. 8, 5, 6)
 #pragma unroll
     for (int sub = 0; sub < 4; ++sub) {
-      const int j = jc + sub * 8;
-      if (row_ok && j < p.d_in) {
-        const int grp = j / p.group;
-        if (grp != cur_grp) {
+      if (grp[sub] >= 0) {
+        if (grp[sub] != cur_grp) {
           if (cur_grp >= 0) {
             atomicAdd(&g.ds[(size_t)o * p.ngroups + cur_grp], p.grad_scale * ds_acc);
             atomicAdd(&g.db[(size_t)o * p.ngroups + cur_grp], p.grad_scale * db_acc);
           }
-          cur_grp = grp; ds_acc = 0.f; db_acc = 0.f;
+          cur_grp = grp[sub]; ds_acc = 0.f; db_acc = 0.f;
         }
-        const float sv = __ldg(g.s + (size_t)o * p.ngroups + grp);
-        const float bv = __ldg(g.b + (size_t)o * p.ngroups + grp);
-        const float rs = 1.0f / sv;
-        const uint4 wraw = __ldg(reinterpret_cast<const uint4*>(g.W0 + (size_t)o * p.d_in + j));
-        const float w0[8] = {bf16_lo(wraw.x), bf16_hi(wraw.x), bf16_lo(wraw.y), bf16_hi(wraw.y),
-                             bf16_lo(wraw.z), bf16_hi(wraw.z), bf16_lo(wraw.w), bf16_hi(wraw.w)};
+        const float rs = 1.0f / sv[sub];
+        const uint4 wr = wraw[sub];
+        const float w0[8] = {bf16_lo(wr.x), bf16_hi(wr.x), bf16_lo(wr.y), bf16_hi(wr.y),
+                             bf16_lo(wr.z), bf16_hi(wr.z), bf16_lo(wr.w), bf16_hi(wr.w)};
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const int idx = sub * 8 + e;
-          const QuantElem q = quantize_elem(merge_elem(w0[e], acc[idx], p.gamma), sv, rs, bv, p.qn, p.qp);
+          const QuantElem q = quantize_elem(merge_elem(w0[e], acc[idx], p.gamma), sv[sub], rs, bv[sub], p.qn, p.qp);
           const float Gv = G[idx];
           if (ste_in_range(q.w, p.qn, p.qp)) {
             ds_acc = fmaf(Gv, q.code - q.w, ds_acc);
@@ -195,43 +268,45 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
     // dB[o,k] += sum_e Gm[e] A[k, jc+e]                                         (Eq. 14)
 #pragma unroll
     for (int k = 0; k < RANK; ++k) {
-      const float* arow = g.A + (size_t)k * p.d_in + jc;
-      float part = 0.f;
+      const float4* arow = reinterpret_cast<const float4*>(As_g + k * 32);
+      float part0 = 0.f, part1 = 0.f;
 #pragma unroll
-      for (int v = 0; v < 8; ++v) {
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (jc + v * 4 < p.d_in) a = __ldg(reinterpret_cast<const float4*>(arow + v * 4));
-        part = fmaf(G[v * 4 + 0], a.x, part);
-        part = fmaf(G[v * 4 + 1], a.y, part);
-        part = fmaf(G[v * 4 + 2], a.z, part);
-        part = fmaf(G[v * 4 + 3], a.w, part);
+      for (int v = 0; v < 8; v += 2) {
+        const float4 a = arow[v], a2 = arow[v + 1];
+        part0 = fmaf(G[v * 4 + 0], a.x, part0);
+        part0 = fmaf(G[v * 4 + 1], a.y, part0);
+        part0 = fmaf(G[v * 4 + 2], a.z, part0);
+        part0 = fmaf(G[v * 4 + 3], a.w, part0);
+        part1 = fmaf(G[v * 4 + 4], a2.x, part1);
+        part1 = fmaf(G[v * 4 + 5], a2.y, part1);
+        part1 = fmaf(G[v * 4 + 6], a2.z, part1);
+        part1 = fmaf(G[v * 4 + 7], a2.w, part1);
       }
-      dBacc[k] += part;
+      dBacc[k] += part0 + part1;
     }
 
     // dA[k, jc+col] += sum_rows B[o,k] Gm[o, col]: transpose through shared memory   (Eq. 13)
-    float* my_stg = stg + (size_t)eg * 128 * STG_LD;
 #pragma unroll
-    for (int e = 0; e < 32; ++e) my_stg[row_in_tile * STG_LD + e] = G[e];
-    ptx::named_bar_sync(1 + eg, 128);
+    for (int e = 0; e < 32; ++e) stg_g[t * STG_LD + e] = G[e];
+    ptx::named_bar_sync(1 + eg, 128);                  // Gm chunk visible; everyone is past the reads of As_g
+    if (cc + 1 < CHUNKS_PER_GROUP) store_a_chunk<RANK>(As_g, t, a_next);
     {
-      const int col = t_in_group & 31, rq = t_in_group >> 5;
+      const int col = t & 31, rq = t >> 5;
       float acc_a[RANK];
 #pragma unroll
       for (int k = 0; k < RANK; ++k) acc_a[k] = 0.f;
+#pragma unroll 4
       for (int rr = 0; rr < 32; ++rr) {
         const int r2 = rq * 32 + rr;
-        const int o2 = m0 + r2;
-        if (o2 >= p.d_out) break;                     // uniform across the warp
-        const float gm = my_stg[r2 * STG_LD + col];
-        const float4* b4 = reinterpret_cast<const float4*>(g.B + (size_t)o2 * RANK);
+        const float gm = stg_g[r2 * STG_LD + col];
+        const float4* b4 = reinterpret_cast<const float4*>(Bs + r2 * RANK);
 #pragma unroll
         for (int k = 0; k < RANK; k += 4) {
-          const float4 bv = __ldg(b4 + (k >> 2));
-          acc_a[k] = fmaf(bv.x, gm, acc_a[k]);
-          acc_a[k + 1] = fmaf(bv.y, gm, acc_a[k + 1]);
-          acc_a[k + 2] = fmaf(bv.z, gm, acc_a[k + 2]);
-          acc_a[k + 3] = fmaf(bv.w, gm, acc_a[k + 3]);
+          const float4 bq = b4[k >> 2];
+          acc_a[k] = fmaf(bq.x, gm, acc_a[k]);
+          acc_a[k + 1] = fmaf(bq.y, gm, acc_a[k + 1]);
+          acc_a[k + 2] = fmaf(bq.z, gm, acc_a[k + 2]);
+          acc_a[k + 3] = fmaf(bq.w, gm, acc_a[k + 3]);
         }
       }
       const int ja = jc + col;
@@ -240,7 +315,7 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
         for (int k = 0; k < RANK; ++k) atomicAdd(&g.dA[(size_t)k * p.d_in + ja], p.gamma * acc_a[k]);
       }
     }
-    ptx::named_bar_sync(1 + eg, 128);
+    ptx::named_bar_sync(1 + eg, 128);                  // staging tile reusable, next A chunk visible
   }
 
   if (row_ok) {
@@ -259,9 +334,9 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
-  float* stg = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES);
-  GemmBarriers* bars =
-      reinterpret_cast<GemmBarriers*>(smem + (size_t)STAGES * STAGE_BYTES + (EPI == EPI_WGRAD ? STG_BYTES : 0));
+  constexpr int EPI_SMEM = (EPI == EPI_WGRAD) ? wgrad_epi_smem_bytes(RANK) : 0;
+  float* epi_smem = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES);
+  GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + (size_t)STAGES * STAGE_BYTES + EPI_SMEM);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = g.tiles_m * g.tiles_n;
@@ -365,10 +440,10 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int tm, tn;
       tile_coords(t, g.tiles_m, g.tiles_n, tm, tn);
       const int m0 = tm * BM, n0 = tn * BN;
-      bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
-      ptx::tc_fence_after_sync();
       const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
       if constexpr (EPI == EPI_STORE) {
+        bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
+        ptx::tc_fence_after_sync();
         const int row = m0 + quarter * 32 + lane;
         constexpr int CHUNKS_PER_GROUP = (BN / 32) / EPI_GROUPS;
 #pragma unroll 1
@@ -397,7 +472,8 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
         }
       } else {
-        wgrad_epilogue_tile<RANK>(g, m0, n0, tmem_acc, quarter, lane, eg, stg, &bars->tmem_empty[acc]);
+        wgrad_epilogue_tile<RANK>(g, m0, n0, tmem_acc, quarter, lane, eg, epi_smem, bars, &bars->tmem_full[acc],
+                                  acc_phase, &bars->tmem_empty[acc]);
       }
       if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1; }
     }
@@ -467,7 +543,7 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
   g.tiles_n = ceil_div(g.N, BN);
   g.num_kb = ceil_div(g.K, BK);
   auto kern = k_gemm_bf16<A_MN, B_MN, EPI, RANK, STAGES>;
-  const size_t smem = gemm_smem_bytes(STAGES, EPI);
+  const size_t smem = gemm_smem_bytes(STAGES, EPI == EPI_WGRAD ? wgrad_epi_smem_bytes(RANK) : 0);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return L4Q_ERR_CUDA;
   const int grid = std::min(g.tiles_m * g.tiles_n, sm_count());
