@@ -97,12 +97,17 @@ size_t wq_scratch_bytes(const l4q_desc* d) {
   return align_up((size_t)d->d_out * (size_t)d->d_in * esz, 256);
 }
 
+size_t factor_scratch_bytes(const l4q_desc* d) {
+  return align_up((size_t)d->d_out * (size_t)d->d_in * sizeof(__half), 256);
+}
+
 inline l4q_status launch_status() { return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA; }
 
 // Merge + fake-quantize the whole weight into `wq` (io dtype) -- the recompute step of fwd and bwd.
+// `fac` (optional, bf16 mode only) also receives the fp16 STE factors the weight-gradient kernel reads.
 template <bool IO_BF16>
 l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const float* B, const float* s,
-                          const float* b, void* wq, cudaStream_t st) {
+                          const float* b, void* wq, __half* fac, cudaStream_t st) {
   const size_t smem = weight_tile_smem_bytes(p.rank);
   auto kern = k_weight_tile<IO_BF16, WT_MODE_DEQUANT>;
   if (smem > 48 * 1024 &&
@@ -110,7 +115,7 @@ l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const
     return L4Q_ERR_CUDA;
   dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
   KernelScope ks(L4Q_KERNEL_DEQUANT, st);
-  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, wq, nullptr, nullptr, nullptr);
+  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, wq, fac, nullptr, nullptr, nullptr);
   return launch_status();
 }
 
@@ -124,7 +129,7 @@ l4q_status launch_pack(const Params& p, const void* W0, const float* A, const fl
     return L4Q_ERR_CUDA;
   dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
   KernelScope ks(L4Q_KERNEL_PACK, st);
-  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, nullptr, codes, s16, b16);
+  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, nullptr, nullptr, codes, s16, b16);
   return launch_status();
 }
 
@@ -137,8 +142,9 @@ size_t l4q_workspace_bytes(const l4q_desc* desc, int op) {
   if (make_params(desc, &p) != L4Q_OK) return 0;
   switch (op) {
     case L4Q_OP_FWD:
-    case L4Q_OP_BWD:
       return wq_scratch_bytes(desc) + 256;
+    case L4Q_OP_BWD:   // W_q for the input gradient, and in bf16 mode the fp16 STE factors for the weight gradient
+      return wq_scratch_bytes(desc) + (desc->io_dtype == L4Q_BF16 ? factor_scratch_bytes(desc) : 0) + 256;
     case L4Q_OP_PACK:
     default:
       return 0;
@@ -159,7 +165,7 @@ l4q_status l4q_linear_fwd(const l4q_desc* desc, const void* X, const void* W0, c
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   void* wq = workspace;
   if (desc->io_dtype == L4Q_F32) {
-    st = launch_dequant<false>(p, W0, A, B, s, b, wq, stream);
+    st = launch_dequant<false>(p, W0, A, B, s, b, wq, nullptr, stream);
     if (st != L4Q_OK) return st;
     GemmView g;
     g.A = reinterpret_cast<const float*>(X); g.a_m = p.d_in; g.a_k = 1;
@@ -170,7 +176,7 @@ l4q_status l4q_linear_fwd(const l4q_desc* desc, const void* X, const void* W0, c
     k_val_gemm<<<grid, V_THREADS, 0, stream>>>(g, reinterpret_cast<float*>(Y));
     return launch_status();
   }
-  st = launch_dequant<true>(p, W0, A, B, s, b, wq, stream);
+  st = launch_dequant<true>(p, W0, A, B, s, b, wq, nullptr, stream);
   if (st != L4Q_OK) return st;
   KernelScope ks(L4Q_KERNEL_GEMM_FWD, stream);
   return gemm_forward_bf16(p, X, wq, Y, stream);
@@ -203,9 +209,13 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
         cudaMemsetAsync(ds, 0, gsz, stream) != cudaSuccess || cudaMemsetAsync(db, 0, gsz, stream) != cudaSuccess)
       return L4Q_ERR_CUDA;
   }
-  if (dX) {
-    st = f32 ? launch_dequant<false>(p, W0, A, B, s, b, wq, stream)
-             : launch_dequant<true>(p, W0, A, B, s, b, wq, stream);
+  // recompute step (App. E.2): W_q for dX and, on the tensor-core path, the STE factors for the weight gradient
+  __half* fac = (!f32 && n_param_out == 4)
+                    ? reinterpret_cast<__half*>(static_cast<unsigned char*>(workspace) + wq_scratch_bytes(desc))
+                    : nullptr;
+  if (dX || fac) {
+    st = f32 ? launch_dequant<false>(p, W0, A, B, s, b, wq, nullptr, stream)
+             : launch_dequant<true>(p, W0, A, B, s, b, wq, fac, stream);
     if (st != L4Q_OK) return st;
   }
   if (f32) {
@@ -236,7 +246,7 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
   }
   if (n_param_out == 4) {
     KernelScope ks(L4Q_KERNEL_GEMM_WGRAD, stream);
-    st = gemm_wgrad_bf16(p, X, dY, W0, A, B, s, b, dA, dB, ds, db, stream);
+    st = gemm_wgrad_bf16(p, X, dY, fac, A, B, dA, dB, ds, db, stream);
     if (st != L4Q_OK) return st;
   }
   return L4Q_OK;
@@ -305,7 +315,7 @@ l4q_status l4q_linear_fwd_static(const l4q_desc* desc, const void* X, const void
   // The whole d_out x d_in region that the GEMM reads is rewritten by the dequantize kernel first,
   // so nothing left in the array by an earlier call is ever read.
   if (desc->io_dtype == L4Q_F32) {
-    st = launch_dequant<false>(p, W0, A, B, s, b, wq, stream);
+    st = launch_dequant<false>(p, W0, A, B, s, b, wq, nullptr, stream);
     if (st != L4Q_OK) return st;
     GemmView g;
     g.A = reinterpret_cast<const float*>(X); g.a_m = p.d_in; g.a_k = 1;
@@ -316,7 +326,7 @@ l4q_status l4q_linear_fwd_static(const l4q_desc* desc, const void* X, const void
     k_val_gemm<<<grid, V_THREADS, 0, stream>>>(g, reinterpret_cast<float*>(Y));
     return launch_status();
   }
-  st = launch_dequant<true>(p, W0, A, B, s, b, wq, stream);
+  st = launch_dequant<true>(p, W0, A, B, s, b, wq, nullptr, stream);
   if (st != L4Q_OK) return st;
   KernelScope ks(L4Q_KERNEL_GEMM_FWD, stream);
   return gemm_forward_bf16(p, X, wq, Y, stream);

@@ -49,6 +49,18 @@ __device__ __forceinline__ bool ste_in_range(float w, float qn, float qp) {
   return (w >= qn - kMaskGuard) && (w <= qp + kMaskGuard);
 }
 
+// What the weight-gradient reduction needs to know about one weight besides G, in one number
+// (App. A.1): where the STE passes the gradient (Q_N <= w <= Q_P) it is dW_q/ds = w~ - w, a
+// value in [-1/2, 1/2]; where w was clamped it is a sentinel, -2 below Q_N and +2 above Q_P
+// (there dW_q/ds = Q_N or Q_P and dW_q/db = 1).  Stored as fp16 between the two kernels of the
+// backward pass.
+constexpr float kSteBelow = -2.f, kSteAbove = 2.f;
+
+__device__ __forceinline__ float ste_factor(const QuantElem& q, float qn, float qp) {
+  if (ste_in_range(q.w, qn, qp)) return q.code - q.w;
+  return q.w < qn ? kSteBelow : kSteAbove;
+}
+
 // W_comb = W0 + gamma * acc, acc = sum_k B[o,k] A[k,j]      (Eq. 7)
 __device__ __forceinline__ float merge_elem(float w0, float acc, float gamma) { return fmaf(gamma, acc, w0); }
 

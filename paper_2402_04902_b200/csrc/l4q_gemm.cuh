@@ -7,8 +7,12 @@
 //   wgrad     G  = dY^T X    A = dY (MN-major),  B = X  (MN-major),  K = tokens   (Eq. 11)
 //
 // The wgrad epilogue never writes G: each 128 x 256 tile of G is reduced from
-// tensor memory into ds, db (Eq. 5-6), dA and dB (Eq. 13-14), recomputing the
-// quantizer state of the tile's weights from W0, A, B, s, b (App. E.2).
+// tensor memory into ds, db (Eq. 5-6), dA and dB (Eq. 13-14).  The quantizer
+// state of the tile's weights (STE gate and dW_q/ds) is recomputed in the same
+// backward call by the weight-tile kernel (App. E.2) and read here as one fp16
+// factor per weight; the contractions with the LoRA factors that give dA and dB
+// are two more tcgen05 MMAs per 128 columns, fed from a bf16 copy of G * m in
+// shared memory.
 //
 // Roles (384 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
 // owner, warps 4..11 = two epilogue groups of 128 threads (each group drains
@@ -38,8 +42,6 @@ constexpr int EPI_GROUPS = 2;
 constexpr int EPI_THREADS = EPI_GROUPS * 128;
 constexpr int ACC_STAGES = 2;
 constexpr int TMEM_COLS = ACC_STAGES * BN;   // 512: all of tensor memory
-constexpr int STG_LD = 33;                   // padded row length of the wgrad staging tile
-constexpr int STG_BYTES = EPI_GROUPS * 128 * STG_LD * 4;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s at B200 clocks
 
 enum { EPI_STORE = 0, EPI_WGRAD = 1 };
@@ -51,14 +53,15 @@ struct GemmArgs {
   __nv_bfloat16* C;            // [M, N] row-major
   // EPI_WGRAD (M = d_out, N = d_in)
   Params p;
-  const __nv_bfloat16* W0;
-  const float *A, *B, *s, *b;
+  const __half* F;             // [d_out, d_in] STE factors of the weights (ste_factor)
+  const float *A, *B;
   float *dA, *dB, *ds, *db;
 };
 
 struct __align__(8) GemmBarriers {
   uint64_t full[8], empty[8];
   uint64_t tmem_full[ACC_STAGES], tmem_empty[ACC_STAGES];
+  uint64_t epi_mma;            // wgrad: the epilogue's own MMAs have completed
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
@@ -97,84 +100,86 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
   tn = in_band / rows;
 }
 
-// Shared memory of the wgrad epilogue (after the pipeline stages):
-//   stg [2 groups][128 rows][33]  Gm chunk, transposed access for the dA column sums
-//   Bs  [128 rows][RANK]          the tile's rows of B (zero beyond d_out)
-//   As  [2 groups][RANK][32]      the current 32-column chunk of A, one copy per epilogue group
-__host__ __device__ constexpr int wgrad_epi_smem_bytes(int rank) {
-  return STG_BYTES + 128 * rank * 4 + EPI_GROUPS * rank * 32 * 4;
+// Shared memory of the wgrad epilogue (after the pipeline stages; every piece starts on a 1 KB boundary):
+//   gm    32 KB            Gm = G * m for 128 columns, bf16, as two 128-row x 64-column tiles in the
+//                          128-byte-swizzled layout TMA would produce.  Read by the tensor cores twice:
+//                          K-major (rows = weight rows, K = columns) for dB, MN-major (the same bytes,
+//                          M = columns, K = weight rows) for dA.
+//   abf   4 x RN x 128 B   bf16 copy of A[:, n0 : n0+256], four K-major tiles of 64 columns
+//   btbf  2 x RN x 128 B   bf16 copy of B[m0 : m0+128, :]^T, two K-major tiles of 64 weight rows
+// RN = max(rank, 16) rows (the MMA's N), rows beyond the rank are zero.
+constexpr int GM_BYTES = 128 * 128 * 2;
+__host__ __device__ constexpr int wgrad_rn(int rank) { return rank < 16 ? 16 : rank; }
+__host__ __device__ constexpr int wgrad_epi_smem_bytes(int rank) { return GM_BYTES + 6 * wgrad_rn(rank) * 128; }
+
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[N]) {
+  static_assert(N == 8 || N == 16 || N == 32, "tcgen05.ld width");
+  if constexpr (N == 8) ptx::tmem_ld_32x8(taddr, r);
+  else if constexpr (N == 16) ptx::tmem_ld_32x16(taddr, r);
+  else ptx::tmem_ld_32x32(taddr, r);
 }
 
-// Loads this thread's share of A[:, jc : jc+32] (RANK x 32 floats = RANK*8 float4 over 128 threads).
-template <int RANK>
-__device__ __forceinline__ void load_a_chunk(const GemmArgs& g, int jc, int t, float4 (&regs)[(RANK * 8 + 127) / 128]) {
-#pragma unroll
-  for (int u = 0; u < (RANK * 8 + 127) / 128; ++u) {
-    const int f = t + u * 128;
-    const int k = f >> 3, v = f & 7;
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (f < RANK * 8 && jc + v * 4 < g.p.d_in) a = __ldg(reinterpret_cast<const float4*>(g.A + (size_t)k * g.p.d_in + jc + v * 4));
-    regs[u] = a;
-  }
-}
-template <int RANK>
-__device__ __forceinline__ void store_a_chunk(float* As_g, int t, const float4 (&regs)[(RANK * 8 + 127) / 128]) {
-#pragma unroll
-  for (int u = 0; u < (RANK * 8 + 127) / 128; ++u) {
-    const int f = t + u * 128;
-    if (f < RANK * 8) reinterpret_cast<float4*>(As_g)[f] = regs[u];      // As_g[k][v*4..] with f = k*8 + v
-  }
-}
-
-// One 128 x 256 tile of G = dY^T X, read from tensor memory and reduced into ds, db, dA, dB.
-// Thread = one weight row (TMEM lane) of one epilogue group; the group owns 4 chunks of 32 columns.
-// Everything that does not depend on the accumulator (B rows, the first A chunk) is fetched before
-// waiting for the MMAs; W0, s, b and the next A chunk are fetched ahead of the arithmetic that
-// precedes their use, so that the loads' latency hides behind the FMA loops.
+// One 128 x 256 tile of G = dY^T X (Eq. 11), read from tensor memory and reduced into ds, db, dA, dB.
+//
+// The quantizer state of the tile's weights comes from the factor array F that the weight-tile kernel
+// of the same backward call wrote (ste_factor): F = w~ - w where the STE passes the gradient, a
+// sentinel where w was clamped.  Per element (thread = one weight row = one TMEM lane):
+//     ds += G * {Q_N | w~ - w | Q_P}      db += G * (1 - m)      Gm = G * m          (Eq. 5, 6, App. A.1)
+// Gm goes to shared memory as bf16 and the two contractions with the LoRA factors run on the tensor
+// cores (Eq. 13-14), 128 columns at a time, into accumulator columns this tile has already drained:
+//     dB[128 rows, r]   += Gm[128, 128] A[:, cols]^T          (K-major Gm)
+//     dA^T[128 cols, r]  = Gm^T[128 cols, 128 rows] B[rows, :] (MN-major view of the same Gm)
+// Their results are read back once per tile and added to dA / dB with fp32 atomics; the accumulator
+// stage is handed back to the main loop only after that.
 template <int RANK>
 __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, int n0, uint32_t tmem_acc, int quarter,
-                                                    int lane, int eg, float* epi_smem, GemmBarriers* bars,
+                                                    int lane, int eg, uint8_t* epi_smem, GemmBarriers* bars,
                                                     uint64_t* tmem_full_bar, uint32_t full_parity,
-                                                    uint64_t* tmem_empty_bar) {
+                                                    uint64_t* tmem_empty_bar, uint32_t& epi_phase) {
+  constexpr int RN = wgrad_rn(RANK);
   const Params& p = g.p;
-  float* stg_g = epi_smem + (size_t)eg * 128 * STG_LD;
-  float* Bs = epi_smem + EPI_GROUPS * 128 * STG_LD;
-  float* As_g = Bs + 128 * RANK + (size_t)eg * RANK * 32;
-  const int t = quarter * 32 + lane;                   // row in tile = thread index within the group
+  uint8_t* gm = epi_smem;
+  uint8_t* abf = gm + GM_BYTES;
+  uint8_t* btbf = abf + 4 * RN * 128;
+  const int t = quarter * 32 + lane;                   // row in tile = TMEM lane = thread index within the group
   const int t256 = eg * 128 + t;
   const int o = m0 + t;
   const bool row_ok = o < p.d_out;
-  constexpr int CHUNKS_PER_GROUP = (BN / 32) / EPI_GROUPS;
-  constexpr int A_REGS = (RANK * 8 + 127) / 128;
+  const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+  constexpr uint32_t DB_COL = 0, DA_COL0 = RN, DA_COL1 = 128;   // result columns inside the drained accumulator
 
-  // ---- before the accumulator is ready ----
-  ptx::named_bar_sync(3, EPI_THREADS);                 // both groups are done with the previous tile's Bs
+  // ---- bf16 copies of the tile's slices of A and B (nothing here depends on the accumulator) ----
+  // The MMAs of the previous tile that read these buffers have completed: every thread waited for them.
 #pragma unroll
-  for (int u = 0; u < (32 * RANK + EPI_THREADS - 1) / EPI_THREADS; ++u) {
-    const int f = t256 + u * EPI_THREADS;              // float4 index into Bs
-    if (f < 32 * RANK) {
-      const int row = f / (RANK / 4), kq = f % (RANK / 4);
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (m0 + row < p.d_out) v = __ldg(reinterpret_cast<const float4*>(g.B + (size_t)(m0 + row) * RANK + kq * 4));
-      reinterpret_cast<float4*>(Bs)[f] = v;
+  for (int u = 0; u < (RN * 32) / EPI_THREADS; ++u) {
+    const int q = t256 + u * EPI_THREADS;              // 16-byte chunk: rank k, columns n0 + 8 jc .. + 7
+    const int k = q >> 5, jc = q & 31;
+    const int col = n0 + jc * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (k < RANK && col < p.d_in) {
+      const float4* src = reinterpret_cast<const float4*>(g.A + (size_t)k * p.d_in + col);
+      const float4 a0 = __ldg(src), a1 = __ldg(src + 1);
+      v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w);
+      v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
+    }
+    *reinterpret_cast<uint4*>(abf + (jc >> 3) * (RN * 128) + k * 128 + (((jc & 7) ^ (k & 7)) << 4)) = v;
+  }
+#pragma unroll
+  for (int u = 0; u < RN / 2; u += 4) {                // thread = (weight row t, half eg of the ranks)
+    const int n = eg * (RN / 2) + u;
+    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row_ok && n < RANK) bv = __ldg(reinterpret_cast<const float4*>(g.B + (size_t)o * RANK + n));
+    const float be[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int nn = n + e;
+      uint8_t* dst = btbf + (t >> 6) * (RN * 128) + nn * 128 + ((((t & 63) >> 3) ^ (nn & 7)) << 4) + (t & 7) * 2;
+      *reinterpret_cast<__nv_bfloat16*>(dst) = __float2bfloat16_rn(be[e]);
     }
   }
-  {
-    float4 a0[A_REGS];
-    load_a_chunk<RANK>(g, n0 + eg * CHUNKS_PER_GROUP * 32, t, a0);
-    store_a_chunk<RANK>(As_g, t, a0);
-  }
-  float brow[RANK];
-#pragma unroll
-  for (int k = 0; k < RANK; k += 4) {
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (row_ok) v = __ldg(reinterpret_cast<const float4*>(g.B + (size_t)o * RANK + k));
-    brow[k] = v.x; brow[k + 1] = v.y; brow[k + 2] = v.z; brow[k + 3] = v.w;
-  }
-  float dBacc[RANK];
-#pragma unroll
-  for (int k = 0; k < RANK; ++k) dBacc[k] = 0.f;
-  ptx::named_bar_sync(3, EPI_THREADS);                 // Bs and the first A chunk are visible
+  ptx::fence_proxy_async_smem();
+  ptx::named_bar_sync(3, EPI_THREADS);
 
   bounded_wait(tmem_full_bar, full_parity, bars);
   ptx::tc_fence_after_sync();
@@ -183,149 +188,129 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
   int cur_grp = -1;
 
 #pragma unroll 1
-  for (int cc = 0; cc < CHUNKS_PER_GROUP; ++cc) {
-    const int c = eg * CHUNKS_PER_GROUP + cc;
-    const int jc = n0 + c * 32;                        // first column of the chunk
-
-    // loads issued ahead of their use
-    uint4 wraw[4];
-    float sv[4], bv[4];
-    int grp[4];
+  for (int h = 0; h < 2; ++h) {                        // 128 columns at a time; a group owns 64 of them
+#pragma unroll 1
+    for (int cc = 0; cc < 2; ++cc) {
+      const int c = h * 4 + eg * 2 + cc;               // 32-column chunk of the tile
+      const int jc = n0 + c * 32;
+      uint4 fr[4];
+      int grp[4];
 #pragma unroll
-    for (int sub = 0; sub < 4; ++sub) {
-      const int j = jc + sub * 8;
-      const bool ok = row_ok && j < p.d_in;
-      grp[sub] = ok ? j / p.group : -1;
-      wraw[sub] = ok ? __ldg(reinterpret_cast<const uint4*>(g.W0 + (size_t)o * p.d_in + j)) : make_uint4(0, 0, 0, 0);
-      sv[sub] = ok ? __ldg(g.s + (size_t)o * p.ngroups + grp[sub]) : 1.f;
-      bv[sub] = ok ? __ldg(g.b + (size_t)o * p.ngroups + grp[sub]) : 0.f;
-    }
-    float4 a_next[A_REGS];
-    if (cc + 1 < CHUNKS_PER_GROUP) load_a_chunk<RANK>(g, jc + 32, t, a_next);
+      for (int sub = 0; sub < 4; ++sub) {
+        const int j = jc + sub * 8;
+        const bool ok = row_ok && j < p.d_in;
+        grp[sub] = ok ? j / p.group : -1;
+        fr[sub] = ok ? __ldg(reinterpret_cast<const uint4*>(g.F + (size_t)o * p.d_in + j)) : make_uint4(0u, 0u, 0u, 0u);
+      }
+      uint32_t raw[32];
+      ptx::tmem_ld_32x32(tmem_acc + lane_base + (uint32_t)(c * 32), raw);
+      ptx::tmem_ld_wait();
+      float G[32];
+#pragma unroll
+      for (int e = 0; e < 32; ++e) G[e] = __uint_as_float(raw[e]);
 
-    uint32_t raw[32];
-    ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), raw);
+#pragma unroll
+      for (int sub = 0; sub < 4; ++sub) {
+        if (grp[sub] >= 0) {
+          if (grp[sub] != cur_grp) {
+            if (cur_grp >= 0) {
+              atomicAdd(&g.ds[(size_t)o * p.ngroups + cur_grp], p.grad_scale * ds_acc);
+              atomicAdd(&g.db[(size_t)o * p.ngroups + cur_grp], p.grad_scale * db_acc);
+            }
+            cur_grp = grp[sub]; ds_acc = 0.f; db_acc = 0.f;
+          }
+          const __half2* fh = reinterpret_cast<const __half2*>(&fr[sub]);
+#pragma unroll
+          for (int e2 = 0; e2 < 4; ++e2) {
+            const float2 f2 = __half22float2(fh[e2]);
+            const float fe[2] = {f2.x, f2.y};
+#pragma unroll
+            for (int e1 = 0; e1 < 2; ++e1) {
+              const int idx = sub * 8 + e2 * 2 + e1;
+              const float f = fe[e1], Gv = G[idx];
+              const bool inr = fabsf(f) < 1.f;           // STE gate m
+              ds_acc = fmaf(Gv, inr ? f : (f < 0.f ? p.qn : p.qp), ds_acc);
+              db_acc += inr ? 0.f : Gv;
+              G[idx] = inr ? Gv : 0.f;                   // G becomes G * m
+            }
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) G[sub * 8 + e] = 0.f;
+        }
+      }
+      // Gm chunk -> shared memory: row t, 16-byte pieces (c & 1) * 4 + v of the 64-column tile (c & 3) >> 1
+      uint8_t* grow = gm + ((c & 3) >> 1) * (GM_BYTES / 2) + t * 128;
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        uint4 o4;
+        o4.x = pack_bf16x2(G[v * 8 + 0], G[v * 8 + 1]); o4.y = pack_bf16x2(G[v * 8 + 2], G[v * 8 + 3]);
+        o4.z = pack_bf16x2(G[v * 8 + 4], G[v * 8 + 5]); o4.w = pack_bf16x2(G[v * 8 + 6], G[v * 8 + 7]);
+        *reinterpret_cast<uint4*>(grow + ((((c & 1) * 4 + v) ^ (t & 7)) << 4)) = o4;
+      }
+    }
+    ptx::fence_proxy_async_smem();                     // Gm visible to the tensor cores
+    ptx::tc_fence_before_sync();                       // the TMEM reads above come before the MMAs below
+    ptx::named_bar_sync(3, EPI_THREADS);
+    if (t256 == 0 && !bars->abort) {
+      ptx::tc_fence_after_sync();
+      constexpr uint32_t idesc_db = ptx::make_idesc_bf16(128, RN, false, false);
+      constexpr uint32_t idesc_da = ptx::make_idesc_bf16(128, RN, true, false);
+      const uint32_t gm_a = ptx::smem_u32(gm), abf_a = ptx::smem_u32(abf), bt_a = ptx::smem_u32(btbf);
+#pragma unroll
+      for (int sb = 0; sb < 2; ++sb) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const uint64_t da = ptx::make_smem_desc_sw128(gm_a + sb * (GM_BYTES / 2) + k * 32, 16, 1024);
+          const uint64_t db = ptx::make_smem_desc_sw128(abf_a + (h * 2 + sb) * (RN * 128) + k * 32, 16, 1024);
+          ptx::mma_bf16_ss(tmem_acc + DB_COL, da, db, idesc_db, (h | sb | k) != 0 ? 1u : 0u);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint64_t da = ptx::make_smem_desc_sw128(gm_a + k * 2048, GM_BYTES / 2, 1024);
+        const uint64_t db = ptx::make_smem_desc_sw128(bt_a + (k >> 2) * (RN * 128) + (k & 3) * 32, 16, 1024);
+        ptx::mma_bf16_ss(tmem_acc + (h == 0 ? DA_COL0 : DA_COL1), da, db, idesc_da, k != 0 ? 1u : 0u);
+      }
+      ptx::mma_commit(&bars->epi_mma);
+    }
+    bounded_wait(&bars->epi_mma, epi_phase, bars);     // Gm reusable; after the second half, results complete
+    epi_phase ^= 1;
+    ptx::tc_fence_after_sync();
+  }
+
+  if (row_ok && cur_grp >= 0) {
+    atomicAdd(&g.ds[(size_t)o * p.ngroups + cur_grp], p.grad_scale * ds_acc);
+    atomicAdd(&g.db[(size_t)o * p.ngroups + cur_grp], p.grad_scale * db_acc);
+  }
+  {  // dB: lane = weight row; group eg takes half of the ranks
+    constexpr int NB = RN / 2;
+    uint32_t r[NB];
+    tmem_ld_cols<NB>(tmem_acc + lane_base + DB_COL + (uint32_t)(eg * NB), r);
     ptx::tmem_ld_wait();
-    if (cc == CHUNKS_PER_GROUP - 1) {                  // accumulator stage fully read by this thread
-      ptx::tc_fence_before_sync();
-      ptx::mbar_arrive(tmem_empty_bar);
+    if (row_ok) {
+#pragma unroll
+      for (int k = 0; k < NB; ++k)
+        if (eg * NB + k < RANK) atomicAdd(&g.dB[(size_t)o * RANK + eg * NB + k], p.gamma * __uint_as_float(r[k]));
     }
-    float G[32];
-#pragma unroll
-    for (int e = 0; e < 32; ++e) G[e] = __uint_as_float(raw[e]);
-
-    // merge: acc[e] = sum_k B[o,k] A[k, jc+e]                                  (Eq. 7)
-    float acc[32];
-#pragma unroll
-    for (int e = 0; e < 32; ++e) acc[e] = 0.f;
-#pragma unroll
-    for (int k = 0; k < RANK; ++k) {
-      const float4* arow = reinterpret_cast<const float4*>(As_g + k * 32);
-#pragma unroll
-      for (int v = 0; v < 8; ++v) {
-        const float4 a = arow[v];
-        acc[v * 4 + 0] = fmaf(brow[k], a.x, acc[v * 4 + 0]);
-        acc[v * 4 + 1] = fmaf(brow[k], a.y, acc[v * 4 + 1]);
-        acc[v * 4 + 2] = fmaf(brow[k], a.z, acc[v * 4 + 2]);
-        acc[v * 4 + 3] = fmaf(brow[k], a.w, acc[v * 4 + 3]);
-      }
-    }
-
-    // quantizer state, STE gate, ds / db partial sums                           (Eq. 8, 5, 6)
-#pragma unroll
-    for (int sub = 0; sub < 4; ++sub) {
-      if (grp[sub] >= 0) {
-        if (grp[sub] != cur_grp) {
-          if (cur_grp >= 0) {
-            atomicAdd(&g.ds[(size_t)o * p.ngroups + cur_grp], p.grad_scale * ds_acc);
-            atomicAdd(&g.db[(size_t)o * p.ngroups + cur_grp], p.grad_scale * db_acc);
-          }
-          cur_grp = grp[sub]; ds_acc = 0.f; db_acc = 0.f;
-        }
-        const float rs = 1.0f / sv[sub];
-        const uint4 wr = wraw[sub];
-        const float w0[8] = {bf16_lo(wr.x), bf16_hi(wr.x), bf16_lo(wr.y), bf16_hi(wr.y),
-                             bf16_lo(wr.z), bf16_hi(wr.z), bf16_lo(wr.w), bf16_hi(wr.w)};
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int idx = sub * 8 + e;
-          const QuantElem q = quantize_elem(merge_elem(w0[e], acc[idx], p.gamma), sv[sub], rs, bv[sub], p.qn, p.qp);
-          const float Gv = G[idx];
-          if (ste_in_range(q.w, p.qn, p.qp)) {
-            ds_acc = fmaf(Gv, q.code - q.w, ds_acc);
-          } else {
-            ds_acc = fmaf(Gv, (q.w < p.qn) ? p.qn : p.qp, ds_acc);
-            db_acc += Gv;
-            G[idx] = 0.f;                              // G becomes G * m
-          }
-        }
-      } else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) G[sub * 8 + e] = 0.f;
-      }
-    }
-
-    // dB[o,k] += sum_e Gm[e] A[k, jc+e]                                         (Eq. 14)
-#pragma unroll
-    for (int k = 0; k < RANK; ++k) {
-      const float4* arow = reinterpret_cast<const float4*>(As_g + k * 32);
-      float part0 = 0.f, part1 = 0.f;
-#pragma unroll
-      for (int v = 0; v < 8; v += 2) {
-        const float4 a = arow[v], a2 = arow[v + 1];
-        part0 = fmaf(G[v * 4 + 0], a.x, part0);
-        part0 = fmaf(G[v * 4 + 1], a.y, part0);
-        part0 = fmaf(G[v * 4 + 2], a.z, part0);
-        part0 = fmaf(G[v * 4 + 3], a.w, part0);
-        part1 = fmaf(G[v * 4 + 4], a2.x, part1);
-        part1 = fmaf(G[v * 4 + 5], a2.y, part1);
-        part1 = fmaf(G[v * 4 + 6], a2.z, part1);
-        part1 = fmaf(G[v * 4 + 7], a2.w, part1);
-      }
-      dBacc[k] += part0 + part1;
-    }
-
-    // dA[k, jc+col] += sum_rows B[o,k] Gm[o, col]: transpose through shared memory   (Eq. 13)
-#pragma unroll
-    for (int e = 0; e < 32; ++e) stg_g[t * STG_LD + e] = G[e];
-    ptx::named_bar_sync(1 + eg, 128);                  // Gm chunk visible; everyone is past the reads of As_g
-    if (cc + 1 < CHUNKS_PER_GROUP) store_a_chunk<RANK>(As_g, t, a_next);
-    {
-      const int col = t & 31, rq = t >> 5;
-      float acc_a[RANK];
-#pragma unroll
-      for (int k = 0; k < RANK; ++k) acc_a[k] = 0.f;
-#pragma unroll 4
-      for (int rr = 0; rr < 32; ++rr) {
-        const int r2 = rq * 32 + rr;
-        const float gm = stg_g[r2 * STG_LD + col];
-        const float4* b4 = reinterpret_cast<const float4*>(Bs + r2 * RANK);
-#pragma unroll
-        for (int k = 0; k < RANK; k += 4) {
-          const float4 bq = b4[k >> 2];
-          acc_a[k] = fmaf(bq.x, gm, acc_a[k]);
-          acc_a[k + 1] = fmaf(bq.y, gm, acc_a[k + 1]);
-          acc_a[k + 2] = fmaf(bq.z, gm, acc_a[k + 2]);
-          acc_a[k + 3] = fmaf(bq.w, gm, acc_a[k + 3]);
-        }
-      }
-      const int ja = jc + col;
-      if (ja < p.d_in) {
-#pragma unroll
-        for (int k = 0; k < RANK; ++k) atomicAdd(&g.dA[(size_t)k * p.d_in + ja], p.gamma * acc_a[k]);
-      }
-    }
-    ptx::named_bar_sync(1 + eg, 128);                  // staging tile reusable, next A chunk visible
   }
-
-  if (row_ok) {
-    if (cur_grp >= 0) {
-      atomicAdd(&g.ds[(size_t)o * p.ngroups + cur_grp], p.grad_scale * ds_acc);
-      atomicAdd(&g.db[(size_t)o * p.ngroups + cur_grp], p.grad_scale * db_acc);
-    }
+  {  // dA: lane = column of the half eg
+    const int col = n0 + eg * 128 + t;
+    constexpr int W = RN < 32 ? RN : 32;
 #pragma unroll
-    for (int k = 0; k < RANK; ++k) atomicAdd(&g.dB[(size_t)o * RANK + k], p.gamma * dBacc[k]);
+    for (int kb = 0; kb < RN; kb += W) {
+      uint32_t r[W];
+      tmem_ld_cols<W>(tmem_acc + lane_base + (eg == 0 ? DA_COL0 : DA_COL1) + (uint32_t)kb, r);
+      ptx::tmem_ld_wait();
+      if (col < p.d_in) {
+#pragma unroll
+        for (int k = 0; k < W; ++k)
+          if (kb + k < RANK) atomicAdd(&g.dA[(size_t)(kb + k) * p.d_in + col], p.gamma * __uint_as_float(r[k]));
+      }
+    }
   }
+  ptx::tc_fence_before_sync();
+  ptx::mbar_arrive(tmem_empty_bar);                    // accumulator stage (and its result columns) free
 }
 
 template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES>
@@ -335,7 +320,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
   constexpr int EPI_SMEM = (EPI == EPI_WGRAD) ? wgrad_epi_smem_bytes(RANK) : 0;
-  float* epi_smem = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES);
+  uint8_t* epi_smem = smem + (size_t)STAGES * STAGE_BYTES;
   GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + (size_t)STAGES * STAGE_BYTES + EPI_SMEM);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -347,6 +332,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::mbar_init(&bars->tmem_full[i], 1);
       ptx::mbar_init(&bars->tmem_empty[i], EPI_THREADS);
     }
+    ptx::mbar_init(&bars->epi_mma, 1);
     bars->abort = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tmap(&tmap_a);
@@ -436,6 +422,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int quarter = warp & 3;
     const int eg = (warp - EPI_FIRST_WARP) >> 2;
     int acc = 0; uint32_t acc_phase = 0;
+    [[maybe_unused]] uint32_t epi_phase = 0;
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
       int tm, tn;
       tile_coords(t, g.tiles_m, g.tiles_n, tm, tn);
@@ -473,7 +460,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         }
       } else {
         wgrad_epilogue_tile<RANK>(g, m0, n0, tmem_acc, quarter, lane, eg, epi_smem, bars, &bars->tmem_full[acc],
-                                  acc_phase, &bars->tmem_empty[acc]);
+                                  acc_phase, &bars->tmem_empty[acc], epi_phase);
       }
       if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1; }
     }
@@ -574,17 +561,16 @@ inline l4q_status gemm_dgrad_bf16(const Params& p, const void* dY, const void* W
 }
 
 // G[d_out, d_in] = dY^T X reduced on chip into dA, dB, ds, db (which must be zero on entry).
-inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY, const void* W0, const float* A,
-                                  const float* B, const float* s, const float* b, float* dA, float* dB, float* ds,
-                                  float* db, cudaStream_t st) {
+inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY, const void* F, const float* A,
+                                  const float* B, float* dA, float* dB, float* ds, float* db, cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BK) || !make_tmap_bf16(&tb, X, p.tokens, p.d_in, BK))
     return L4Q_ERR_CUDA;
   GemmArgs g{};
   g.M = p.d_out; g.N = p.d_in; g.K = p.tokens;
   g.p = p;
-  g.W0 = reinterpret_cast<const __nv_bfloat16*>(W0);
-  g.A = A; g.B = B; g.s = s; g.b = b;
+  g.F = reinterpret_cast<const __half*>(F);
+  g.A = A; g.B = B;
   g.dA = dA; g.dB = dB; g.ds = ds; g.db = db;
   switch (p.rank) {
     case 8: return launch_gemm<true, true, EPI_WGRAD, 8, 3>(ta, tb, g, st);

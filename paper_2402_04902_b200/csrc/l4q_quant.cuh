@@ -40,6 +40,7 @@ __global__ void __launch_bounds__(WT_THREADS)
 k_weight_tile(Params p, const void* __restrict__ W0, const float* __restrict__ A, const float* __restrict__ B,
               const float* __restrict__ s, const float* __restrict__ b,
               void* __restrict__ wq_out,                       // MODE_DEQUANT: [d_out, d_in] io dtype
+              __half* __restrict__ f_out,                      // MODE_DEQUANT, optional: STE factors [d_out, d_in]
               uint32_t* __restrict__ codes, __half* __restrict__ s16, __half* __restrict__ b16) {  // MODE_PACK
   extern __shared__ __align__(16) float smem_f[];
   const int r = p.rank;
@@ -100,14 +101,21 @@ k_weight_tile(Params p, const void* __restrict__ W0, const float* __restrict__ A
       sv = s[(size_t)o * p.ngroups + grp];
       bvv = b[(size_t)o * p.ngroups + grp];
       const float rs = 1.0f / sv;
-      float wq[8];
+      float wq[8], fac[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const QuantElem q = quantize_elem(merge_elem(w0[j], acc[i][j], p.gamma), sv, rs, bvv, p.qn, p.qp);
         code[j] = q.code;
         wq[j] = q.wq;
+        fac[j] = ste_factor(q, p.qn, p.qp);
       }
       if constexpr (MODE == WT_MODE_DEQUANT) {
+        if (f_out != nullptr) {
+          __half2 h[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) h[j] = __floats2half2_rn(fac[2 * j], fac[2 * j + 1]);
+          *reinterpret_cast<uint4*>(f_out + (size_t)o * p.d_in + col) = *reinterpret_cast<const uint4*>(h);
+        }
         if constexpr (IO_BF16) {
           uint4 out;
           out.x = pack_bf16x2(wq[0], wq[1]); out.y = pack_bf16x2(wq[2], wq[3]);

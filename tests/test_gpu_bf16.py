@@ -77,8 +77,10 @@ def test_bf16_backward_is_linear_in_dY_and_additive_over_token_shards():
     second = {k: (v[256:] if k in ("X", "dY") else v) for k, v in arrays.items()}
     o1 = gh.run_layer(cfg, first, do_fwd=False)
     o2 = gh.run_layer(cfg, second, do_fwd=False)
-    for k in ("dA", "dB", "ds", "db"):
-        assert pu.rel_l2(o1[k] + o2[k], full[k]) <= 1e-3, k
+    # ds, db are fp32 sums of G; dA, dB contract a bf16 copy of G * m on the tensor cores, and
+    # rounding G1 and G2 to bf16 separately differs from rounding G1 + G2 by ~2^-9 per element
+    for k, tol in (("dA", 1e-2), ("dB", 1e-2), ("ds", 1e-3), ("db", 1e-3)):
+        assert pu.rel_l2(o1[k] + o2[k], full[k]) <= tol, k
     assert np.array_equal(np.vstack([o1["dX"], o2["dX"]]), full["dX"])
     doubled = dict(arrays); doubled["dY"] = arrays["dY"] * np.float32(2.0)      # exact in bf16
     o3 = gh.run_layer(cfg, doubled, do_fwd=False)
