@@ -100,6 +100,47 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
   tn = in_band / rows;
 }
 
+// Work distribution over the persistent CTAs: tile t goes to CTA t mod gridDim.x, so the CTAs of a
+// wave work on neighbouring tiles and share operand panels in L2.  With TAIL_SPLIT (wgrad) the tiles
+// of the last, partial wave are additionally cut along K into `split` slices, one per otherwise idle
+// CTA: the reductions of the wgrad epilogue are linear in G and accumulate with atomics, so a partial
+// sum over tokens is just one more contribution.
+struct WorkUnit { int tile, kb0, kb1; };
+
+__host__ __device__ inline int tail_split_factor(int tiles, int grid, int num_kb) {
+  const int tail = tiles % grid;
+  if (tail == 0) return 1;
+  const int split = grid / tail;
+  return split < 1 ? 1 : (split > num_kb ? num_kb : split);
+}
+
+template <bool TAIL_SPLIT>
+struct WorkIter {
+  int next_tile, num_tiles, num_kb, first_tail, tail, split;
+  bool tail_done;
+  __device__ WorkIter(int tiles, int kblocks) : next_tile(blockIdx.x), num_tiles(tiles), num_kb(kblocks) {
+    const int grid = gridDim.x;
+    first_tail = TAIL_SPLIT ? (tiles / grid) * grid : tiles;
+    tail = tiles - first_tail;
+    split = TAIL_SPLIT ? tail_split_factor(tiles, grid, kblocks) : 1;
+    tail_done = false;
+  }
+  __device__ bool next(WorkUnit& u) {
+    if (next_tile < first_tail) {
+      u.tile = next_tile; u.kb0 = 0; u.kb1 = num_kb;
+      next_tile += gridDim.x;
+      return true;
+    }
+    if (tail_done || (int)blockIdx.x >= tail * split) return false;
+    tail_done = true;
+    const int slice = blockIdx.x / tail;
+    u.tile = first_tail + blockIdx.x % tail;
+    u.kb0 = (int)((long long)num_kb * slice / split);
+    u.kb1 = (int)((long long)num_kb * (slice + 1) / split);
+    return u.kb1 > u.kb0;
+  }
+};
+
 // Shared memory of the wgrad epilogue (after the pipeline stages; every piece starts on a 1 KB boundary):
 //   gm    32 KB            Gm = G * m for 128 columns, bf16, as two 128-row x 64-column tiles in the
 //                          128-byte-swizzled layout TMA would produce.  Read by the tensor cores twice:
@@ -325,6 +366,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = g.tiles_m * g.tiles_n;
+  constexpr bool TAIL_SPLIT = (EPI == EPI_WGRAD);
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&bars->full[i], 1); ptx::mbar_init(&bars->empty[i], 1); }
@@ -351,11 +393,13 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      for (int t = blockIdx.x; t < num_tiles && !bars->abort; t += gridDim.x) {
+      WorkIter<TAIL_SPLIT> work(num_tiles, g.num_kb);
+      WorkUnit u;
+      while (!bars->abort && work.next(u)) {
         int tm, tn;
-        tile_coords(t, g.tiles_m, g.tiles_n, tm, tn);
+        tile_coords(u.tile, g.tiles_m, g.tiles_n, tm, tn);
         const int m0 = tm * BM, n0 = tn * BN;
-        for (int kb = 0; kb < g.num_kb && !bars->abort; ++kb) {
+        for (int kb = u.kb0; kb < u.kb1 && !bars->abort; ++kb) {
           bounded_wait(&bars->empty[stage], phase ^ 1, bars);
           if (bars->abort) break;
           uint8_t* sa = stage_base + (size_t)stage * STAGE_BYTES;
@@ -392,12 +436,14 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       constexpr uint32_t B_LBO = B_MN ? (BK * 128) : 16, B_SBO = 1024, B_KSTEP = B_MN ? 2048 : 32;
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
-      for (int t = blockIdx.x; t < num_tiles && !bars->abort; t += gridDim.x) {
+      WorkIter<TAIL_SPLIT> work(num_tiles, g.num_kb);
+      WorkUnit u;
+      while (!bars->abort && work.next(u)) {
         bounded_wait(&bars->tmem_empty[acc], acc_phase ^ 1, bars);
         if (bars->abort) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < g.num_kb; ++kb) {
+        for (int kb = u.kb0; kb < u.kb1; ++kb) {
           bounded_wait(&bars->full[stage], phase, bars);
           if (bars->abort) break;
           ptx::tc_fence_after_sync();
@@ -407,7 +453,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t da = ptx::make_smem_desc_sw128(sa + k * A_KSTEP, A_LBO, A_SBO);
             const uint64_t db = ptx::make_smem_desc_sw128(sb + k * B_KSTEP, B_LBO, B_SBO);
-            ptx::mma_bf16_ss(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+            ptx::mma_bf16_ss(d_tmem, da, db, idesc, (kb != u.kb0 || k != 0) ? 1u : 0u);
           }
           ptx::mma_commit(&bars->empty[stage]);       // smem stage reusable once these MMAs retire
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -423,9 +469,11 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int eg = (warp - EPI_FIRST_WARP) >> 2;
     int acc = 0; uint32_t acc_phase = 0;
     [[maybe_unused]] uint32_t epi_phase = 0;
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+    WorkIter<TAIL_SPLIT> work(num_tiles, g.num_kb);
+    WorkUnit u;
+    while (work.next(u)) {
       int tm, tn;
-      tile_coords(t, g.tiles_m, g.tiles_n, tm, tn);
+      tile_coords(u.tile, g.tiles_m, g.tiles_n, tm, tn);
       const int m0 = tm * BM, n0 = tn * BN;
       const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
       if constexpr (EPI == EPI_STORE) {
@@ -533,7 +581,9 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
   const size_t smem = gemm_smem_bytes(STAGES, EPI == EPI_WGRAD ? wgrad_epi_smem_bytes(RANK) : 0);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return L4Q_ERR_CUDA;
-  const int grid = std::min(g.tiles_m * g.tiles_n, sm_count());
+  const int tiles = g.tiles_m * g.tiles_n, sms = sm_count();
+  int grid = std::min(tiles, sms);
+  if (EPI == EPI_WGRAD && tiles < sms) grid = tiles * std::min(sms / tiles, g.num_kb);   // K slices for the idle SMs
   kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, g);
   return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
 }
