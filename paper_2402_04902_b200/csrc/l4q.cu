@@ -11,6 +11,7 @@
 #include "l4q_quant.cuh"
 #include "l4q_val.cuh"
 #include "l4q_gemm.cuh"
+#include "l4q_wtile.cuh"
 
 using namespace l4q;
 
@@ -108,6 +109,13 @@ inline l4q_status launch_status() { return cudaGetLastError() == cudaSuccess ? L
 template <bool IO_BF16>
 l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const float* B, const float* s,
                           const float* b, void* wq, __half* fac, cudaStream_t st) {
+  if constexpr (IO_BF16) {
+    const int mode = fac ? WT2_DEQUANT_F : WT2_DEQUANT;
+    if (wtile_tc_supported(p, mode)) {               // tensor-core merge, TMA in and out
+      KernelScope ks(L4Q_KERNEL_DEQUANT, st);
+      return launch_wtile_tc(mode, p, W0, A, B, s, b, wq, fac, nullptr, nullptr, st);
+    }
+  }
   const size_t smem = weight_tile_smem_bytes(p.rank);
   auto kern = k_weight_tile<IO_BF16, WT_MODE_DEQUANT>;
   if (smem > 48 * 1024 &&
@@ -122,6 +130,12 @@ l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const
 template <bool IO_BF16>
 l4q_status launch_pack(const Params& p, const void* W0, const float* A, const float* B, const float* s,
                        const float* b, uint32_t* codes, __half* s16, __half* b16, cudaStream_t st) {
+  if constexpr (IO_BF16) {
+    if (wtile_tc_supported(p, WT2_PACK)) {
+      KernelScope ks(L4Q_KERNEL_PACK, st);
+      return launch_wtile_tc(WT2_PACK, p, W0, A, B, s, b, codes, nullptr, s16, b16, st);
+    }
+  }
   const size_t smem = weight_tile_smem_bytes(p.rank);
   auto kern = k_weight_tile<IO_BF16, WT_MODE_PACK>;
   if (smem > 48 * 1024 &&
@@ -378,8 +392,8 @@ l4q_status l4q_profile_read(int kernel, uint64_t* launches, double* total_ms) {
 
 const char* l4q_kernel_name(int kernel) {
   switch (kernel) {
-    case L4Q_KERNEL_DEQUANT: return "k_weight_tile<dequant>";
-    case L4Q_KERNEL_PACK: return "k_weight_tile<pack>";
+    case L4Q_KERNEL_DEQUANT: return "weight tile: merge + fake-quantize";
+    case L4Q_KERNEL_PACK: return "weight tile: merge + quantize + pack";
     case L4Q_KERNEL_GEMM_FWD: return "k_gemm_bf16<fwd>";
     case L4Q_KERNEL_GEMM_DGRAD: return "k_gemm_bf16<dgrad>";
     case L4Q_KERNEL_GEMM_WGRAD: return "k_gemm_bf16<wgrad>";

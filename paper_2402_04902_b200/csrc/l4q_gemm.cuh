@@ -71,7 +71,8 @@ inline size_t gemm_smem_bytes(int stages, int epi_bytes) {
 }
 
 // Bounded mbarrier wait.  Returns immediately once the CTA's abort flag is set.
-__device__ __forceinline__ void bounded_wait(uint64_t* bar, uint32_t parity, GemmBarriers* bars) {
+template <class Barriers>
+__device__ __forceinline__ void bounded_wait(uint64_t* bar, uint32_t parity, Barriers* bars) {
   if (ptx::mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
   uint32_t spins = 0;
