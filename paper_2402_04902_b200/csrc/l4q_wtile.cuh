@@ -48,6 +48,7 @@ struct WtileArgs {
   int n_out;               // staging buffers for the second output (F or codes): 0, 1 or 2
   int out_bytes;           // bytes of one such buffer
   int atoms;               // swizzle atoms per operand row: ceil(2 rank / 32)
+  int ngt;                 // upper bound of the quantization groups a 128-column tile intersects
 };
 
 struct __align__(8) WtileBarriers {
@@ -61,9 +62,12 @@ struct __align__(8) WtileBarriers {
   volatile uint32_t abort;
 };
 
+// s and b of a tile in shared memory: two buffers of [128 rows][s x ngt | b x ngt] floats (1 KB multiples).
+__host__ __device__ inline size_t wtile_sb_bytes(int ngt) { return 2 * (size_t)WT2_ROWS * 2 * ngt * sizeof(float); }
+
 inline size_t wtile_smem_bytes(const WtileArgs& a) {
   return 1024 + (size_t)a.n_stages * WT2_STAGE_BYTES + (size_t)a.n_out * a.out_bytes +
-         2 * (size_t)a.atoms * WT2_ATOM_BYTES + sizeof(WtileBarriers);
+         2 * (size_t)a.atoms * WT2_ATOM_BYTES + wtile_sb_bytes(a.ngt) + sizeof(WtileBarriers);
 }
 
 // Tile i of this CTA: row tiles of one column panel go to neighbouring CTAs.
@@ -73,6 +77,13 @@ __device__ __forceinline__ bool wtile_coords(const WtileArgs& a, int i, int& m0,
   m0 = (t % a.tiles_m) * WT2_ROWS;
   n0 = (t / a.tiles_m) * WT2_COLS;
   return true;
+}
+
+// x = hi + lo with hi, lo representable in tf32 (low 13 mantissa bits clear): hi keeps the leading 10
+// mantissa bits of x (truncation), lo the leading bits of the exact remainder.  Plain logic ops.
+__device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
+  hi = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+  lo = __uint_as_float(__float_as_uint(x - hi) & 0xFFFFE000u);
 }
 
 // Builds the split operands of one tile in shared memory, K-major with the 128-byte swizzle:
@@ -98,8 +109,8 @@ __device__ __forceinline__ void wtile_prep_operands(const WtileArgs& a, int m0, 
     float ah[4], al[4], bh[4], bl[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      ah[e] = ptx::round_tf32(av[e]);  al[e] = ptx::round_tf32(av[e] - ah[e]);
-      bh[e] = ptx::round_tf32(bvv[e]); bl[e] = ptx::round_tf32(bvv[e] - bh[e]);
+      split_tf32(av[e], ah[e], al[e]);
+      split_tf32(bvv[e], bh[e], bl[e]);
     }
     const int ch = kc, cl = (r >> 2) + kc;           // 16-byte chunk index of the head / tail within the row
     const uint32_t off_h = (uint32_t)(ch >> 3) * WT2_ATOM_BYTES + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
@@ -136,7 +147,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
   uint8_t* out_base = stage_base + (size_t)a.n_stages * WT2_STAGE_BYTES;
   uint8_t* acat = out_base + (size_t)a.n_out * a.out_bytes;
   uint8_t* bcat = acat + (size_t)a.atoms * WT2_ATOM_BYTES;
-  WtileBarriers* bars = reinterpret_cast<WtileBarriers*>(bcat + (size_t)a.atoms * WT2_ATOM_BYTES);
+  float* sb_base = reinterpret_cast<float*>(bcat + (size_t)a.atoms * WT2_ATOM_BYTES);
+  WtileBarriers* bars = reinterpret_cast<WtileBarriers*>(reinterpret_cast<uint8_t*>(sb_base) + wtile_sb_bytes(a.ngt));
   const Params& p = a.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr bool HAS_OUT1 = (MODE != WT2_DEQUANT);
@@ -261,30 +273,66 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     int acc = 0; uint32_t acc_phase = 0;
     int ob = 0; uint32_t out_round = 0;                         // uses of staging buffer `ob` so far
     int m0, n0;
+    // s and b reach the arithmetic through shared memory: the four warps of column slice 0 (one thread
+    // per weight row) copy the tile's values of their row, one tile ahead, with asynchronous 4-byte
+    // copies; all epilogue threads meet at a barrier at the end of every tile.  (Loading them per thread
+    // would touch 32 different lines per instruction, sixteen times over, and starve the TMA loads.)
+    const int sbw = 2 * a.ngt;                                  // floats per row: s x ngt | b x ngt
+    auto stage_sb = [&](int m0_, int n0_, int buf) {
+      if (sl != 0) return;
+      float* dst = sb_base + ((size_t)buf * WT2_ROWS + row) * sbw;
+      const int o_ = m0_ + row;
+      const int g_first = n0_ / p.group;
+      for (int k = 0; k < a.ngt; ++k) {
+        const int g = g_first + k;
+        if (o_ < p.d_out && g < p.ngroups) {
+          ptx::cp_async_4(dst + k, a.s + (size_t)o_ * p.ngroups + g);
+          ptx::cp_async_4(dst + a.ngt + k, a.b + (size_t)o_ * p.ngroups + g);
+        } else {
+          dst[k] = 1.f; dst[a.ngt + k] = 0.f;
+        }
+      }
+      ptx::cp_async_commit();
+    };
     if (wtile_coords(a, 0, m0, n0)) {
+      stage_sb(m0, n0, 0);
       wtile_prep_operands(a, m0, n0, et, acat, bcat);
       ptx::fence_proxy_async_smem();
       ptx::mbar_arrive(&bars->prep_full);
+      ptx::cp_async_wait_all();
     }
+    ptx::named_bar_sync(1, WT2_EPI_THREADS);
     for (int i = 0; wtile_coords(a, i, m0, n0); ++i) {
       const int o = m0 + row;
       const bool row_ok = o < p.d_out;
       const int jc = n0 + sl * 32;
       float sv[4], bv[4];
       int grp[4];
+      uint32_t first_mask = 0;                                  // bit sub: the piece is the first of its group
+      {
+        const int g_first = n0 / p.group;
+        const int g0 = jc / p.group;
+        const int rem0 = jc - g0 * p.group;
+        const float* src = sb_base + ((size_t)(i & 1) * WT2_ROWS + row) * sbw;
 #pragma unroll
-      for (int sub = 0; sub < 4; ++sub) {
-        const int j = jc + sub * 8;
-        const bool ok = row_ok && j < p.d_in;
-        grp[sub] = ok ? j / p.group : -1;
-        sv[sub] = ok ? __ldg(a.s + (size_t)o * p.ngroups + grp[sub]) : 1.f;
-        bv[sub] = ok ? __ldg(a.b + (size_t)o * p.ngroups + grp[sub]) : 0.f;
+        for (int sub = 0; sub < 4; ++sub) {
+          int rem = rem0 + sub * 8, g = g0;
+#pragma unroll
+          for (int c = 0; c < 3; ++c)
+            if (rem >= p.group) { rem -= p.group; ++g; }
+          const bool ok = row_ok && jc + sub * 8 < p.d_in;
+          grp[sub] = ok ? g : -1;
+          if (rem == 0) first_mask |= 1u << sub;
+          sv[sub] = ok ? src[g - g_first] : 1.f;
+          bv[sub] = ok ? src[a.ngt + g - g_first] : 0.f;
+        }
       }
       bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
       ptx::tc_fence_after_sync();
       {  // the MMAs of this tile have completed: their operands may be replaced by the next tile's
         int m1, n1;
         if (wtile_coords(a, i + 1, m1, n1)) {
+          stage_sb(m1, n1, (i + 1) & 1);
           wtile_prep_operands(a, m1, n1, et, acat, bcat);
           ptx::fence_proxy_async_smem();
           ptx::mbar_arrive(&bars->prep_full);
@@ -303,13 +351,14 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       uint8_t* wrow = stage_base + (size_t)stage * WT2_STAGE_BYTES + (sl >> 1) * (WT2_STAGE_BYTES / 2) + row * 128;
       [[maybe_unused]] uint8_t* out1 = out_base + (size_t)ob * a.out_bytes;
       [[maybe_unused]] uint32_t ucodes[32];
+      float rs = 1.f;
 #pragma unroll
       for (int sub = 0; sub < 4; ++sub) {
         const uint32_t chunk = (uint32_t)((((sl & 1) * 4 + sub) ^ (row & 7)) << 4);
         const uint4 wr = *reinterpret_cast<const uint4*>(wrow + chunk);
         const float w0[8] = {bf16_lo(wr.x), bf16_hi(wr.x), bf16_lo(wr.y), bf16_hi(wr.y),
                              bf16_lo(wr.z), bf16_hi(wr.z), bf16_lo(wr.w), bf16_hi(wr.w)};
-        const float rs = 1.0f / sv[sub];
+        if (sub == 0 || ((first_mask >> sub) & 1u)) rs = 1.0f / sv[sub];         // one reciprocal per group
         float wq[8], fac[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
@@ -333,7 +382,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
               *reinterpret_cast<const uint4*>(h);
         }
         if constexpr (MODE == WT2_PACK) {
-          if (grp[sub] >= 0 && ((jc + sub * 8) % p.group) == 0) {
+          if (grp[sub] >= 0 && ((first_mask >> sub) & 1u)) {                   // first piece of its group
             a.s16[(size_t)o * p.ngroups + grp[sub]] = __float2half_rn(sv[sub]);
             a.b16[(size_t)o * p.ngroups + grp[sub]] = __float2half_rn(fmaf(sv[sub], p.qn, bv[sub]));
           }
@@ -354,6 +403,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
       ptx::fence_proxy_async_smem();                   // the stores above are read by TMA
       ptx::mbar_arrive(&bars->written[stage]);
+      ptx::cp_async_wait_all();                        // this thread's copies of the next tile's s, b have landed
+      ptx::named_bar_sync(1, WT2_EPI_THREADS);         // ... and so have everyone's
       if (++stage == a.n_stages) { stage = 0; phase ^= 1; }
       if (++acc == WT2_ACC) { acc = 0; acc_phase ^= 1; }
       if constexpr (HAS_OUT1) {
@@ -391,24 +442,15 @@ inline bool make_tmap_words(CUtensorMap* m, const void* base, uint64_t rows, uin
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Whether the tensor-core weight-tile kernel covers this problem (otherwise the plain-ALU kernel runs).
-inline bool wtile_tc_supported(const Params& p, int mode) {
-  if (p.rank % 8 != 0 || p.rank > 64) return false;
-  if (mode == WT2_PACK) {
-    if (p.bits != 3 && p.bits != 4) return false;
-    const long long words = ((long long)p.d_in * p.bits) >> 5;
-    if (((long long)p.d_in * p.bits) % 32 != 0 || (words * 4) % 16 != 0) return false;   // TMA row pitch
-  }
-  return true;
-}
-
 // Shared-memory plan: LoRA operands first, then as many W0 stages as fit (a second staging buffer for
 // the extra output only if three stages still fit beside it).
 inline bool wtile_plan(WtileArgs& a, int mode) {
   const Params& p = a.p;
   a.atoms = (2 * p.rank + 31) / 32;
+  a.ngt = std::min(p.ngroups, (WT2_COLS - 1) / p.group + 2);
   a.out_bytes = mode == WT2_DEQUANT_F ? WT2_STAGE_BYTES : mode == WT2_PACK ? WT2_ROWS * (WT2_COLS * p.bits / 8) : 0;
-  const long long budget = 227 * 1024 - 1024 - (long long)sizeof(WtileBarriers) - 2LL * a.atoms * WT2_ATOM_BYTES;
+  const long long budget = 227 * 1024 - 1024 - (long long)sizeof(WtileBarriers) - 2LL * a.atoms * WT2_ATOM_BYTES -
+                           (long long)wtile_sb_bytes(a.ngt);
   a.n_out = a.out_bytes ? 2 : 0;
   long long stages = (budget - (long long)a.n_out * a.out_bytes) / WT2_STAGE_BYTES;
   if (a.n_out == 2 && stages < 3) {
@@ -418,6 +460,19 @@ inline bool wtile_plan(WtileArgs& a, int mode) {
   if (stages < 2) return false;
   a.n_stages = (int)std::min<long long>(stages, WT2_MAX_STAGES);
   return true;
+}
+
+// Whether the tensor-core weight-tile kernel covers this problem (otherwise the plain-ALU kernel runs).
+inline bool wtile_tc_supported(const Params& p, int mode) {
+  if (p.rank % 8 != 0 || p.rank > 64) return false;
+  if (mode == WT2_PACK) {
+    if (p.bits != 3 && p.bits != 4) return false;
+    const long long words = ((long long)p.d_in * p.bits) >> 5;
+    if (((long long)p.d_in * p.bits) % 32 != 0 || (words * 4) % 16 != 0) return false;   // TMA row pitch
+  }
+  WtileArgs a{};
+  a.p = p;
+  return wtile_plan(a, mode);                       // the shared-memory plan must fit (rank 64 with the factor output does not)
 }
 
 // mode WT2_DEQUANT: out0 = W_q.  WT2_DEQUANT_F: out0 = W_q, out1 = STE factors.  WT2_PACK: out0 = codes.
