@@ -74,7 +74,7 @@ def peaks() -> dict:
 class ClockSampler:
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, device_index: int, period_s: float = 0.02):
+    def __init__(self, device_index: int, period_s: float = 0.005):
         self.samples, self.reasons = [], set()
         self.max_mhz = None
         self._stop = threading.Event()
@@ -313,7 +313,8 @@ def run_ours(args, layers, wl_name):
         G = c.d_in // c.group_size
         small = 4.0 * c.rank * (c.d_in + c.d_out)
         pack_bytes += c.d_out * c.d_in * (2 + c.bits / 8) + c.d_out * G * 12 + small
-        deq_bytes += 2 * (c.d_out * c.d_in * 4 + c.d_out * G * 8 + small)      # two launches per step (fwd, bwd)
+        # two launches per step: forward (W0 in, W_q out) and backward (W0 in, W_q and the fp16 STE factors out)
+        deq_bytes += (c.d_out * c.d_in * 4 + c.d_out * G * 8 + small) + (c.d_out * c.d_in * 6 + c.d_out * G * 8 + small)
     kernels = {}
     for name, (n, ms) in prof.items():
         if n:
@@ -381,7 +382,7 @@ def run_ours(args, layers, wl_name):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="llama7b_mlp", choices=sorted(workloads()))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -1,0 +1,141 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times
+(same entry points, same workspace, whole layer in one call), on outputs the fp64
+oracle can compute one slice at a time:
+
+  * a sample of weight rows  -> codes (bit-exact up to in-band ties), Y on a token
+    sample, and ds, db, dB of those rows over ALL tokens;
+  * one group-aligned slice of weight columns -> dX on a token sample and dA of
+    those columns over ALL tokens and ALL rows.
+
+Restricting the oracle to a row slice (W0, B, s, b rows; dY columns) or to a column
+slice made of whole quantization groups (W0, A, X columns; s, b groups) reproduces
+exactly the corresponding entries of the full result: every output entry checked
+here is a sum over the untouched dimension only.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import l4q_oracle as orc
+from paper_2402_04902_b200 import binding as l4q
+from paper_2402_04902_b200 import synth
+
+import gpu_harness as gh
+import parity_utils as pu
+
+pytestmark = pytest.mark.gpu
+
+N_TOKEN_SAMPLE = 192
+
+
+def _row_sample(d_out):
+    """Two blocks at tile boundaries (first rows, last rows) and one in the middle."""
+    mid = (d_out // 2 // 8) * 8 + 3
+    rows = list(range(0, 24)) + list(range(mid, mid + 16)) + list(range(d_out - 24, d_out))
+    return np.array(sorted(set(rows)), dtype=np.int64)
+
+
+def _run_full(cfg, arrays):
+    d = l4q.to_device(cfg, arrays)
+    desc = l4q.make_desc(cfg)
+    outs = l4q.alloc_outputs(cfg)
+    pk = l4q.alloc_pack_outputs(cfg)
+    ws = l4q.alloc_workspace(desc, l4q.L4Q_OP_BWD)
+    l4q.l4q_linear_fwd(desc, d["X"], d["W0"], d["A"], d["B"], d["s"], d["b"], outs["Y"], ws)
+    l4q.l4q_linear_bwd(desc, d["X"], d["dY"], d["W0"], d["A"], d["B"], d["s"], d["b"],
+                       outs["dX"], outs["dA"], outs["dB"], outs["ds"], outs["db"], ws)
+    l4q.l4q_pack_int(desc, d["W0"], d["A"], d["B"], d["s"], d["b"], pk["codes"], pk["s16"], pk["b16"])
+    l4q.l4q_check()
+    return outs, pk
+
+
+def _check_full_size(cfg, seed=0, layer_id=0):
+    gh.ensure_built()
+    arrays = synth.make_layer_inputs(cfg, seed=seed, layer_id=layer_id)
+    outs, pk = _run_full(cfg, arrays)
+    spec = pu.spec_of(cfg)
+    qn, _ = orc.grid_bounds(spec)
+    g = cfg.group_size
+    rng = np.random.default_rng(1234)
+    tok = np.sort(rng.choice(cfg.tokens, size=N_TOKEN_SAMPLE, replace=False))
+    A64 = arrays["A"].astype(np.float64)
+    X64 = arrays["X"].astype(np.float64)
+
+    # ---------------- row slice ----------------
+    rows = _row_sample(cfg.d_out)
+    W0r = arrays["W0"][rows].astype(np.float64)
+    Br = arrays["B"][rows].astype(np.float64)
+    sr = arrays["s"][rows].astype(np.float64)
+    br = arrays["b"][rows].astype(np.float64)
+    w = orc.prequant(spec, orc.merge(spec, W0r, A64, Br), sr, br)
+    got_u = orc.unpack_int(spec, pk["codes"][torch.from_numpy(rows).cuda()].cpu().numpy().view(np.uint32), cfg.d_in)
+    res = pu.check_codes(got_u, spec, w)
+    print(cfg.name, "codes on", rows.size, "rows:", res)
+    assert res["out_of_band"] == 0, res
+    assert res["mismatches"] <= max(1.0, res["allowed"]), res
+    codes_r = got_u + qn
+    s16_ref, b16_ref = orc.pack_int(spec, W0r, A64, Br, sr, br)[1:]
+    ridx = torch.from_numpy(rows).cuda()
+    assert np.array_equal(pk["s16"][ridx].cpu().numpy().view(np.uint16), s16_ref.view(np.uint16))
+    assert np.array_equal(pk["b16"][ridx].cpu().numpy().view(np.uint16), b16_ref.view(np.uint16))
+
+    Y_ref = orc.forward(spec, X64[tok], W0r, A64, Br, sr, br, bf16_reference=True, codes=codes_r)
+    Y_got = outs["Y"][torch.from_numpy(tok).cuda()][:, ridx].double().cpu().numpy()
+    dYr = arrays["dY"][:, rows].astype(np.float64)
+    g_rows = orc.backward(spec, X64, dYr, W0r, A64, Br, sr, br, bf16_reference=True, codes=codes_r)
+    errs = {"Y": pu.max_rel_err(Y_got, Y_ref)}
+    for k in ("ds", "db", "dB"):
+        errs[k] = pu.rel_l2(outs[k][ridx].double().cpu().numpy(), g_rows[k])
+    del dYr, g_rows
+
+    # ---------------- column slice: whole groups covering >= 128 columns, away from column 0 ----------------
+    ncols = g * max(1, 128 // g)
+    c0 = (cfg.d_in // 2 // g) * g
+    cols = np.arange(c0, c0 + ncols)
+    gcols = np.arange(c0 // g, (c0 + ncols) // g)
+    W0c = arrays["W0"][:, cols].astype(np.float64)
+    Ac = A64[:, cols]
+    sc = arrays["s"][:, gcols].astype(np.float64)
+    bc = arrays["b"][:, gcols].astype(np.float64)
+    B64 = arrays["B"].astype(np.float64)
+    wc = orc.prequant(spec, orc.merge(spec, W0c, Ac, B64), sc, bc)
+    all_codes = orc.unpack_int(spec, pk["codes"].cpu().numpy().view(np.uint32), cfg.d_in)[:, cols]
+    res_c = pu.check_codes(all_codes, spec, wc)
+    print(cfg.name, "codes on", cols.size, "columns:", res_c)
+    assert res_c["out_of_band"] == 0, res_c
+    assert res_c["mismatches"] <= max(1.0, res_c["allowed"]), res_c
+    codes_c = all_codes + qn
+    dY64 = arrays["dY"].astype(np.float64)
+    g_cols = orc.backward(spec, X64[:, cols], dY64, W0c, Ac, B64, sc, bc, bf16_reference=True, codes=codes_c)
+    cidx = torch.from_numpy(cols).cuda()
+    errs["dX"] = pu.max_rel_err(outs["dX"][torch.from_numpy(tok).cuda()][:, cidx].double().cpu().numpy(),
+                                g_cols["dX"][tok])
+    errs["dA"] = pu.rel_l2(outs["dA"][:, cidx].double().cpu().numpy(), g_cols["dA"])
+    # the same slice also gives ds, db of every row for these groups
+    gidx = torch.from_numpy(gcols).cuda()
+    errs["ds_cols"] = pu.rel_l2(outs["ds"][:, gidx].double().cpu().numpy(), g_cols["ds"])
+    errs["db_cols"] = pu.rel_l2(outs["db"][:, gidx].double().cpu().numpy(), g_cols["db"])
+
+    print(cfg.name, {k: f"{v:.2e}" for k, v in errs.items()})
+    assert errs["Y"] <= pu.TOL_OUT["bf16"], errs
+    assert errs["dX"] <= pu.TOL_OUT["bf16"], errs
+    for k in ("ds", "db", "dB", "dA", "ds_cols", "db_cols"):
+        assert errs[k] <= pu.TOL_GRAD["bf16"], errs
+
+
+def test_full_size_llama7b_attention_projection():       # config 2
+    _check_full_size(synth.CONFIG2)
+
+
+def test_full_size_llama7b_mlp_up():                     # config 3, 4096 -> 11008
+    _check_full_size(synth.CONFIG3A)
+
+
+def test_full_size_llama7b_mlp_down_3bit_rank64():       # config 4, 11008 -> 4096, 3-bit, group 64, rank 64
+    _check_full_size(synth.CONFIG4B, layer_id=1)
+
+
+def test_full_size_mistral_kv_projection():              # config 5: the narrow GQA projection 4096 -> 1024
+    layers = synth.mistral_block_layers()
+    kv = min(layers, key=lambda c: c.d_out)
+    _check_full_size(kv, layer_id=layers.index(kv))
