@@ -309,7 +309,7 @@ def run_ours(args, layers, wl_name):
         mm = 2.0 * c.tokens * c.d_out * c.d_in
         gemm_flops["gemm_fwd"] += mm
         gemm_flops["gemm_dgrad"] += mm
-        gemm_flops["gemm_wgrad"] += mm + 6.0 * c.d_out * c.d_in * c.rank
+        gemm_flops["gemm_wgrad"] += mm + 4.0 * c.d_out * c.d_in * c.rank      # G tiles + the dA, dB contractions
         G = c.d_in // c.group_size
         small = 4.0 * c.rank * (c.d_in + c.d_out)
         pack_bytes += c.d_out * c.d_in * (2 + c.bits / 8) + c.d_out * G * 12 + small
