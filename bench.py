@@ -195,6 +195,7 @@ def run_ours(args, layers, wl_name):
 
     from paper_2402_04902_b200 import binding as l4q
     from paper_2402_04902_b200 import build as l4q_build
+    from paper_2402_04902_b200 import dp
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -243,8 +244,7 @@ def run_ours(args, layers, wl_name):
                                o["dX"], o["dA"], o["dB"], o["ds"], o["db"], l["ws"])
             l4q.l4q_pack_int(l["desc"], d["W0"], d["A"], d["B"], d["s"], d["b"], pk["codes"], pk["s16"], pk["b16"])
             if world > 1:
-                for k in ("dA", "dB", "ds", "db"):
-                    dist.all_reduce(o[k])
+                dp.allreduce_param_grads(o)
             if e2e:
                 for k in ("dA", "dB", "ds", "db"):
                     l["grads_host"][k].copy_(o[k], non_blocking=True)
