@@ -49,6 +49,7 @@ struct WtileArgs {
   int out_bytes;           // bytes of one such buffer
   int atoms;               // swizzle atoms per operand row: ceil(2 rank / 32)
   int ngt;                 // upper bound of the quantization groups a 128-column tile intersects
+  int n_opbuf;             // MMA operand buffers ([A slice | B slice] each): 2 up to rank 32, else 1
 };
 
 struct __align__(8) WtileBarriers {
@@ -56,7 +57,7 @@ struct __align__(8) WtileBarriers {
   uint64_t empty[WT2_MAX_STAGES];     // the stage may be overwritten (its store has read it)
   uint64_t written[WT2_MAX_STAGES];   // the epilogue has written the stage's outputs
   uint64_t out_empty[2];              // second-output staging buffer may be overwritten
-  uint64_t prep_full;                 // split LoRA operands of the next tile are in shared memory
+  uint64_t prep_full[2];              // split LoRA operands are complete in operand buffer b
   uint64_t tmem_full[WT2_ACC], tmem_empty[WT2_ACC];
   uint32_t tmem_base;
   volatile uint32_t abort;
@@ -67,17 +68,36 @@ __host__ __device__ inline size_t wtile_sb_bytes(int ngt) { return 2 * (size_t)W
 
 inline size_t wtile_smem_bytes(const WtileArgs& a) {
   return 1024 + (size_t)a.n_stages * WT2_STAGE_BYTES + (size_t)a.n_out * a.out_bytes +
-         2 * (size_t)a.atoms * WT2_ATOM_BYTES + wtile_sb_bytes(a.ngt) + sizeof(WtileBarriers);
+         2 * (size_t)a.n_opbuf * a.atoms * WT2_ATOM_BYTES + wtile_sb_bytes(a.ngt) + sizeof(WtileBarriers);
 }
 
-// Tile i of this CTA: row tiles of one column panel go to neighbouring CTAs.
-__device__ __forceinline__ bool wtile_coords(const WtileArgs& a, int i, int& m0, int& n0) {
-  const int t = blockIdx.x + i * gridDim.x;
-  if (t >= a.tiles_m * a.tiles_n) return false;
-  m0 = (t % a.tiles_m) * WT2_ROWS;
-  n0 = (t / a.tiles_m) * WT2_COLS;
-  return true;
-}
+// The tiles of one CTA: tile t of the column-panel-major sequence (row tiles of one column panel are
+// consecutive) goes to CTA t mod gridDim.x.  Coordinates advance without divisions.
+struct TileCursor {
+  int t, total, tm, tn, tiles_m, dm, dn;
+  __device__ explicit TileCursor(const WtileArgs& a) {
+    total = a.tiles_m * a.tiles_n;
+    tiles_m = a.tiles_m;
+    t = blockIdx.x;
+    tn = t / tiles_m; tm = t - tn * tiles_m;
+    dn = (int)gridDim.x / tiles_m; dm = (int)gridDim.x - dn * tiles_m;
+  }
+  __device__ bool valid() const { return t < total; }
+  __device__ void next() {
+    t += gridDim.x; tn += dn; tm += dm;
+    if (tm >= tiles_m) { tm -= tiles_m; ++tn; }
+  }
+  __device__ int m0() const { return tm * WT2_ROWS; }
+  __device__ int n0() const { return tn * WT2_COLS; }
+  // coordinates of this CTA's tile k (small) steps ahead; false beyond the end
+  __device__ bool peek(int k, int& m0_, int& n0_) const {
+    if (t + k * (int)gridDim.x >= total) return false;
+    int m = tm + k * dm, n = tn + k * dn;
+    while (m >= tiles_m) { m -= tiles_m; ++n; }
+    m0_ = m * WT2_ROWS; n0_ = n * WT2_COLS;
+    return true;
+  }
+};
 
 // x = hi + lo with hi, lo representable in tf32 (low 13 mantissa bits clear): hi keeps the leading 10
 // mantissa bits of x (truncation), lo the leading bits of the exact remainder.  Plain logic ops.
@@ -86,54 +106,47 @@ __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
   lo = __uint_as_float(__float_as_uint(x - hi) & 0xFFFFE000u);
 }
 
-// Builds the split operands of one tile in shared memory, K-major with the 128-byte swizzle:
+// MMA operands of one tile in shared memory, K-major with the 128-byte swizzle:
 //   acat row n = column n0 + n of the weight:  [ hi(A[0..r, col]) | lo(A[0..r, col]) ]
 //   bcat row m = row m0 + m of the weight:      [ hi(B[row, 0..r]) | lo(B[row, 0..r]) ]
-// A work item is 4 consecutive ranks of one row; a warp takes 32 consecutive rows of the same ranks, so
-// its reads of A are coalesced and its 16-byte shared-memory writes are conflict-free.
-__device__ __forceinline__ void wtile_prep_operands(const WtileArgs& a, int m0, int n0, int et, uint8_t* acat,
-                                                    uint8_t* bcat) {
+// A work item is 4 consecutive ranks (kc) of one row of both slices (32 r items per tile); a warp takes 32
+// consecutive rows of the same ranks, so its reads of A are coalesced and its 16-byte shared-memory writes
+// are conflict-free.
+struct OperandItem { float av[4]; float4 bv; };
+
+__device__ __forceinline__ void operand_item_load(const WtileArgs& a, int m0, int n0, int idx, OperandItem& it) {
   const Params& p = a.p;
-  const int r = p.rank;
-  for (int idx = et; idx < 32 * r; idx += WT2_EPI_THREADS) {
-    const int row = idx & 127, kc = idx >> 7;        // ranks 4 kc .. 4 kc + 3
-    float av[4] = {0.f, 0.f, 0.f, 0.f};
-    const int col = n0 + row;
-    if (col < p.d_in) {
+  const int row = idx & 127, kc = idx >> 7, col = n0 + row;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) av[e] = __ldg(a.A + (size_t)(4 * kc + e) * p.d_in + col);
-    }
-    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (m0 + row < p.d_out) bv = __ldg(reinterpret_cast<const float4*>(a.B + (size_t)(m0 + row) * r + 4 * kc));
-    const float bvv[4] = {bv.x, bv.y, bv.z, bv.w};
-    float ah[4], al[4], bh[4], bl[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      split_tf32(av[e], ah[e], al[e]);
-      split_tf32(bvv[e], bh[e], bl[e]);
-    }
-    const int ch = kc, cl = (r >> 2) + kc;           // 16-byte chunk index of the head / tail within the row
-    const uint32_t off_h = (uint32_t)(ch >> 3) * WT2_ATOM_BYTES + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
-    const uint32_t off_l = (uint32_t)(cl >> 3) * WT2_ATOM_BYTES + row * 128 + (((cl & 7) ^ (row & 7)) << 4);
-    *reinterpret_cast<float4*>(acat + off_h) = make_float4(ah[0], ah[1], ah[2], ah[3]);
-    *reinterpret_cast<float4*>(acat + off_l) = make_float4(al[0], al[1], al[2], al[3]);
-    *reinterpret_cast<float4*>(bcat + off_h) = make_float4(bh[0], bh[1], bh[2], bh[3]);
-    *reinterpret_cast<float4*>(bcat + off_l) = make_float4(bl[0], bl[1], bl[2], bl[3]);
-  }
+  for (int e = 0; e < 4; ++e) it.av[e] = (col < p.d_in) ? __ldg(a.A + (size_t)(4 * kc + e) * p.d_in + col) : 0.f;
+  it.bv = (m0 + row < p.d_out) ? __ldg(reinterpret_cast<const float4*>(a.B + (size_t)(m0 + row) * p.rank + 4 * kc))
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
-// 32 unsigned codes -> bitstream words, code j at bit j * BITS (LSB first).
-template <int BITS>
-__device__ __forceinline__ void pack_codes32(const uint32_t (&u)[32], uint32_t (&w)[BITS]) {
+__device__ __forceinline__ void operand_item_store(const WtileArgs& a, int idx, const OperandItem& it, uint8_t* acat,
+                                                   uint8_t* bcat) {
+  const int row = idx & 127, kc = idx >> 7;
+  const float bvv[4] = {it.bv.x, it.bv.y, it.bv.z, it.bv.w};
+  float ah[4], al[4], bh[4], bl[4];
 #pragma unroll
-  for (int i = 0; i < BITS; ++i) w[i] = 0u;
-#pragma unroll
-  for (int j = 0; j < 32; ++j) {
-    const int bit = j * BITS, word = bit >> 5, off = bit & 31;
-    w[word] |= u[j] << off;
-    if (off + BITS > 32) w[word + 1] |= u[j] >> (32 - off);
+  for (int e = 0; e < 4; ++e) {
+    split_tf32(it.av[e], ah[e], al[e]);
+    split_tf32(bvv[e], bh[e], bl[e]);
   }
+  const int ch = kc, cl = (a.p.rank >> 2) + kc;      // 16-byte chunk index of the head / tail within the row
+  const uint32_t off_h = (uint32_t)(ch >> 3) * WT2_ATOM_BYTES + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
+  const uint32_t off_l = (uint32_t)(cl >> 3) * WT2_ATOM_BYTES + row * 128 + (((cl & 7) ^ (row & 7)) << 4);
+  *reinterpret_cast<float4*>(acat + off_h) = make_float4(ah[0], ah[1], ah[2], ah[3]);
+  *reinterpret_cast<float4*>(acat + off_l) = make_float4(al[0], al[1], al[2], al[3]);
+  *reinterpret_cast<float4*>(bcat + off_h) = make_float4(bh[0], bh[1], bh[2], bh[3]);
+  *reinterpret_cast<float4*>(bcat + off_l) = make_float4(bl[0], bl[1], bl[2], bl[3]);
 }
+
+// Adding and subtracting 1.5 * 2^23 rounds |x| < 2^22 to the nearest integer, ties to even, exactly like
+// rintf, on the FP32 add pipe; the low mantissa bits of the intermediate sum hold that integer.
+constexpr float kRoundMagic = 12582912.0f;
+constexpr int kRoundMagicBits = 0x4B400000;
+constexpr int WT2_CARRY = 2;                        // operand items a thread carries between tiles (rank <= 32)
 
 template <int MODE>
 __global__ void __launch_bounds__(WT2_THREADS, 1)
@@ -145,9 +158,9 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
   uint8_t* out_base = stage_base + (size_t)a.n_stages * WT2_STAGE_BYTES;
-  uint8_t* acat = out_base + (size_t)a.n_out * a.out_bytes;
-  uint8_t* bcat = acat + (size_t)a.atoms * WT2_ATOM_BYTES;
-  float* sb_base = reinterpret_cast<float*>(bcat + (size_t)a.atoms * WT2_ATOM_BYTES);
+  uint8_t* op_base = out_base + (size_t)a.n_out * a.out_bytes;          // operand buffer b: [acat | bcat]
+  const uint32_t op_half = (uint32_t)a.atoms * WT2_ATOM_BYTES;           // bytes of one acat or bcat
+  float* sb_base = reinterpret_cast<float*>(op_base + (size_t)a.n_opbuf * 2 * op_half);
   WtileBarriers* bars = reinterpret_cast<WtileBarriers*>(reinterpret_cast<uint8_t*>(sb_base) + wtile_sb_bytes(a.ngt));
   const Params& p = a.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -160,7 +173,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       ptx::mbar_init(&bars->written[i], WT2_EPI_THREADS);
     }
     for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->out_empty[i], 1);
-    ptx::mbar_init(&bars->prep_full, WT2_EPI_THREADS);
+    for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->prep_full[i], WT2_EPI_THREADS);
     for (int i = 0; i < WT2_ACC; ++i) {
       ptx::mbar_init(&bars->tmem_full[i], 1);
       ptx::mbar_init(&bars->tmem_empty[i], WT2_EPI_THREADS);
@@ -184,8 +197,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     // ------------------------------ TMA loads of W0 ---------------------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      int m0, n0;
-      for (int i = 0; !bars->abort && wtile_coords(a, i, m0, n0); ++i) {
+      for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next()) {
+        const int m0 = cur.m0(), n0 = cur.n0();
         bounded_wait(&bars->empty[stage], phase ^ 1, bars);
         if (bars->abort) break;
         uint8_t* dst = stage_base + (size_t)stage * WT2_STAGE_BYTES;
@@ -200,12 +213,12 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     // ------------------------------ merge MMAs --------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc = ptx::make_idesc_tf32(WT2_ROWS, WT2_COLS);
-      const uint32_t acat_a = ptx::smem_u32(acat), bcat_a = ptx::smem_u32(bcat);
       const int r = p.rank, ksteps = r >> 3;
       int acc = 0; uint32_t acc_phase = 0;
-      int m0, n0;
-      for (int i = 0; !bars->abort && wtile_coords(a, i, m0, n0); ++i) {
-        bounded_wait(&bars->prep_full, (uint32_t)(i & 1), bars);
+      int buf = 0; uint32_t buf_phase = 0;
+      for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next()) {
+        const uint32_t acat_a = ptx::smem_u32(op_base) + (uint32_t)buf * 2 * op_half, bcat_a = acat_a + op_half;
+        bounded_wait(&bars->prep_full[buf], buf_phase, bars);
         bounded_wait(&bars->tmem_empty[acc], acc_phase ^ 1, bars);
         if (bars->abort) break;
         ptx::tc_fence_after_sync();
@@ -226,6 +239,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
         }
         ptx::mma_commit(&bars->tmem_full[acc]);
         if (++acc == WT2_ACC) { acc = 0; acc_phase ^= 1; }
+        if (++buf == a.n_opbuf) { buf = 0; buf_phase ^= 1; }
       }
     }
     __syncwarp();
@@ -234,8 +248,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       int ob = 0;
-      int m0, n0;
-      for (int i = 0; !bars->abort && wtile_coords(a, i, m0, n0); ++i) {
+      for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next()) {
+        const int m0 = cur.m0(), n0 = cur.n0();
         bounded_wait(&bars->written[stage], phase, bars);
         if (bars->abort) break;
         const uint8_t* src = stage_base + (size_t)stage * WT2_STAGE_BYTES;
@@ -271,12 +285,40 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     int stage = 0; uint32_t phase = 0;
     int acc = 0; uint32_t acc_phase = 0;
-    int ob = 0; uint32_t out_round = 0;                         // uses of staging buffer `ob` so far
-    int m0, n0;
-    // s and b reach the arithmetic through shared memory: the four warps of column slice 0 (one thread
-    // per weight row) copy the tile's values of their row, one tile ahead, with asynchronous 4-byte
-    // copies; all epilogue threads meet at a barrier at the end of every tile.  (Loading them per thread
-    // would touch 32 different lines per instruction, sixteen times over, and starve the TMA loads.)
+    int ob = 0; uint32_t out_round = 0;                         // completed rounds over the staging buffers
+    const int r = p.rank;
+    const int L = a.n_opbuf;
+    const int n_items = 32 * r;                                 // (row, 4 ranks) operand items per tile
+
+    // ---- MMA operands.  Two buffers (rank <= 32): the factors of tile i + 2 are loaded one tile before they
+    //      are stored, so the merge runs two tiles ahead and no load latency is exposed.  One buffer: the
+    //      operands of tile i + 1 are loaded and stored once the MMAs of tile i have completed. ----
+    auto prep_now = [&](int m0_, int n0_, int buf) {
+      uint8_t* acat = op_base + (size_t)buf * 2 * op_half;
+      for (int idx = et; idx < n_items; idx += WT2_EPI_THREADS) {
+        OperandItem it_;
+        operand_item_load(a, m0_, n0_, idx, it_);
+        operand_item_store(a, idx, it_, acat, acat + op_half);
+      }
+    };
+    OperandItem carry[WT2_CARRY];
+    auto carry_load = [&](int m0_, int n0_) {
+#pragma unroll
+      for (int j = 0; j < WT2_CARRY; ++j)
+        if (et + j * WT2_EPI_THREADS < n_items) operand_item_load(a, m0_, n0_, et + j * WT2_EPI_THREADS, carry[j]);
+    };
+    auto carry_store = [&](int buf) {
+      uint8_t* acat = op_base + (size_t)buf * 2 * op_half;
+#pragma unroll
+      for (int j = 0; j < WT2_CARRY; ++j)
+        if (et + j * WT2_EPI_THREADS < n_items)
+          operand_item_store(a, et + j * WT2_EPI_THREADS, carry[j], acat, acat + op_half);
+    };
+
+    // ---- s and b reach the arithmetic through shared memory: the four warps of column slice 0 (one thread
+    //      per weight row) copy the tile's values of their row, one tile ahead, with asynchronous 4-byte
+    //      copies; all epilogue threads meet at a barrier at the end of every tile.  (Loading them per thread
+    //      touches 32 different lines per instruction, sixteen times over, and starves the TMA loads.) ----
     const int sbw = 2 * a.ngt;                                  // floats per row: s x ngt | b x ngt
     auto stage_sb = [&](int m0_, int n0_, int buf) {
       if (sl != 0) return;
@@ -294,55 +336,77 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
       ptx::cp_async_commit();
     };
-    if (wtile_coords(a, 0, m0, n0)) {
-      stage_sb(m0, n0, 0);
-      wtile_prep_operands(a, m0, n0, et, acat, bcat);
-      ptx::fence_proxy_async_smem();
-      ptx::mbar_arrive(&bars->prep_full);
+
+    // ---- quantization groups of the four 8-column pieces this thread owns (g % 8 == 0: one group each).
+    //      They depend on the tile's column only and are recomputed when it changes. ----
+    int gi[4] = {0, 0, 0, 0};                                   // group index relative to the tile's first group
+    uint32_t first_mask = 0, valid_mask = 0;                    // bit sub: first piece of its group / inside d_in
+    int g_first = 0, groups_n0 = -1;
+    auto set_groups = [&](int n0_) {
+      const int jc = n0_ + sl * 32;
+      g_first = n0_ / p.group;
+      const int g0 = jc / p.group;
+      const int rem0 = jc - g0 * p.group;
+      first_mask = 0; valid_mask = 0;
+#pragma unroll
+      for (int sub = 0; sub < 4; ++sub) {
+        int rem = rem0 + sub * 8, g = g0;
+#pragma unroll
+        for (int c = 0; c < 3; ++c)
+          if (rem >= p.group) { rem -= p.group; ++g; }
+        gi[sub] = g - g_first;
+        if (rem == 0) first_mask |= 1u << sub;
+        if (jc + sub * 8 < p.d_in) valid_mask |= 1u << sub;
+      }
+      groups_n0 = n0_;
+    };
+
+    // ------------------------------ prologue ------------------------------
+    TileCursor cur(a);
+    {
+      int mb, nb;
+      if (cur.valid()) stage_sb(cur.m0(), cur.n0(), 0);
+      for (int k = 0; k < L; ++k) {
+        if (cur.peek(k, mb, nb)) {
+          prep_now(mb, nb, k);
+          ptx::fence_proxy_async_smem();
+          ptx::mbar_arrive(&bars->prep_full[k]);
+        }
+      }
+      if (L == 2 && cur.peek(2, mb, nb)) carry_load(mb, nb);
       ptx::cp_async_wait_all();
     }
     ptx::named_bar_sync(1, WT2_EPI_THREADS);
-    for (int i = 0; wtile_coords(a, i, m0, n0); ++i) {
+    const int qn_bits = kRoundMagicBits + (int)p.qn;
+
+    for (int i = 0; cur.valid(); cur.next(), ++i) {
+      const int m0 = cur.m0(), n0 = cur.n0();
       const int o = m0 + row;
       const bool row_ok = o < p.d_out;
-      const int jc = n0 + sl * 32;
+      if (n0 != groups_n0) set_groups(n0);
       float sv[4], bv[4];
-      int grp[4];
-      uint32_t first_mask = 0;                                  // bit sub: the piece is the first of its group
       {
-        const int g_first = n0 / p.group;
-        const int g0 = jc / p.group;
-        const int rem0 = jc - g0 * p.group;
         const float* src = sb_base + ((size_t)(i & 1) * WT2_ROWS + row) * sbw;
 #pragma unroll
         for (int sub = 0; sub < 4; ++sub) {
-          int rem = rem0 + sub * 8, g = g0;
-#pragma unroll
-          for (int c = 0; c < 3; ++c)
-            if (rem >= p.group) { rem -= p.group; ++g; }
-          const bool ok = row_ok && jc + sub * 8 < p.d_in;
-          grp[sub] = ok ? g : -1;
-          if (rem == 0) first_mask |= 1u << sub;
-          sv[sub] = ok ? src[g - g_first] : 1.f;
-          bv[sub] = ok ? src[a.ngt + g - g_first] : 0.f;
+          const bool ok = row_ok && ((valid_mask >> sub) & 1u);
+          sv[sub] = ok ? src[gi[sub]] : 1.f;
+          bv[sub] = ok ? src[a.ngt + gi[sub]] : 0.f;
         }
       }
       bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
       ptx::tc_fence_after_sync();
-      {  // the MMAs of this tile have completed: their operands may be replaced by the next tile's
+      {  // the MMAs of this tile have completed: its operand buffer is free for the tile L steps ahead
         int m1, n1;
-        if (wtile_coords(a, i + 1, m1, n1)) {
-          stage_sb(m1, n1, (i + 1) & 1);
-          wtile_prep_operands(a, m1, n1, et, acat, bcat);
+        const int buf = i % L;
+        if (cur.peek(L, m1, n1)) {
+          if (L == 2) carry_store(buf); else prep_now(m1, n1, 0);
           ptx::fence_proxy_async_smem();
-          ptx::mbar_arrive(&bars->prep_full);
+          ptx::mbar_arrive(&bars->prep_full[buf]);
         }
+        if (L == 2 && cur.peek(3, m1, n1)) carry_load(m1, n1);
+        if (cur.peek(1, m1, n1)) stage_sb(m1, n1, (i + 1) & 1);
       }
-      uint32_t raw[32];
-      ptx::tmem_ld_32x32(tmem_base + lane_base + (uint32_t)(acc * WT2_COLS + sl * 32), raw);
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before_sync();
-      ptx::mbar_arrive(&bars->tmem_empty[acc]);
 
       bounded_wait(&bars->full[stage], phase, bars);
       if constexpr (HAS_OUT1) {
@@ -350,55 +414,82 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
       uint8_t* wrow = stage_base + (size_t)stage * WT2_STAGE_BYTES + (sl >> 1) * (WT2_STAGE_BYTES / 2) + row * 128;
       [[maybe_unused]] uint8_t* out1 = out_base + (size_t)ob * a.out_bytes;
-      [[maybe_unused]] uint32_t ucodes[32];
+      [[maybe_unused]] uint32_t words[4] = {0u, 0u, 0u, 0u};    // WT2_PACK: this thread's 32 codes
       float rs = 1.f;
 #pragma unroll
-      for (int sub = 0; sub < 4; ++sub) {
-        const uint32_t chunk = (uint32_t)((((sl & 1) * 4 + sub) ^ (row & 7)) << 4);
-        const uint4 wr = *reinterpret_cast<const uint4*>(wrow + chunk);
-        const float w0[8] = {bf16_lo(wr.x), bf16_hi(wr.x), bf16_lo(wr.y), bf16_hi(wr.y),
-                             bf16_lo(wr.z), bf16_hi(wr.z), bf16_lo(wr.w), bf16_hi(wr.w)};
-        if (sub == 0 || ((first_mask >> sub) & 1u)) rs = 1.0f / sv[sub];         // one reciprocal per group
-        float wq[8], fac[8];
+      for (int half = 0; half < 2; ++half) {                    // 16 columns at a time
+        uint32_t raw[16];
+        ptx::tmem_ld_32x16(tmem_base + lane_base + (uint32_t)(acc * WT2_COLS + sl * 32 + half * 16), raw);
+        ptx::tmem_ld_wait();
+        if (half == 1) {
+          ptx::tc_fence_before_sync();
+          ptx::mbar_arrive(&bars->tmem_empty[acc]);
+        }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const QuantElem q = quantize_elem(merge_elem(w0[e], __uint_as_float(raw[sub * 8 + e]), p.gamma), sv[sub], rs,
-                                            bv[sub], p.qn, p.qp);
-          wq[e] = q.wq;
-          fac[e] = ste_factor(q, p.qn, p.qp);
-          if constexpr (MODE == WT2_PACK) ucodes[sub * 8 + e] = (uint32_t)(int)(q.code - p.qn);
-        }
-        if constexpr (MODE != WT2_PACK) {
-          uint4 o4;
-          o4.x = pack_bf16x2(wq[0], wq[1]); o4.y = pack_bf16x2(wq[2], wq[3]);
-          o4.z = pack_bf16x2(wq[4], wq[5]); o4.w = pack_bf16x2(wq[6], wq[7]);
-          *reinterpret_cast<uint4*>(wrow + chunk) = o4;                       // in place, same swizzled position
-        }
-        if constexpr (MODE == WT2_DEQUANT_F) {
-          __half2 h[4];
+        for (int s2 = 0; s2 < 2; ++s2) {
+          const int sub = half * 2 + s2;
+          const uint32_t chunk = (uint32_t)((((sl & 1) * 4 + sub) ^ (row & 7)) << 4);
+          const uint4 wr = *reinterpret_cast<const uint4*>(wrow + chunk);
+          const float w0[8] = {bf16_lo(wr.x), bf16_hi(wr.x), bf16_lo(wr.y), bf16_hi(wr.y),
+                               bf16_lo(wr.z), bf16_hi(wr.z), bf16_lo(wr.w), bf16_hi(wr.w)};
+          if (sub == 0 || ((first_mask >> sub) & 1u)) rs = 1.0f / sv[sub];        // one reciprocal per group
+          const float s_ = sv[sub], b_ = bv[sub];
+          float wq[8], fac[8];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) h[e] = __floats2half2_rn(fac[2 * e], fac[2 * e + 1]);
-          *reinterpret_cast<uint4*>(out1 + (sl >> 1) * (WT2_STAGE_BYTES / 2) + row * 128 + chunk) =
-              *reinterpret_cast<const uint4*>(h);
-        }
-        if constexpr (MODE == WT2_PACK) {
-          if (grp[sub] >= 0 && ((first_mask >> sub) & 1u)) {                   // first piece of its group
-            a.s16[(size_t)o * p.ngroups + grp[sub]] = __float2half_rn(sv[sub]);
-            a.b16[(size_t)o * p.ngroups + grp[sub]] = __float2half_rn(fmaf(sv[sub], p.qn, bv[sub]));
+          for (int e = 0; e < 8; ++e) {
+            // Eq. 7-9 and the STE factor: the arithmetic of quantize_elem / ste_factor, with the rounding
+            // done by the magic-number add (exact for the clamped range)
+            const float wc = merge_elem(w0[e], __uint_as_float(raw[s2 * 8 + e]), p.gamma);
+            const float w = (wc - b_) * rs;
+            const float wcl = fminf(fmaxf(w, p.qn), p.qp);
+            const float y = wcl + kRoundMagic;
+            const float code = y - kRoundMagic;
+            wq[e] = fmaf(code, s_, b_);
+            if constexpr (MODE == WT2_DEQUANT_F) {
+              const float t = w - wcl;                                            // 0 inside [Q_N, Q_P]
+              const float sentinel = __uint_as_float((__float_as_uint(t) & 0x80000000u) | 0x40000000u);   // +-2
+              fac[e] = (fabsf(t) > kMaskGuard) ? sentinel : code - w;
+            }
+            if constexpr (MODE == WT2_PACK) {                                     // code j of 32 at bit j * bits
+              const uint32_t u = (uint32_t)(__float_as_int(y) - qn_bits);
+              const int j = sub * 8 + e;
+              if (p.bits == 4) {
+                words[j >> 3] |= u << ((j & 7) * 4);
+              } else {
+                const int bit = j * 3, wd = bit >> 5, off = bit & 31;
+                words[wd] |= u << off;
+                if (off > 29) words[wd + 1] |= u >> (32 - off);
+              }
+            }
+          }
+          if constexpr (MODE != WT2_PACK) {
+            uint4 o4;
+            o4.x = pack_bf16x2(wq[0], wq[1]); o4.y = pack_bf16x2(wq[2], wq[3]);
+            o4.z = pack_bf16x2(wq[4], wq[5]); o4.w = pack_bf16x2(wq[6], wq[7]);
+            *reinterpret_cast<uint4*>(wrow + chunk) = o4;                         // in place, same swizzled position
+          }
+          if constexpr (MODE == WT2_DEQUANT_F) {
+            __half2 h[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) h[e] = __floats2half2_rn(fac[2 * e], fac[2 * e + 1]);
+            *reinterpret_cast<uint4*>(out1 + (sl >> 1) * (WT2_STAGE_BYTES / 2) + row * 128 + chunk) =
+                *reinterpret_cast<const uint4*>(h);
+          }
+          if constexpr (MODE == WT2_PACK) {
+            if (row_ok && ((valid_mask & first_mask) >> sub) & 1u) {              // first piece of its group
+              a.s16[(size_t)o * p.ngroups + g_first + gi[sub]] = __float2half_rn(s_);
+              a.b16[(size_t)o * p.ngroups + g_first + gi[sub]] = __float2half_rn(fmaf(s_, p.qn, b_));
+            }
           }
         }
       }
       if constexpr (MODE == WT2_PACK) {
         // staging row = the tile's 128 codes of this weight row; this thread owns 32 of them
         if (p.bits == 4) {
-          uint32_t w[4];
-          pack_codes32<4>(ucodes, w);
-          *reinterpret_cast<uint4*>(out1 + row * 64 + sl * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(out1 + row * 64 + sl * 16) = make_uint4(words[0], words[1], words[2], words[3]);
         } else {
-          uint32_t w[3];
-          pack_codes32<3>(ucodes, w);
           uint32_t* dst = reinterpret_cast<uint32_t*>(out1 + row * 48 + sl * 12);
-          dst[0] = w[0]; dst[1] = w[1]; dst[2] = w[2];
+          dst[0] = words[0]; dst[1] = words[1]; dst[2] = words[2];
         }
       }
       ptx::fence_proxy_async_smem();                   // the stores above are read by TMA
@@ -448,8 +539,10 @@ inline bool wtile_plan(WtileArgs& a, int mode) {
   const Params& p = a.p;
   a.atoms = (2 * p.rank + 31) / 32;
   a.ngt = std::min(p.ngroups, (WT2_COLS - 1) / p.group + 2);
+  a.n_opbuf = (32 * p.rank <= WT2_CARRY * WT2_EPI_THREADS) ? 2 : 1;
   a.out_bytes = mode == WT2_DEQUANT_F ? WT2_STAGE_BYTES : mode == WT2_PACK ? WT2_ROWS * (WT2_COLS * p.bits / 8) : 0;
-  const long long budget = 227 * 1024 - 1024 - (long long)sizeof(WtileBarriers) - 2LL * a.atoms * WT2_ATOM_BYTES -
+  const long long budget = 227 * 1024 - 1024 - (long long)sizeof(WtileBarriers) -
+                           2LL * a.n_opbuf * a.atoms * WT2_ATOM_BYTES -
                            (long long)wtile_sb_bytes(a.ngt);
   a.n_out = a.out_bytes ? 2 : 0;
   long long stages = (budget - (long long)a.n_out * a.out_bytes) / WT2_STAGE_BYTES;
