@@ -15,11 +15,14 @@
 //   * 16 epilogue warps (thread = one weight row x 32 columns) read the merge from tensor memory with
 //     tcgen05.ld, the W0 tile from shared memory in 16-byte pieces, and do the quantizer arithmetic.
 //
-// Roles (640 threads): warp 0 = TMA loads, warp 1 = MMA issuer + TMEM owner, warp 2 = TMA stores,
-// warps 4..19 = epilogue (warp w: TMEM lane quarter w % 4, column slice (w - 4) / 4).  The epilogue warps
-// also build the split LoRA operands of the NEXT tile as soon as the MMAs of the current one have
-// completed, so the merge of tile t + 1 overlaps the quantizer arithmetic of tile t.
-// Every wait is bounded (see bounded_wait).
+// Roles (640 threads): warp 0 = TMA loads, warp 1 = MMA issuer + TMEM owner, warp 2 = TMA stores (one
+// thread each), warps 4..19 = epilogue (warp w: TMEM lane quarter w % 4, column slice (w - 4) / 4).  The
+// epilogue threads also prepare the MMA operands (split the tile's slices of A and B into tf32 head / tail,
+// swizzled K-major): with two operand buffers (rank <= 32) they load the factors of tile t + 3 and store
+// those of tile t + 2 while working on tile t, so the merge runs two tiles ahead; with one buffer (rank 64)
+// the operands of tile t + 1 are built once the MMAs of tile t have completed.  s and b of a tile are copied
+// to shared memory one tile ahead by one thread per weight row.  Every mbarrier wait is bounded (see
+// bounded_wait); the one block-level barrier per tile is reached unconditionally by all epilogue threads.
 #pragma once
 
 #include "l4q_common.cuh"
@@ -50,7 +53,13 @@ struct WtileArgs {
   int atoms;               // swizzle atoms per operand row: ceil(2 rank / 32)
   int ngt;                 // upper bound of the quantization groups a 128-column tile intersects
   int n_opbuf;             // MMA operand buffers ([A slice | B slice] each): 2 up to rank 32, else 1
+  int group_shift;         // log2(group size) if it is a power of two, else -1
 };
+
+// column / group size without a division in the common power-of-two case
+__device__ __forceinline__ int group_of(const WtileArgs& a, int col) {
+  return a.group_shift >= 0 ? (col >> a.group_shift) : (col / a.p.group);
+}
 
 struct __align__(8) WtileBarriers {
   uint64_t full[WT2_MAX_STAGES];      // W0 tile has landed in the stage
@@ -324,7 +333,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       if (sl != 0) return;
       float* dst = sb_base + ((size_t)buf * WT2_ROWS + row) * sbw;
       const int o_ = m0_ + row;
-      const int g_first = n0_ / p.group;
+      const int g_first = group_of(a, n0_);
       for (int k = 0; k < a.ngt; ++k) {
         const int g = g_first + k;
         if (o_ < p.d_out && g < p.ngroups) {
@@ -344,8 +353,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     int g_first = 0, groups_n0 = -1;
     auto set_groups = [&](int n0_) {
       const int jc = n0_ + sl * 32;
-      g_first = n0_ / p.group;
-      const int g0 = jc / p.group;
+      g_first = group_of(a, n0_);
+      const int g0 = group_of(a, jc);
       const int rem0 = jc - g0 * p.group;
       first_mask = 0; valid_mask = 0;
 #pragma unroll
@@ -540,6 +549,9 @@ inline bool wtile_plan(WtileArgs& a, int mode) {
   a.atoms = (2 * p.rank + 31) / 32;
   a.ngt = std::min(p.ngroups, (WT2_COLS - 1) / p.group + 2);
   a.n_opbuf = (32 * p.rank <= WT2_CARRY * WT2_EPI_THREADS) ? 2 : 1;
+  a.group_shift = -1;
+  for (int sh = 3; sh < 31; ++sh)
+    if ((1 << sh) == p.group) a.group_shift = sh;
   a.out_bytes = mode == WT2_DEQUANT_F ? WT2_STAGE_BYTES : mode == WT2_PACK ? WT2_ROWS * (WT2_COLS * p.bits / 8) : 0;
   const long long budget = 227 * 1024 - 1024 - (long long)sizeof(WtileBarriers) -
                            2LL * a.n_opbuf * a.atoms * WT2_ATOM_BYTES -
