@@ -127,6 +127,36 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Initialisation of the quantization parameters from a weight (Sec. 3.3, Eq. 15; App. B).
+ * In: W [d_out, d_in] (io_dtype; normally W0).  Out: s, b [d_out, d_in / group_size] (fp32), overwritten.
+ * `method` (with Q_N = -2^(bits-1), Q_P = 2^(bits-1) - 1 of Eq. 3, per group):
+ *   L4Q_INIT_LSQ_PLUS  s = max(|mu - 3 sigma|, |mu + 3 sigma|) / 2^(bits-1),  b = 0
+ *                      (mu, sigma: mean and population standard deviation of the group)
+ *   L4Q_INIT_SYMM      s = max|W| / 2^(bits-1),                               b = 0
+ *   L4Q_INIT_ASYMM     s = (max W - min W) / (Q_P - Q_N),                     b = min W - s Q_N
+ *   L4Q_INIT_L4Q       s = max(|min W / Q_N|, |max W / Q_P|),                 b = 0          (Eq. 15)
+ * These are the parameters of the signed grid; without L4Q_FLAG_SIGNED_GRID the same quantizer is
+ * written for the grid [0, 2^bits - 1], i.e. b + s Q_N is returned as b (ASYMM: b = min W).
+ * s is floored at 1e-8 (a constant group would give s = 0; Eq. 3 needs s > 0).
+ * desc->tokens, rank and alpha are ignored.  Needs no workspace.
+ */
+enum { L4Q_INIT_LSQ_PLUS = 0, L4Q_INIT_SYMM = 1, L4Q_INIT_ASYMM = 2, L4Q_INIT_L4Q = 3 };
+l4q_status l4q_init_params(const l4q_desc* desc, const void* W, int method, float* s, float* b, void* cuda_stream);
+
+/*
+ * Error sums of Table 4 for the current parameters:
+ *   errors[0] = E_quant = sum over all weights of |W_comb - W_q|              (Eq. 7-9)
+ *   errors[1] = E_clip  = the part of that sum from weights outside the quantization range, i.e.
+ *                         where the STE gate of App. A.1 is closed (same 2^-10 guard band as the backward)
+ * (the paper gives the two names and their values, not a formula: this is the reading taken).
+ * In: W0 (io_dtype), A, B, s, b (fp32).  Out: errors, two doubles in DEVICE memory, overwritten;
+ * accumulated with fp64 atomics from fp32 partial sums, so the last digits depend on the order.
+ * Needs no workspace.
+ */
+l4q_status l4q_quant_error(const l4q_desc* desc, const void* W0, const float* A, const float* B,
+                           const float* s, const float* b, double* errors, void* cuda_stream);
+
+/*
  * Forward pass for callers that cannot hand the library any scratch memory.
  * (The paper has no counterpart; this entry point exists for integration only.)
  *
@@ -184,7 +214,9 @@ enum {
   L4Q_KERNEL_GEMM_WGRAD = 4,  /* dY^T X tiles reduced into ds, db, dA, dB (Eq. 11, 5-6, 13-14) */
   L4Q_KERNEL_VAL_GEMM = 5,    /* fp32 validation GEMM                                       */
   L4Q_KERNEL_VAL_WGRAD = 6,   /* fp32 validation weight-gradient reduction                  */
-  L4Q_KERNEL_COUNT = 7
+  L4Q_KERNEL_INIT = 7,        /* per-group initialisation of s, b (App. B)                  */
+  L4Q_KERNEL_ERROR = 8,       /* E_quant, E_clip sums (Table 4)                             */
+  L4Q_KERNEL_COUNT = 9
 };
 l4q_status l4q_profile_enable(int enable);
 l4q_status l4q_profile_read(int kernel, uint64_t* launches, double* total_ms);

@@ -32,7 +32,7 @@ notes of the repository):
   * dX = dY W_q is the textbook linear backward (the paper never prints it);
   * the packed export format (bit order, fp16 parameters) is this library's.
 
-Pinned by tests/test_oracle_pins.py and tests/test_oracle_bruteforce.py
+Pinned by tests/test_oracle_pins.py and tests/test_oracle_init_pins.py
 against: B = 0 => merge == W0; grid membership; zero clipping under the
 Asymm / L4Q_init initialisations (Table 4, "Initial" E_clip = 0.0); the LoRA
 limits of Eq. 1-2; finite differences of the STE surrogate; a hand-worked
@@ -210,3 +210,67 @@ def unpack_int(spec: L4QSpec, codes: np.ndarray, d_in: int) -> np.ndarray:
     stream = np.unpackbits(codes.view(np.uint8), axis=1, bitorder="little")[:, : d_in * n]
     bits = stream.reshape(o, d_in, n).astype(np.int64)
     return (bits << np.arange(n, dtype=np.int64)).sum(axis=2)
+
+
+# ---------------------------------------------------------------------------
+# Quantization-parameter initialisation (Sec. 3.3, Eq. 15; App. B) and the
+# error sums of Table 4.
+# ---------------------------------------------------------------------------
+
+INIT_METHODS = ("lsq+", "symm", "asymm", "l4q")
+S_FLOOR = 1e-8          # s > 0 is a precondition of Eq. 3; a constant group would give s = 0
+
+
+def init_params(spec: L4QSpec, W, method: str):
+    """s, b [o, i/g] of every group of the weight W [o, i], App. B, as printed for the
+    signed grid [Q_N, Q_P] = [-2^(n-1), 2^(n-1) - 1]:
+
+        LSQ+_init  s = max(|mu - 3 sigma|, |mu + 3 sigma|) / 2^(n-1),  b = 0
+        Symm       s = max|W| / 2^(n-1),                               b = 0
+        Asymm      s = (max W - min W) / (Q_P - Q_N),                  b = min W - s Q_N
+        L4Q_init   s = max(|min W / Q_N|, |max W / Q_P|),              b = 0      (Eq. 15)
+
+    mu, sigma: mean and (population) standard deviation of the group.  On the shifted grid
+    [0, 2^n - 1] the same quantizer has b' = b + s Q_N (Q_N of the signed grid), which is
+    what is returned when ``spec.signed_grid`` is False.  s is floored at S_FLOOR.
+    """
+    W = _f64(W)
+    g, n = spec.group_size, spec.bits
+    o, i = W.shape
+    Wg = W.reshape(o, i // g, g)
+    qn_s, qp_s = -(2 ** (n - 1)), 2 ** (n - 1) - 1
+    lo, hi = Wg.min(axis=2), Wg.max(axis=2)
+    b = np.zeros_like(lo)
+    if method == "lsq+":
+        mu, sigma = Wg.mean(axis=2), Wg.std(axis=2)
+        s = np.maximum(np.abs(mu - 3.0 * sigma), np.abs(mu + 3.0 * sigma)) / 2.0 ** (n - 1)
+    elif method == "symm":
+        s = np.abs(Wg).max(axis=2) / 2.0 ** (n - 1)
+    elif method == "asymm":
+        s = (hi - lo) / float(qp_s - qn_s)
+        s = np.maximum(s, S_FLOOR)
+        b = lo - s * qn_s
+    elif method == "l4q":
+        s = np.maximum(np.abs(lo / qn_s), np.abs(hi / qp_s))
+    else:
+        raise ValueError(f"unknown initialisation {method!r}")
+    s = np.maximum(s, S_FLOOR)
+    if not spec.signed_grid:
+        b = b + s * qn_s
+    return s, b
+
+
+def quant_error(spec: L4QSpec, W0, A, B, s, b):
+    """(E_quant, E_clip) of Table 4 for the merged weight.
+
+    The paper names them "sum of quantization errors" and "clipping errors caused by
+    overflowed outliers" without a formula; the reading taken here:
+        E_quant = sum over all weights of |W_comb - W_q|,
+        E_clip  = the part of that sum that comes from weights outside the quantization
+                  range, i.e. where the STE gate of App. A.1 is closed (same guard band).
+    """
+    w, _, W_q = fake_quant_weight(spec, W0, A, B, s, b)
+    err = np.abs(merge(spec, W0, A, B) - W_q)
+    qn, qp = grid_bounds(spec)
+    clipped = (w < qn - spec.mask_guard) | (w > qp + spec.mask_guard)
+    return float(err.sum()), float(err[clipped].sum())

@@ -27,13 +27,14 @@ EXPORTED_SYMBOLS = (
     "l4q_workspace_bytes", "l4q_linear_fwd", "l4q_linear_bwd", "l4q_pack_int",
     "l4q_check", "l4q_launch_count", "l4q_status_string",
     "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
-    "l4q_linear_fwd_static",
+    "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error",
 )
+INIT_METHODS = {"lsq+": 0, "symm": 1, "asymm": 2, "l4q": 3}
 
 L4Q_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 KERNEL_IDS = {"dequant": 0, "pack": 1, "gemm_fwd": 2, "gemm_dgrad": 3, "gemm_wgrad": 4, "val_gemm": 5,
-              "val_wgrad": 6}
+              "val_wgrad": 6, "init": 7, "error": 8}
 
 
 class L4QDesc(ctypes.Structure):
@@ -77,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.l4q_linear_bwd.argtypes = [dp, vp, vp, vp, fp, fp, fp, fp, vp, fp, fp, fp, fp, vp, sz, vp]
         L.l4q_pack_int.restype = ctypes.c_int
         L.l4q_pack_int.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp, vp, vp, sz, vp]
+        L.l4q_init_params.restype = ctypes.c_int
+        L.l4q_init_params.argtypes = [dp, vp, ctypes.c_int, fp, fp, vp]
+        L.l4q_quant_error.restype = ctypes.c_int
+        L.l4q_quant_error.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp]
         L.l4q_check.restype = ctypes.c_int
         L.l4q_check.argtypes = [vp]
         L.l4q_launch_count.restype = ctypes.c_uint64
@@ -158,6 +163,21 @@ def l4q_pack_int(desc: L4QDesc, W0, A, B, s, b, codes, s_fp16, b_fp16, workspace
                             _ptr(s_fp16), _ptr(b_fp16), _ptr(workspace),
                             workspace.numel() if workspace is not None else 0, _stream(stream))
     _raise(st, "l4q_pack_int")
+
+
+def l4q_init_params(desc: L4QDesc, W, method: str, s, b, stream=None) -> None:
+    """s, b of every group from the weight W (App. B); method in INIT_METHODS."""
+    st = lib().l4q_init_params(ctypes.byref(desc), _ptr(W), INIT_METHODS[method], _ptr(s), _ptr(b), _stream(stream))
+    _raise(st, "l4q_init_params")
+
+
+def l4q_quant_error(desc: L4QDesc, W0, A, B, s, b, errors, stream=None) -> None:
+    """errors: CUDA tensor of two float64, receives (E_quant, E_clip) of Table 4."""
+    if errors.dtype != torch.float64 or errors.numel() < 2:
+        raise ValueError("errors must be a float64 CUDA tensor with two elements")
+    st = lib().l4q_quant_error(ctypes.byref(desc), _ptr(W0), _ptr(A), _ptr(B), _ptr(s), _ptr(b), _ptr(errors),
+                               _stream(stream))
+    _raise(st, "l4q_quant_error")
 
 
 def l4q_check(stream=None) -> None:

@@ -123,7 +123,7 @@ l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const
     return L4Q_ERR_CUDA;
   dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
   KernelScope ks(L4Q_KERNEL_DEQUANT, st);
-  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, wq, fac, nullptr, nullptr, nullptr);
+  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, wq, fac, nullptr, nullptr, nullptr, nullptr);
   return launch_status();
 }
 
@@ -143,7 +143,7 @@ l4q_status launch_pack(const Params& p, const void* W0, const float* A, const fl
     return L4Q_ERR_CUDA;
   dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
   KernelScope ks(L4Q_KERNEL_PACK, st);
-  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, nullptr, nullptr, codes, s16, b16);
+  kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, nullptr, nullptr, codes, s16, b16, nullptr);
   return launch_status();
 }
 
@@ -284,6 +284,49 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
                                     : launch_pack<false>(p, W0, A, B, s, b, codes, s16, b16, stream);
 }
 
+l4q_status l4q_init_params(const l4q_desc* desc, const void* W, int method, float* s, float* b, void* cuda_stream) {
+  l4q_desc d2;
+  if (!desc) return L4Q_ERR_INVALID_ARG;
+  d2 = *desc;
+  d2.tokens = 1; d2.rank = 8; d2.alpha = 1.f; d2.grad_scale = 1.f;      // unused by this op
+  Params p;
+  l4q_status st = make_params(&d2, &p);
+  if (st != L4Q_OK) return st;
+  if (!W || !s || !b || !aligned16(W)) return L4Q_ERR_INVALID_ARG;
+  if (method < L4Q_INIT_LSQ_PLUS || method > L4Q_INIT_L4Q) return L4Q_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const long long groups = (long long)p.d_out * p.ngroups;
+  const int blocks = (int)std::min<long long>((groups + 7) / 8, (long long)sm_count() * 16);
+  const bool signed_grid = (desc->flags & L4Q_FLAG_SIGNED_GRID) != 0;
+  KernelScope ks(L4Q_KERNEL_INIT, stream);
+  if (desc->io_dtype == L4Q_BF16) k_init_params<true><<<blocks, 256, 0, stream>>>(p, method, signed_grid, W, s, b);
+  else k_init_params<false><<<blocks, 256, 0, stream>>>(p, method, signed_grid, W, s, b);
+  return launch_status();
+}
+
+l4q_status l4q_quant_error(const l4q_desc* desc, const void* W0, const float* A, const float* B, const float* s,
+                           const float* b, double* errors, void* cuda_stream) {
+  Params p;
+  l4q_status st = make_params(desc, &p);
+  if (st != L4Q_OK) return st;
+  if (!W0 || !A || !B || !s || !b || !errors) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(W0) || !aligned16(A) || (reinterpret_cast<uintptr_t>(errors) & 7u)) return L4Q_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(errors, 0, 2 * sizeof(double), stream) != cudaSuccess) return L4Q_ERR_CUDA;
+  const size_t smem = weight_tile_smem_bytes(p.rank);
+  dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
+  auto launch = [&](auto kern) -> l4q_status {
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+    KernelScope ks(L4Q_KERNEL_ERROR, stream);
+    kern<<<grid, WT_THREADS, smem, stream>>>(p, W0, A, B, s, b, nullptr, nullptr, nullptr, nullptr, nullptr, errors);
+    return launch_status();
+  };
+  return desc->io_dtype == L4Q_BF16 ? launch(k_weight_tile<true, WT_MODE_ERROR>)
+                                    : launch(k_weight_tile<false, WT_MODE_ERROR>);
+}
+
 // ---- forward without caller-provided scratch --------------------------------------------------
 // Scratch for the dequantized weight of l4q_linear_fwd_static.  Lives in the library image: every
 // device that loads the library reserves these bytes until the process exits.
@@ -399,6 +442,8 @@ const char* l4q_kernel_name(int kernel) {
     case L4Q_KERNEL_GEMM_WGRAD: return "k_gemm_bf16<wgrad>";
     case L4Q_KERNEL_VAL_GEMM: return "k_val_gemm";
     case L4Q_KERNEL_VAL_WGRAD: return "k_val_wgrad";
+    case L4Q_KERNEL_INIT: return "k_init_params";
+    case L4Q_KERNEL_ERROR: return "k_weight_tile<error sums>";
     default: return "unknown kernel";
   }
 }

@@ -16,7 +16,7 @@ constexpr int WT_ROWS = 64;      // rows of W per block
 constexpr int WT_COLS = 256;     // columns of W per block
 constexpr int WT_THREADS = 256;  // 8 warps; warp w owns rows [8w, 8w+8), lane l columns [8l, 8l+8)
 
-enum { WT_MODE_DEQUANT = 0, WT_MODE_PACK = 1 };
+enum { WT_MODE_DEQUANT = 0, WT_MODE_PACK = 1, WT_MODE_ERROR = 2 };
 
 inline size_t weight_tile_smem_bytes(int rank) {
   return (size_t)rank * (WT_COLS + WT_ROWS) * sizeof(float);
@@ -41,7 +41,8 @@ k_weight_tile(Params p, const void* __restrict__ W0, const float* __restrict__ A
               const float* __restrict__ s, const float* __restrict__ b,
               void* __restrict__ wq_out,                       // MODE_DEQUANT: [d_out, d_in] io dtype
               __half* __restrict__ f_out,                      // MODE_DEQUANT, optional: STE factors [d_out, d_in]
-              uint32_t* __restrict__ codes, __half* __restrict__ s16, __half* __restrict__ b16) {  // MODE_PACK
+              uint32_t* __restrict__ codes, __half* __restrict__ s16, __half* __restrict__ b16,    // MODE_PACK
+              double* __restrict__ err) {            // MODE_ERROR: {E_quant, E_clip}, accumulated
   extern __shared__ __align__(16) float smem_f[];
   const int r = p.rank;
   float4* A_lo = reinterpret_cast<float4*>(smem_f);            // [r][32]: columns 8l .. 8l+3 of lane l
@@ -84,6 +85,7 @@ k_weight_tile(Params p, const void* __restrict__ W0, const float* __restrict__ A
       for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(bv[i], av[j], acc[i][j]);
   }
 
+  [[maybe_unused]] float e_quant = 0.f, e_clip = 0.f;          // MODE_ERROR: this thread's share of the sums
   const int col = col0 + lane * 8;
   const bool col_ok = col < p.d_in;
   const int grp = col_ok ? col / p.group : 0;
@@ -108,6 +110,11 @@ k_weight_tile(Params p, const void* __restrict__ W0, const float* __restrict__ A
         code[j] = q.code;
         wq[j] = q.wq;
         fac[j] = ste_factor(q, p.qn, p.qp);
+        if constexpr (MODE == WT_MODE_ERROR) {                 // |W_comb - W_q|, and its part outside the range
+          const float e = fabsf(merge_elem(w0[j], acc[i][j], p.gamma) - q.wq);
+          e_quant += e;
+          if (!ste_in_range(q.w, p.qn, p.qp)) e_clip += e;
+        }
       }
       if constexpr (MODE == WT_MODE_DEQUANT) {
         if (f_out != nullptr) {
@@ -151,6 +158,78 @@ k_weight_tile(Params p, const void* __restrict__ W0, const float* __restrict__ A
         b16[(size_t)o * p.ngroups + grp] = __float2half_rn(fmaf(sv, p.qn, bvv));
       }
     }
+  }
+  if constexpr (MODE == WT_MODE_ERROR) {
+    // warp sums, then one fp64 atomic per warp and sum
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      e_quant += __shfl_down_sync(0xffffffffu, e_quant, off);
+      e_clip += __shfl_down_sync(0xffffffffu, e_clip, off);
+    }
+    if (lane == 0) {
+      atomicAdd(&err[0], (double)e_quant);
+      atomicAdd(&err[1], (double)e_clip);
+    }
+  }
+}
+
+// Per-group initialisation of the quantization parameters (Sec. 3.3, Eq. 15; App. B): one warp per group,
+// lane = one 8-element piece.  Results on the signed grid of Eq. 3 are shifted to the unsigned grid
+// (b' = b + s Q_N) when the layer uses that one.  s is floored at 1e-8 (Eq. 3 needs s > 0).
+enum { INIT_LSQ_PLUS = 0, INIT_SYMM = 1, INIT_ASYMM = 2, INIT_L4Q = 3 };
+
+template <bool IO_BF16>
+__global__ void __launch_bounds__(256)
+k_init_params(Params p, int method, bool signed_grid, const void* __restrict__ W, float* __restrict__ s_out,
+              float* __restrict__ b_out) {
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const long long total = (long long)p.d_out * p.ngroups;
+  const int pieces = p.group >> 3;
+  const float qn_s = -(float)(1 << (p.bits - 1)), qp_s = (float)((1 << (p.bits - 1)) - 1);
+  for (long long gidx = warp0; gidx < total; gidx += nwarps) {
+    const long long row = gidx / p.ngroups;
+    const int grp = (int)(gidx - row * p.ngroups);
+    const size_t base = (size_t)row * p.d_in + (size_t)grp * p.group;
+    float lo = INFINITY, hi = -INFINITY, sum = 0.f;
+    for (int c = lane; c < pieces; c += 32) {
+      float v[8];
+      load_w0_vec8<IO_BF16>(W, base + (size_t)c * 8, v);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { lo = fminf(lo, v[j]); hi = fmaxf(hi, v[j]); sum += v[j]; }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, off));
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, off));
+      sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    }
+    float sc = 0.f, bs = 0.f;
+    if (method == INIT_LSQ_PLUS) {
+      const float mu = sum / (float)p.group;
+      float ss = 0.f;                                  // second pass: sum of squared deviations
+      for (int c = lane; c < pieces; c += 32) {
+        float v[8];
+        load_w0_vec8<IO_BF16>(W, base + (size_t)c * 8, v);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) ss = fmaf(v[j] - mu, v[j] - mu, ss);
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+      const float sigma = sqrtf(ss / (float)p.group);
+      sc = fmaxf(fabsf(mu - 3.f * sigma), fabsf(mu + 3.f * sigma)) / (float)(1 << (p.bits - 1));
+    } else if (method == INIT_SYMM) {
+      sc = fmaxf(fabsf(lo), fabsf(hi)) / (float)(1 << (p.bits - 1));
+    } else if (method == INIT_ASYMM) {
+      sc = fmaxf((hi - lo) / (qp_s - qn_s), 1e-8f);
+      bs = signed_grid ? lo - sc * qn_s : lo;          // unsigned grid: b' = b + s Q_N = min W exactly
+    } else {
+      sc = fmaxf(fabsf(lo / qn_s), fabsf(hi / qp_s));
+    }
+    sc = fmaxf(sc, 1e-8f);
+    if (!signed_grid && method != INIT_ASYMM) bs = sc * qn_s;   // b = 0 on the signed grid
+    if (lane == 0) { s_out[gidx] = sc; b_out[gidx] = bs; }
   }
 }
 
