@@ -127,6 +127,22 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Inference with the fully quantized layer (Sec. 3.2, App. F): Y = X W_q^T, where the weight is rebuilt
+ * on the fly from the export of l4q_pack_int,
+ *     W_q[o, j] = u[o, j] * s_fp16[o, j / group_size] + b_fp16[o, j / group_size]     (Eq. 9, unsigned code u)
+ * and never exists in memory as a whole (bits / 8 bytes per weight are read).
+ * In: X [tokens, d_in] bf16; codes [d_out, d_in * bits / 32] uint32, s_fp16, b_fp16 [d_out, d_in / group_size]
+ * exactly as written by l4q_pack_int.  Out: Y [tokens, d_out] bf16, overwritten.  W_q is formed in fp32 and
+ * rounded to bf16 for the tensor cores, accumulation is fp32.
+ * Meant for the few-token regime of App. F (a step of batch 1..64); larger token counts work (in tiles of 128
+ * tokens, each of which reads the weight again).  io_dtype must be L4Q_BF16, bits 3 or 4, group_size a multiple
+ * of 32 and d_in * bits / 8 a multiple of 16 (else L4Q_ERR_UNSUPPORTED); rank, alpha and flags are ignored.
+ * Needs no workspace.
+ */
+l4q_status l4q_linear_infer(const l4q_desc* desc, const void* X, const uint32_t* codes, const uint16_t* s_fp16,
+                            const uint16_t* b_fp16, void* Y, void* cuda_stream);
+
+/*
  * Initialisation of the quantization parameters from a weight (Sec. 3.3, Eq. 15; App. B).
  * In: W [d_out, d_in] (io_dtype; normally W0).  Out: s, b [d_out, d_in / group_size] (fp32), overwritten.
  * `method` (with Q_N = -2^(bits-1), Q_P = 2^(bits-1) - 1 of Eq. 3, per group):
@@ -216,7 +232,8 @@ enum {
   L4Q_KERNEL_VAL_WGRAD = 6,   /* fp32 validation weight-gradient reduction                  */
   L4Q_KERNEL_INIT = 7,        /* per-group initialisation of s, b (App. B)                  */
   L4Q_KERNEL_ERROR = 8,       /* E_quant, E_clip sums (Table 4)                             */
-  L4Q_KERNEL_COUNT = 9
+  L4Q_KERNEL_INFER = 9,       /* Y = X W_q^T from the packed export (App. F)                */
+  L4Q_KERNEL_COUNT = 10
 };
 l4q_status l4q_profile_enable(int enable);
 l4q_status l4q_profile_read(int kernel, uint64_t* launches, double* total_ms);

@@ -274,3 +274,24 @@ def quant_error(spec: L4QSpec, W0, A, B, s, b):
     qn, qp = grid_bounds(spec)
     clipped = (w < qn - spec.mask_guard) | (w > qp + spec.mask_guard)
     return float(err.sum()), float(err[clipped].sum())
+
+
+# ---------------------------------------------------------------------------
+# Fully quantized inference (Sec. 3.2, App. F): only the export is kept.
+# ---------------------------------------------------------------------------
+
+def infer(spec: L4QSpec, X, codes: np.ndarray, s16, b16, bf16_reference: bool = False) -> np.ndarray:
+    """Y = X W_q^T with the weight rebuilt from the export of :func:`pack_int`:
+    W_q[o, j] = u[o, j] * s16[o, j // g] + b16[o, j // g]   (Eq. 9 on the unsigned code).
+
+    ``bf16_reference``: W_q is rounded to bf16 before the product and Y after it, as a
+    bf16 tensor-core path does (fp32 accumulation is taken as exact here).
+    """
+    X = _f64(X)
+    u = _f64(unpack_int(spec, codes, X.shape[1]))
+    g = spec.group_size
+    W_q = u * _expand_groups(_f64(s16), g) + _expand_groups(_f64(b16), g)
+    if bf16_reference:
+        W_q = round_to_bf16(W_q)
+    Y = X @ W_q.T
+    return round_to_bf16(Y) if bf16_reference else Y

@@ -27,14 +27,14 @@ EXPORTED_SYMBOLS = (
     "l4q_workspace_bytes", "l4q_linear_fwd", "l4q_linear_bwd", "l4q_pack_int",
     "l4q_check", "l4q_launch_count", "l4q_status_string",
     "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
-    "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error",
+    "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error", "l4q_linear_infer",
 )
 INIT_METHODS = {"lsq+": 0, "symm": 1, "asymm": 2, "l4q": 3}
 
 L4Q_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 KERNEL_IDS = {"dequant": 0, "pack": 1, "gemm_fwd": 2, "gemm_dgrad": 3, "gemm_wgrad": 4, "val_gemm": 5,
-              "val_wgrad": 6, "init": 7, "error": 8}
+              "val_wgrad": 6, "init": 7, "error": 8, "infer": 9}
 
 
 class L4QDesc(ctypes.Structure):
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.l4q_linear_bwd.argtypes = [dp, vp, vp, vp, fp, fp, fp, fp, vp, fp, fp, fp, fp, vp, sz, vp]
         L.l4q_pack_int.restype = ctypes.c_int
         L.l4q_pack_int.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp, vp, vp, sz, vp]
+        L.l4q_linear_infer.restype = ctypes.c_int
+        L.l4q_linear_infer.argtypes = [dp, vp, vp, vp, vp, vp, vp]
         L.l4q_init_params.restype = ctypes.c_int
         L.l4q_init_params.argtypes = [dp, vp, ctypes.c_int, fp, fp, vp]
         L.l4q_quant_error.restype = ctypes.c_int
@@ -163,6 +165,13 @@ def l4q_pack_int(desc: L4QDesc, W0, A, B, s, b, codes, s_fp16, b_fp16, workspace
                             _ptr(s_fp16), _ptr(b_fp16), _ptr(workspace),
                             workspace.numel() if workspace is not None else 0, _stream(stream))
     _raise(st, "l4q_pack_int")
+
+
+def l4q_linear_infer(desc: L4QDesc, X, codes, s_fp16, b_fp16, Y, stream=None) -> None:
+    """Y = X W_q^T from the packed export of l4q_pack_int (few-token inference, App. F)."""
+    st = lib().l4q_linear_infer(ctypes.byref(desc), _ptr(X), _ptr(codes), _ptr(s_fp16), _ptr(b_fp16), _ptr(Y),
+                                _stream(stream))
+    _raise(st, "l4q_linear_infer")
 
 
 def l4q_init_params(desc: L4QDesc, W, method: str, s, b, stream=None) -> None:

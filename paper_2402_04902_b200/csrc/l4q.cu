@@ -12,6 +12,7 @@
 #include "l4q_val.cuh"
 #include "l4q_gemm.cuh"
 #include "l4q_wtile.cuh"
+#include "l4q_infer.cuh"
 
 using namespace l4q;
 
@@ -284,6 +285,23 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
                                     : launch_pack<false>(p, W0, A, B, s, b, codes, s16, b16, stream);
 }
 
+l4q_status l4q_linear_infer(const l4q_desc* desc, const void* X, const uint32_t* codes, const uint16_t* s_fp16,
+                            const uint16_t* b_fp16, void* Y, void* cuda_stream) {
+  if (!desc) return L4Q_ERR_INVALID_ARG;
+  l4q_desc d2 = *desc;
+  d2.rank = 8; d2.alpha = 1.f; d2.grad_scale = 1.f;                     // unused by this op
+  Params p;
+  l4q_status st = make_params(&d2, &p);
+  if (st != L4Q_OK) return st;
+  if (!X || !codes || !s_fp16 || !b_fp16 || !Y) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(codes) || !aligned16(Y)) return L4Q_ERR_INVALID_ARG;
+  if (desc->io_dtype != L4Q_BF16 || !infer_supported(p)) return L4Q_ERR_UNSUPPORTED;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  KernelScope ks(L4Q_KERNEL_INFER, stream);
+  return launch_infer_bf16(p, X, codes, reinterpret_cast<const __half*>(s_fp16),
+                           reinterpret_cast<const __half*>(b_fp16), Y, stream);
+}
+
 l4q_status l4q_init_params(const l4q_desc* desc, const void* W, int method, float* s, float* b, void* cuda_stream) {
   l4q_desc d2;
   if (!desc) return L4Q_ERR_INVALID_ARG;
@@ -444,6 +462,7 @@ const char* l4q_kernel_name(int kernel) {
     case L4Q_KERNEL_VAL_WGRAD: return "k_val_wgrad";
     case L4Q_KERNEL_INIT: return "k_init_params";
     case L4Q_KERNEL_ERROR: return "k_weight_tile<error sums>";
+    case L4Q_KERNEL_INFER: return "k_infer_bf16";
     default: return "unknown kernel";
   }
 }

@@ -529,13 +529,14 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
 // host side
 // ---------------------------------------------------------------------------
 
-// uint32 row-major matrix [rows, words]; box = [box_words, 128 rows], no swizzle (code words of the export).
-inline bool make_tmap_words(CUtensorMap* m, const void* base, uint64_t rows, uint64_t words, uint32_t box_words) {
+// uint32 row-major matrix [rows, words]; box = [box_words, box_rows], no swizzle (code words of the export).
+inline bool make_tmap_words(CUtensorMap* m, const void* base, uint64_t rows, uint64_t words, uint32_t box_words,
+                            uint32_t box_rows = 128) {
   PFN_encodeTiled enc = get_encode_fn();
   if (!enc) return false;
   const cuuint64_t gdim[2] = {words, rows};
   const cuuint64_t gstride[1] = {words * 4};
-  const cuuint32_t box[2] = {box_words, 128};
+  const cuuint32_t box[2] = {box_words, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), gdim, gstride, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

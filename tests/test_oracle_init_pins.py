@@ -97,3 +97,38 @@ def test_quant_error_brute_force():
 def test_constant_group_gets_the_floor():
     s, b = orc.init_params(_spec(), np.zeros((1, 4)), "l4q")
     assert s[0, 0] == orc.S_FLOOR
+
+
+# ---- fully quantized inference (Sec. 3.2, App. F) ----
+
+def test_infer_equals_forward_when_the_export_is_lossless():
+    # s and b + s Q_N exactly representable in fp16 => the export loses nothing and inference reproduces Eq. 10
+    rng = np.random.default_rng(3)
+    for bits, signed in ((4, False), (3, True)):
+        spec = orc.L4QSpec(rank=2, alpha=4.0, bits=bits, group_size=32, signed_grid=signed)
+        W0, A, B = rng.normal(0, 0.3, (5, 64)), rng.normal(0, 1, (2, 64)), rng.normal(0, 0.05, (5, 2))
+        s = rng.integers(1, 8, (5, 2)) / 64.0                    # multiples of 2^-6: exact in fp16
+        b = rng.integers(-32, 32, (5, 2)) / 32.0
+        X = rng.normal(0, 1, (7, 64))
+        codes, s16, b16 = orc.pack_int(spec, W0, A, B, s, b)
+        assert np.array_equal(s16.astype(np.float64), s)
+        Y = orc.forward(spec, X, W0, A, B, s, b)
+        assert np.allclose(orc.infer(spec, X, codes, s16, b16), Y, rtol=1e-13, atol=1e-13)
+
+
+def test_infer_brute_force_from_the_bitstream():
+    rng = np.random.default_rng(4)
+    spec = orc.L4QSpec(rank=1, alpha=1.0, bits=3, group_size=32)
+    u = rng.integers(0, 8, (2, 32))
+    words = np.zeros((2, 3), dtype=np.uint64)
+    for o in range(2):
+        for j in range(32):
+            for k in range(3):                                   # bit k of code j sits at stream bit 3 j + k
+                pos = 3 * j + k
+                words[o, pos // 32] |= np.uint64(((int(u[o, j]) >> k) & 1) << (pos % 32))
+    s16 = np.array([[0.25], [0.5]], dtype=np.float16)
+    b16 = np.array([[-1.0], [0.125]], dtype=np.float16)
+    X = rng.normal(0, 1, (3, 32))
+    Y = [[sum(X[t, j] * (u[o, j] * float(s16[o, 0]) + float(b16[o, 0])) for j in range(32)) for o in range(2)]
+         for t in range(3)]
+    assert np.allclose(orc.infer(spec, X, words.astype(np.uint32), s16, b16), np.array(Y), rtol=1e-13)
