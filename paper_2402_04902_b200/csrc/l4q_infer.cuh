@@ -42,6 +42,7 @@ struct InferArgs {
   int tokens, d_in, d_out, bits, group, ngroups;
   int tile_n;                              // weight rows per tile
   int group_shift;                         // log2(group size) if it is a power of two, else -1
+  int x_rows;                              // token rows a TMA box of X brings in (8 .. 128)
   int tiles_m, tiles_n, num_kb;
   const __half *s16, *b16;
   __nv_bfloat16* Y;
@@ -134,7 +135,9 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
         for (int kb = 0; kb < a.num_kb && !bars->abort; ++kb) {
           bounded_wait(&bars->empty_op[stage], phase ^ 1, bars);
           if (bars->abort) break;
-          ptx::mbar_arrive_expect_tx(&bars->full_x[stage], INF_X_BYTES);
+          // only the rows that hold tokens are copied; the other rows of the operand are never stored
+          // from (an MMA output row depends on its own input row only)
+          ptx::mbar_arrive_expect_tx(&bars->full_x[stage], (uint32_t)(2 * a.x_rows * 128));
           ptx::tma_load_2d(x_tile(stage), &tmap_x, &bars->full_x[stage], kb * INF_BK, m0);
           ptx::tma_load_2d(x_tile(stage) + INF_X_BYTES / 2, &tmap_x, &bars->full_x[stage], kb * INF_BK + 64, m0);
           if (++stage == INF_OP_STAGES) { stage = 0; phase ^= 1; }
@@ -338,7 +341,8 @@ inline l4q_status launch_infer_bf16(const Params& p, const void* X, const uint32
   a.s16 = s16; a.b16 = b16;
   a.Y = reinterpret_cast<__nv_bfloat16*>(Y);
   CUtensorMap tx, tc;
-  if (!make_tmap_bf16(&tx, X, p.tokens, p.d_in, INF_M)) return L4Q_ERR_CUDA;
+  a.x_rows = std::min(INF_M, (p.tokens + 7) / 8 * 8);
+  if (!make_tmap_bf16(&tx, X, p.tokens, p.d_in, a.x_rows)) return L4Q_ERR_CUDA;
   if (!make_tmap_words(&tc, codes, p.d_out, ((uint64_t)p.d_in * p.bits) >> 5, 4 * p.bits, a.tile_n)) return L4Q_ERR_CUDA;
   const size_t smem = infer_smem_bytes();
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
