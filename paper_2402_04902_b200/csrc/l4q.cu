@@ -298,6 +298,9 @@ l4q_status l4q_linear_infer(const l4q_desc* desc, const void* X, const uint32_t*
   if (desc->io_dtype != L4Q_BF16 || !infer_supported(p)) return L4Q_ERR_UNSUPPORTED;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   KernelScope ks(L4Q_KERNEL_INFER, stream);
+  if (gemv_supported(p))                                                 // 1 or 2 tokens: matrix-vector kernel
+    return launch_infer_gemv(p, X, codes, reinterpret_cast<const __half*>(s_fp16),
+                             reinterpret_cast<const __half*>(b_fp16), Y, stream);
   return launch_infer_bf16(p, X, codes, reinterpret_cast<const __half*>(s_fp16),
                            reinterpret_cast<const __half*>(b_fp16), Y, stream);
 }

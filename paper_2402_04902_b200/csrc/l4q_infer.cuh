@@ -68,17 +68,20 @@ inline size_t infer_smem_bytes() {
 // of 1.0 (one shift and one logic op, no integer-to-float conversion).  The caller folds the affine map back:
 // u * s + b = m * (2^BITS s) + (b - 2^BITS s), a single fma.
 template <int BITS>
-__device__ __forceinline__ void unpack_codes32(const uint32_t (&w)[BITS], float (&m)[32]) {
+__device__ __forceinline__ float unpack_code(const uint32_t (&w)[BITS], int j) {      // j: compile-time after unrolling
   constexpr int POS = 23 - BITS;                               // bit position of the code inside the mantissa
   constexpr uint32_t MASK = ((1u << BITS) - 1u) << POS;
+  const int bit = j * BITS, wd = bit >> 5, off = bit & 31;
+  uint32_t v;
+  if (off + BITS > 32) v = __funnelshift_r(w[wd], w[wd + 1 < BITS ? wd + 1 : wd], off) << POS;   // code straddles two words
+  else v = (off <= POS) ? (w[wd] << (POS - off)) : (w[wd] >> (off - POS));
+  return __uint_as_float((v & MASK) | 0x3F800000u);
+}
+
+template <int BITS>
+__device__ __forceinline__ void unpack_codes32(const uint32_t (&w)[BITS], float (&m)[32]) {
 #pragma unroll
-  for (int j = 0; j < 32; ++j) {
-    const int bit = j * BITS, wd = bit >> 5, off = bit & 31;
-    uint32_t v;
-    if (off + BITS > 32) v = __funnelshift_r(w[wd], w[wd + 1], off) << POS;      // code straddles two words
-    else v = (off <= POS) ? (w[wd] << (POS - off)) : (w[wd] >> (off - POS));
-    m[j] = __uint_as_float((v & MASK) | 0x3F800000u);
-  }
+  for (int j = 0; j < 32; ++j) m[j] = unpack_code<BITS>(w, j);
 }
 
 template <int BITS>
@@ -301,6 +304,153 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, INF_ACC * INF_ACC_COLS);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// One or two tokens: a plain-ALU matrix-vector kernel.  With so few tokens there is nothing for the tensor
+// cores to amortise (an MMA has a fixed cost per 16 values of k), while 1 + tokens FMAs per weight keep the
+// FP32 pipe below the time the packed weight needs to arrive from HBM.
+//   * X is copied to shared memory once per CTA as fp32, together with the sum of each 32-value piece;
+//   * a warp owns GEMV_ROWS weight rows at a time and walks along k; a lane takes 32 codes of each row
+//     (16 or 12 contiguous bytes: the warp reads 512 / 384 contiguous bytes per row) and the matching 32
+//     values of X, so the reads of X are shared by the rows;
+//   * codes become m = 1 + u / 2^bits (unpack_codes32); per piece  sum x W_q = (2^bits s) sum x m + (b - 2^bits s) sum x.
+// ---------------------------------------------------------------------------
+constexpr int GEMV_ROWS = 2;
+constexpr int GEMV_THREADS = 256;
+
+template <int BITS, int TOK>
+__global__ void __launch_bounds__(GEMV_THREADS)
+k_infer_gemv(const __nv_bfloat16* __restrict__ X, const uint32_t* __restrict__ codes, const __half* __restrict__ s16,
+             const __half* __restrict__ b16, __nv_bfloat16* __restrict__ Y, int d_in, int d_out, int group_shift,
+             int group, int ngroups) {
+  extern __shared__ __align__(16) float gemv_smem[];
+  const int units = d_in >> 5;                                  // 32-code pieces per row
+  // X in shared memory as [token][v = 0..7][unit][4]: value k = 32 unit + 4 v + e of a token.  A lane owns a
+  // unit, so for a fixed v the 32 lanes of a warp read 32 consecutive float4 (no bank conflicts); with the
+  // natural [token][k] layout their float4 would be 128 bytes apart and hit the same four banks.
+  float* xs = gemv_smem;
+  float* xsum = gemv_smem + (size_t)TOK * d_in;                 // [TOK][units]
+  for (int i = threadIdx.x; i < TOK * d_in; i += GEMV_THREADS) {
+    const int t = i / d_in, k = i - t * d_in;
+    xs[(size_t)t * d_in + ((size_t)((k >> 2) & 7) * units + (k >> 5)) * 4 + (k & 3)] = __bfloat162float(X[i]);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < TOK * units; i += GEMV_THREADS) {
+    const int t = i / units, u = i - t * units;
+    float a = 0.f;
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+      const float4 x4 = *reinterpret_cast<const float4*>(xs + (size_t)t * d_in + ((size_t)v * units + u) * 4);
+      a += (x4.x + x4.y) + (x4.z + x4.w);
+    }
+    xsum[i] = a;
+  }
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warps_total = gridDim.x * (GEMV_THREADS / 32);
+  const int row_words = (d_in * BITS) >> 5;
+  constexpr float kScale = (float)(1 << BITS);
+  for (int r0 = (blockIdx.x * (GEMV_THREADS / 32) + warp) * GEMV_ROWS; r0 < d_out; r0 += warps_total * GEMV_ROWS) {
+    float acc[GEMV_ROWS][TOK];
+#pragma unroll
+    for (int r = 0; r < GEMV_ROWS; ++r)
+#pragma unroll
+      for (int t = 0; t < TOK; ++t) acc[r][t] = 0.f;
+    for (int u = lane; u < units; u += 32) {
+      const int g = group_shift >= 0 ? ((u << 5) >> group_shift) : ((u << 5) / group);
+      float dot[GEMV_ROWS][TOK];
+#pragma unroll
+      for (int r = 0; r < GEMV_ROWS; ++r)
+#pragma unroll
+        for (int t = 0; t < TOK; ++t) dot[r][t] = 0.f;
+      uint32_t w[GEMV_ROWS][BITS];
+#pragma unroll
+      for (int r = 0; r < GEMV_ROWS; ++r) {
+        const int row = min(r0 + r, d_out - 1);                 // rows beyond the weight repeat the last one, unused
+        const uint32_t* src = codes + (size_t)row * row_words + (size_t)u * BITS;
+        if constexpr (BITS == 4) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+          w[r][0] = v.x; w[r][1] = v.y; w[r][2] = v.z; w[r][3] = v.w;
+        } else {
+#pragma unroll
+          for (int i = 0; i < BITS; ++i) w[r][i] = __ldg(src + i);
+        }
+      }
+#pragma unroll
+      for (int v = 0; v < 8; ++v) {                             // 4 values of k at a time: x of every token, code of every row
+        float4 x4[TOK];
+#pragma unroll
+        for (int t = 0; t < TOK; ++t)
+          x4[t] = *reinterpret_cast<const float4*>(xs + (size_t)t * d_in + ((size_t)v * units + u) * 4);
+#pragma unroll
+        for (int r = 0; r < GEMV_ROWS; ++r) {
+          const float m0 = unpack_code<BITS>(w[r], v * 4 + 0), m1 = unpack_code<BITS>(w[r], v * 4 + 1);
+          const float m2 = unpack_code<BITS>(w[r], v * 4 + 2), m3 = unpack_code<BITS>(w[r], v * 4 + 3);
+#pragma unroll
+          for (int t = 0; t < TOK; ++t) {
+            dot[r][t] = fmaf(x4[t].x, m0, dot[r][t]);
+            dot[r][t] = fmaf(x4[t].y, m1, dot[r][t]);
+            dot[r][t] = fmaf(x4[t].z, m2, dot[r][t]);
+            dot[r][t] = fmaf(x4[t].w, m3, dot[r][t]);
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < GEMV_ROWS; ++r) {
+        const int row = min(r0 + r, d_out - 1);
+        const float s_ = __half2float(__ldg(s16 + (size_t)row * ngroups + g));
+        const float b_ = __half2float(__ldg(b16 + (size_t)row * ngroups + g));
+        const float s2 = s_ * kScale, b2 = b_ - s2;
+#pragma unroll
+        for (int t = 0; t < TOK; ++t) acc[r][t] += fmaf(s2, dot[r][t], b2 * xsum[t * units + u]);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < GEMV_ROWS; ++r)
+#pragma unroll
+      for (int t = 0; t < TOK; ++t) {
+        float v = acc[r][t];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (lane == 0 && r0 + r < d_out) Y[(size_t)t * d_out + r0 + r] = __float2bfloat16_rn(v);
+      }
+  }
+}
+
+inline size_t gemv_smem_bytes(int tokens, int d_in) { return (size_t)tokens * (d_in + (d_in >> 5)) * sizeof(float); }
+
+inline bool gemv_supported(const Params& p) {
+  return p.tokens <= 2 && p.d_in % 32 == 0     // measured: beyond two tokens the tensor-core kernel is the faster one
+         && gemv_smem_bytes(p.tokens, p.d_in) <= 200 * 1024;
+}
+
+inline l4q_status launch_infer_gemv(const Params& p, const void* X, const uint32_t* codes, const __half* s16,
+                                    const __half* b16, void* Y, cudaStream_t st) {
+  int shift = -1;
+  for (int sh = 5; sh < 31; ++sh)
+    if ((1 << sh) == p.group) shift = sh;
+  const size_t smem = gemv_smem_bytes(p.tokens, p.d_in);
+  const int quads = ceil_div(p.d_out, GEMV_ROWS);
+  // several CTAs per SM (registers and shared memory permitting): more loads in flight, finer balance
+  const int per_sm = std::max(1, std::min(6, (int)((200 * 1024) / std::max<size_t>(smem, 1))));
+  const int grid = std::min(ceil_div(quads, GEMV_THREADS / 32), sm_count() * per_sm);
+  auto launch = [&](auto kern) -> l4q_status {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+    kern<<<grid, GEMV_THREADS, smem, st>>>(reinterpret_cast<const __nv_bfloat16*>(X), codes, s16, b16,
+                                           reinterpret_cast<__nv_bfloat16*>(Y), p.d_in, p.d_out, shift, p.group, p.ngroups);
+    return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
+  };
+  const int key = p.bits * 10 + p.tokens;
+  switch (key) {
+    case 41: return launch(k_infer_gemv<4, 1>);
+    case 42: return launch(k_infer_gemv<4, 2>);
+    case 31: return launch(k_infer_gemv<3, 1>);
+    case 32: return launch(k_infer_gemv<3, 2>);
+    default: return L4Q_ERR_UNSUPPORTED;
   }
 }
 

@@ -41,7 +41,7 @@ def _run(cfg, seed):
     return err
 
 
-@pytest.mark.parametrize("tokens", [1, 5, 64, 200])
+@pytest.mark.parametrize("tokens", [1, 2, 3, 4, 5, 64, 200])
 @pytest.mark.parametrize("bits,group", [(4, 128), (3, 64), (4, 32), (3, 96)])
 def test_infer_few_tokens(tokens, bits, group):
     # d_in = 1152 = 9 k-blocks of 128 = 36 x 32 = 12 x 96; d_out = 200 leaves a ragged 64-row tile
