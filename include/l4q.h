@@ -173,6 +173,17 @@ l4q_status l4q_quant_error(const l4q_desc* desc, const void* W0, const float* A,
                            const float* s, const float* b, double* errors, void* cuda_stream);
 
 /*
+ * One AdamW step (App. D: "AdamW ... with a weight decay of 0.01") for one trainable tensor of the layer
+ * (A, B, s or b), fused into a single pass over param, grad, m and v (all fp32, n elements, device memory):
+ *     p <- p - lr * weight_decay * p
+ *     m <- beta1 m + (1 - beta1) g          v <- beta2 v + (1 - beta2) g^2
+ *     p <- p - lr * (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps)
+ * `step` counts from 1.  param, m and v are updated in place; grad is read only.
+ */
+l4q_status l4q_adamw_step(float* param, const float* grad, float* m, float* v, size_t n, int64_t step, float lr,
+                          float beta1, float beta2, float eps, float weight_decay, void* cuda_stream);
+
+/*
  * Forward pass for callers that cannot hand the library any scratch memory.
  * (The paper has no counterpart; this entry point exists for integration only.)
  *
@@ -233,7 +244,8 @@ enum {
   L4Q_KERNEL_INIT = 7,        /* per-group initialisation of s, b (App. B)                  */
   L4Q_KERNEL_ERROR = 8,       /* E_quant, E_clip sums (Table 4)                             */
   L4Q_KERNEL_INFER = 9,       /* Y = X W_q^T from the packed export (App. F)                */
-  L4Q_KERNEL_COUNT = 10
+  L4Q_KERNEL_ADAMW = 10,      /* AdamW update of one parameter tensor (App. D)              */
+  L4Q_KERNEL_COUNT = 11
 };
 l4q_status l4q_profile_enable(int enable);
 l4q_status l4q_profile_read(int kernel, uint64_t* launches, double* total_ms);

@@ -295,3 +295,25 @@ def infer(spec: L4QSpec, X, codes: np.ndarray, s16, b16, bf16_reference: bool = 
         W_q = round_to_bf16(W_q)
     Y = X @ W_q.T
     return round_to_bf16(Y) if bf16_reference else Y
+
+
+# ---------------------------------------------------------------------------
+# Optimizer step for the trainable parameters A, B, s, b (App. D: AdamW with weight decay 0.01).
+# ---------------------------------------------------------------------------
+
+def adamw_step(param, grad, m, v, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+               eps: float = 1e-8, weight_decay: float = 0.01):
+    """One AdamW update (decoupled weight decay), the published algorithm step by step:
+        p  <- p - lr * wd * p
+        m  <- beta1 m + (1 - beta1) g            v <- beta2 v + (1 - beta2) g^2
+        mh <- m / (1 - beta1^t)                  vh <- v / (1 - beta2^t)
+        p  <- p - lr * mh / (sqrt(vh) + eps)
+    ``step`` t counts from 1.  Returns (param, m, v) as new fp64 arrays."""
+    p, g, m, v = _f64(param), _f64(grad), _f64(m), _f64(v)
+    p = p - lr * weight_decay * p
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    mh = m / (1.0 - beta1 ** step)
+    vh = v / (1.0 - beta2 ** step)
+    p = p - lr * mh / (np.sqrt(vh) + eps)
+    return p, m, v

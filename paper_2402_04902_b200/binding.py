@@ -27,14 +27,14 @@ EXPORTED_SYMBOLS = (
     "l4q_workspace_bytes", "l4q_linear_fwd", "l4q_linear_bwd", "l4q_pack_int",
     "l4q_check", "l4q_launch_count", "l4q_status_string",
     "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
-    "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error", "l4q_linear_infer",
+    "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error", "l4q_linear_infer", "l4q_adamw_step",
 )
 INIT_METHODS = {"lsq+": 0, "symm": 1, "asymm": 2, "l4q": 3}
 
 L4Q_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 KERNEL_IDS = {"dequant": 0, "pack": 1, "gemm_fwd": 2, "gemm_dgrad": 3, "gemm_wgrad": 4, "val_gemm": 5,
-              "val_wgrad": 6, "init": 7, "error": 8, "infer": 9}
+              "val_wgrad": 6, "init": 7, "error": 8, "infer": 9, "adamw": 10}
 
 
 class L4QDesc(ctypes.Structure):
@@ -80,6 +80,9 @@ def lib() -> ctypes.CDLL:
         L.l4q_pack_int.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp, vp, vp, sz, vp]
         L.l4q_linear_infer.restype = ctypes.c_int
         L.l4q_linear_infer.argtypes = [dp, vp, vp, vp, vp, vp, vp]
+        L.l4q_adamw_step.restype = ctypes.c_int
+        L.l4q_adamw_step.argtypes = [fp, fp, fp, fp, sz, ctypes.c_int64, ctypes.c_float, ctypes.c_float,
+                                     ctypes.c_float, ctypes.c_float, ctypes.c_float, vp]
         L.l4q_init_params.restype = ctypes.c_int
         L.l4q_init_params.argtypes = [dp, vp, ctypes.c_int, fp, fp, vp]
         L.l4q_quant_error.restype = ctypes.c_int
@@ -172,6 +175,17 @@ def l4q_linear_infer(desc: L4QDesc, X, codes, s_fp16, b_fp16, Y, stream=None) ->
     st = lib().l4q_linear_infer(ctypes.byref(desc), _ptr(X), _ptr(codes), _ptr(s_fp16), _ptr(b_fp16), _ptr(Y),
                                 _stream(stream))
     _raise(st, "l4q_linear_infer")
+
+
+def l4q_adamw_step(param, grad, m, v, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+                   eps: float = 1e-8, weight_decay: float = 0.01, stream=None) -> None:
+    """In-place AdamW update of one fp32 parameter tensor (App. D); step counts from 1."""
+    for t in (param, grad, m, v):
+        if t.dtype != torch.float32 or t.numel() != param.numel():
+            raise ValueError("AdamW tensors must be float32 and of one size")
+    st = lib().l4q_adamw_step(_ptr(param), _ptr(grad), _ptr(m), _ptr(v), param.numel(), int(step), float(lr),
+                              float(beta1), float(beta2), float(eps), float(weight_decay), _stream(stream))
+    _raise(st, "l4q_adamw_step")
 
 
 def l4q_init_params(desc: L4QDesc, W, method: str, s, b, stream=None) -> None:

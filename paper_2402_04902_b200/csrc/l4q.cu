@@ -2,6 +2,7 @@
 // layout and kernel launches.  One translation unit; the kernels live in the
 // headers included below.
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -305,6 +306,20 @@ l4q_status l4q_linear_infer(const l4q_desc* desc, const void* X, const uint32_t*
                            reinterpret_cast<const __half*>(b_fp16), Y, stream);
 }
 
+l4q_status l4q_adamw_step(float* param, const float* grad, float* m, float* v, size_t n, int64_t step, float lr,
+                          float beta1, float beta2, float eps, float weight_decay, void* cuda_stream) {
+  if (!param || !grad || !m || !v || n == 0 || step < 1) return L4Q_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f) || !(lr == lr))
+    return L4Q_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const double c1 = 1.0 - std::pow((double)beta1, (double)step), c2 = 1.0 - std::pow((double)beta2, (double)step);
+  const int blocks = (int)std::min<size_t>((n + 255) / 256, (size_t)sm_count() * 8);
+  KernelScope ks(L4Q_KERNEL_ADAMW, stream);
+  k_adamw<<<blocks, 256, 0, stream>>>(param, grad, m, v, n, lr, beta1, beta2, eps, weight_decay, (float)(1.0 / c1),
+                                      (float)(1.0 / c2));
+  return launch_status();
+}
+
 l4q_status l4q_init_params(const l4q_desc* desc, const void* W, int method, float* s, float* b, void* cuda_stream) {
   l4q_desc d2;
   if (!desc) return L4Q_ERR_INVALID_ARG;
@@ -466,6 +481,7 @@ const char* l4q_kernel_name(int kernel) {
     case L4Q_KERNEL_INIT: return "k_init_params";
     case L4Q_KERNEL_ERROR: return "k_weight_tile<error sums>";
     case L4Q_KERNEL_INFER: return "k_infer_bf16";
+    case L4Q_KERNEL_ADAMW: return "k_adamw";
     default: return "unknown kernel";
   }
 }

@@ -233,4 +233,23 @@ k_init_params(Params p, int method, bool signed_grid, const void* __restrict__ W
   }
 }
 
+// One AdamW update of a parameter tensor (App. D: AdamW, decoupled weight decay), everything in one pass:
+//   p <- p - lr wd p;  m <- b1 m + (1 - b1) g;  v <- b2 v + (1 - b2) g^2;  p <- p - lr (m / c1) / (sqrt(v / c2) + eps)
+// with the bias corrections c1 = 1 - b1^t, c2 = 1 - b2^t computed on the host in double precision.
+__global__ void __launch_bounds__(256)
+k_adamw(float* __restrict__ param, const float* __restrict__ grad, float* __restrict__ m, float* __restrict__ v,
+        size_t n, float lr, float beta1, float beta2, float eps, float weight_decay, float inv_c1, float inv_c2) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const float g = grad[i];
+    float p = param[i];
+    p = fmaf(-lr * weight_decay, p, p);
+    const float mi = fmaf(beta1, m[i], (1.f - beta1) * g);
+    const float vi = fmaf(beta2, v[i], (1.f - beta2) * g * g);
+    m[i] = mi;
+    v[i] = vi;
+    param[i] = p - lr * (mi * inv_c1) / (sqrtf(vi * inv_c2) + eps);
+  }
+}
+
 }  // namespace l4q

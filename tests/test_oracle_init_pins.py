@@ -132,3 +132,27 @@ def test_infer_brute_force_from_the_bitstream():
     Y = [[sum(X[t, j] * (u[o, j] * float(s16[o, 0]) + float(b16[o, 0])) for j in range(32)) for o in range(2)]
          for t in range(3)]
     assert np.allclose(orc.infer(spec, X, words.astype(np.uint32), s16, b16), np.array(Y), rtol=1e-13)
+
+
+# ---- AdamW (App. D) ----
+
+def test_adamw_matches_the_library_optimizer():
+    import torch
+    rng = np.random.default_rng(5)
+    p0 = rng.normal(0, 1, (7, 5))
+    p_t = torch.tensor(p0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.AdamW([p_t], lr=3e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.01)
+    p, m, v = p0.copy(), np.zeros_like(p0), np.zeros_like(p0)
+    for step in range(1, 6):
+        g = rng.normal(0, 1, p0.shape)
+        p_t.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        p, m, v = orc.adamw_step(p, g, m, v, step, lr=3e-3)
+        assert np.allclose(p, p_t.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_adamw_first_step_is_a_sign_step():
+    # t = 1: mh = g, vh = g^2, so the update is -lr * g / (|g| + eps) on top of the decay
+    p, g = np.array([1.0, -2.0, 0.5]), np.array([0.3, -4.0, 1e-3])
+    got, _, _ = orc.adamw_step(p, g, np.zeros(3), np.zeros(3), 1, lr=0.1, weight_decay=0.0)
+    assert np.allclose(got, p - 0.1 * g / (np.abs(g) + 1e-8), rtol=1e-12)
