@@ -331,10 +331,12 @@ def run_ours(args, layers, wl_name):
             k["gbs"] = deq_bytes * steps_timed / (k["total_ms"] * 1e-3) / 1e9
     dominant = max(kernels, key=lambda n: kernels[n]["total_ms"]) if kernels else None
     traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    tpath = os.path.join(ROOT, "profiles", f"dram_traffic_{wl_name}.txt")
     if os.path.exists(tpath):
-        tj = json.load(open(tpath))
-        traffic = tj.get(wl_name, {}).get(dominant)
+        for ln in open(tpath):
+            f = ln.split()
+            if len(f) == 2 and f[0] == dominant:
+                traffic = float(f[1])
     roofline = None
     if dominant in gemm_flops:
         ach = kernels[dominant]["tflops"]
