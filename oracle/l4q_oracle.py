@@ -317,3 +317,70 @@ def adamw_step(param, grad, m, v, step: int, lr: float, beta1: float = 0.9, beta
     vh = v / (1.0 - beta2 ** step)
     p = p - lr * mh / (np.sqrt(vh) + eps)
     return p, m, v
+
+
+# ---------------------------------------------------------------------------
+# The two layers L4Q is set against (Sec. 2.1 and 3.1): plain LoRA and QAT-LoRA, which
+# keeps the quantized frozen weight and the high-precision LoRA path apart.
+# ---------------------------------------------------------------------------
+
+def lora_forward(spec: L4QSpec, X, W0, A, B, bf16_reference: bool = False) -> np.ndarray:
+    """Eq. 1: Y = X W0^T + gamma (X A^T) B^T  (X~ = X A^T is the input of B)."""
+    X = _f64(X)
+    Xt = X @ _f64(A).T
+    Y = X @ _f64(W0).T + spec.gamma * (Xt @ _f64(B).T)
+    return round_to_bf16(Y) if bf16_reference else Y
+
+
+def lora_backward(spec: L4QSpec, X, dY, W0, A, B, bf16_reference: bool = False) -> dict:
+    """Eq. 2 in this file's layout, and the input gradient of Eq. 1:
+        dA = gamma (dY B)^T X         dB = gamma dY^T X~,  X~ = X A^T
+        dX = dY W0 + gamma (dY B) A
+    """
+    X, dY, A, B = _f64(X), _f64(dY), _f64(A), _f64(B)
+    dYt = dY @ B                                    # gradient at the output of A, [M, r]
+    Xt = X @ A.T
+    dX = dY @ _f64(W0) + spec.gamma * (dYt @ A)
+    if bf16_reference:
+        dX = round_to_bf16(dX)
+    return {"dX": dX, "dA": spec.gamma * (dYt.T @ X), "dB": spec.gamma * (dY.T @ Xt)}
+
+
+def qat_lora_forward(spec: L4QSpec, X, W0, A, B, s, b, bf16_reference: bool = False, codes=None) -> np.ndarray:
+    """QAT-LoRA (Sec. 3.1): the frozen weight alone goes through the quantizer of Eq. 3 / Eq. 8-9
+    and the LoRA path of Eq. 1 is added in high precision:
+        Y = X Q(W0)^T + gamma (X A^T) B^T.
+    """
+    X = _f64(X)
+    zero_B = np.zeros((np.shape(W0)[0], spec.rank))
+    _, _, Wq = fake_quant_weight(spec, W0, A, zero_B, s, b, codes)
+    if bf16_reference:
+        Wq = round_to_bf16(Wq)
+    Y = X @ Wq.T + spec.gamma * ((X @ _f64(A).T) @ _f64(B).T)
+    return round_to_bf16(Y) if bf16_reference else Y
+
+
+def qat_lora_backward(spec: L4QSpec, X, dY, W0, A, B, s, b, bf16_reference: bool = False, codes=None) -> dict:
+    """Backward of QAT-LoRA.  The LoRA factors get the LoRA gradients of Eq. 2, the quantizer gets
+    the LSQ gradients of Eq. 5-6 from the full weight gradient G = dY^T X (the cost Sec. 3.1 points
+    out), with w = (W0 - b) / s: the two sets of parameters do not see each other.
+        dX = dY Q(W0) + gamma (dY B) A
+    """
+    X, dY, A, B = _f64(X), _f64(dY), _f64(A), _f64(B)
+    g = spec.group_size
+    qn, qp = grid_bounds(spec)
+    zero_B = np.zeros((np.shape(W0)[0], spec.rank))
+    w, wt, Wq = fake_quant_weight(spec, W0, A, zero_B, s, b, codes)
+    if bf16_reference:
+        Wq = round_to_bf16(Wq)
+    dYt = dY @ B
+    dX = dY @ Wq + spec.gamma * (dYt @ A)
+    if bf16_reference:
+        dX = round_to_bf16(dX)
+    G = dY.T @ X
+    in_range = (w >= qn - spec.mask_guard) & (w <= qp + spec.mask_guard)
+    dWq_ds = np.where(in_range, wt - w, np.where(w < qn, float(qn), float(qp)))
+    o, i = G.shape
+    ds = spec.grad_scale * (G * dWq_ds).reshape(o, i // g, g).sum(axis=2)
+    db = spec.grad_scale * (G * (1.0 - in_range)).reshape(o, i // g, g).sum(axis=2)
+    return {"dX": dX, "dA": spec.gamma * (dYt.T @ X), "dB": spec.gamma * (dY.T @ (X @ A.T)), "ds": ds, "db": db}
