@@ -18,6 +18,10 @@ N > 1 (launched by torch.distributed.run, one rank per GPU): data parallel over
 tokens -- every rank runs the same layers on its own token batch (weak scaling)
 and the parameter gradients are all-reduced (sum) over NCCL each step.
 
+`--layer lora|qat_lora` runs the LoRA (Eq. 1-2) or QAT-LoRA (Sec. 3.1) layer instead, through
+l4q_lora_linear_fwd / l4q_lora_linear_bwd, for the per-step cost comparison (no export step; the
+flop count is that layer's own).  The default, `--layer l4q`, is the benchmark proper.
+
 `--impl reference` times the fp64 CPU oracle (oracle/), as it stands, on the
 host cores on a bounded slice of the same workload.
 """
@@ -51,11 +55,15 @@ def workloads() -> dict:
     }
 
 
-def layer_flops(cfg, tokens=None, d_out=None) -> float:
-    """Algorithmic flops of fwd + bwd of one linear: three M*o*i products, merge twice, dA and dB."""
+def layer_flops(cfg, tokens=None, d_out=None, layer="l4q") -> float:
+    """Algorithmic flops of fwd + bwd of one linear: three M*o*i products, merge twice, dA and dB.
+    LoRA: two M*o*i products and six rank-side products; QAT-LoRA adds the full weight gradient."""
     M = cfg.tokens if tokens is None else tokens
     o = cfg.d_out if d_out is None else d_out
-    return 6.0 * M * o * cfg.d_in + 8.0 * o * cfg.d_in * cfg.rank
+    if layer == "l4q":
+        return 6.0 * M * o * cfg.d_in + 8.0 * o * cfg.d_in * cfg.rank
+    side = 6.0 * M * cfg.rank * (cfg.d_in + o)
+    return (4.0 if layer == "lora" else 6.0) * M * o * cfg.d_in + side
 
 
 def peaks() -> dict:
@@ -215,6 +223,8 @@ def run_ours(args, layers, wl_name):
     # ---- synthetic layers: weights shared by all ranks, activations per rank (data parallel) ----
     L = []
     h2d = d2h = 0
+    grad_names = ("dA", "dB") if args.layer == "lora" else ("dA", "dB", "ds", "db")
+    kind = l4q.LORA_KINDS.get(args.layer)
     for li, cfg in enumerate(layers):
         arrays = synth.make_layer_inputs(cfg, seed=0, layer_id=li, need_acts=False)
         acts = synth.make_layer_acts(cfg, seed=1000 + rank, layer_id=li)
@@ -227,8 +237,11 @@ def run_ours(args, layers, wl_name):
         desc = l4q.make_desc(cfg)
         outs = l4q.alloc_outputs(cfg, device=dev)
         pk = l4q.alloc_pack_outputs(cfg, device=dev)
-        ws = l4q.alloc_workspace(desc, l4q.L4Q_OP_BWD, device=dev)
-        grads_host = {k: torch.empty_like(outs[k], device="cpu").pin_memory() for k in ("dA", "dB", "ds", "db")}
+        if args.layer == "l4q":
+            ws = l4q.alloc_workspace(desc, l4q.L4Q_OP_BWD, device=dev)
+        else:
+            ws = l4q.alloc_lora_workspace(desc, l4q.LORA_KINDS[args.layer], l4q.L4Q_OP_BWD, device=dev)
+        grads_host = {k: torch.empty_like(outs[k], device="cpu").pin_memory() for k in grad_names}
         L.append(dict(cfg=cfg, desc=desc, d=d, outs=outs, pk=pk, ws=ws, host=host, grads_host=grads_host))
         h2d += host["X"].numel() * 2 + host["dY"].numel() * 2
         d2h += sum(t.numel() * 4 for t in grads_host.values())
@@ -239,14 +252,23 @@ def run_ours(args, layers, wl_name):
             if e2e:
                 d["X"].copy_(l["host"]["X"], non_blocking=True)
                 d["dY"].copy_(l["host"]["dY"], non_blocking=True)
-            l4q.l4q_linear_fwd(l["desc"], d["X"], d["W0"], d["A"], d["B"], d["s"], d["b"], o["Y"], l["ws"])
-            l4q.l4q_linear_bwd(l["desc"], d["X"], d["dY"], d["W0"], d["A"], d["B"], d["s"], d["b"],
-                               o["dX"], o["dA"], o["dB"], o["ds"], o["db"], l["ws"])
-            l4q.l4q_pack_int(l["desc"], d["W0"], d["A"], d["B"], d["s"], d["b"], pk["codes"], pk["s16"], pk["b16"])
+            if kind is None:
+                l4q.l4q_linear_fwd(l["desc"], d["X"], d["W0"], d["A"], d["B"], d["s"], d["b"], o["Y"], l["ws"])
+                l4q.l4q_linear_bwd(l["desc"], d["X"], d["dY"], d["W0"], d["A"], d["B"], d["s"], d["b"],
+                                   o["dX"], o["dA"], o["dB"], o["ds"], o["db"], l["ws"])
+                l4q.l4q_pack_int(l["desc"], d["W0"], d["A"], d["B"], d["s"], d["b"], pk["codes"], pk["s16"],
+                                 pk["b16"])
+            else:
+                qat = args.layer == "qat_lora"
+                sq, bq = (d["s"], d["b"]) if qat else (None, None)
+                l4q.l4q_lora_linear_fwd(l["desc"], kind, d["X"], d["W0"], d["A"], d["B"], sq, bq, o["Y"], l["ws"])
+                l4q.l4q_lora_linear_bwd(l["desc"], kind, d["X"], d["dY"], d["W0"], d["A"], d["B"], sq, bq, o["dX"],
+                                        o["dA"], o["dB"], o["ds"] if qat else None, o["db"] if qat else None,
+                                        l["ws"])
             if world > 1:
-                dp.allreduce_param_grads(o)
+                dp.allreduce_param_grads({k: o[k] for k in grad_names} if kind else o)
             if e2e:
-                for k in ("dA", "dB", "ds", "db"):
+                for k in grad_names:
                     l["grads_host"][k].copy_(o[k], non_blocking=True)
 
     def timed(e2e: bool, steps: int, warmup: int):
@@ -269,7 +291,7 @@ def run_ours(args, layers, wl_name):
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
         return float(ms.item())
 
-    flops_step_rank = sum(layer_flops(l["cfg"]) for l in L)
+    flops_step_rank = sum(layer_flops(l["cfg"], layer=args.layer) for l in L)
     tokens_step_rank = L[0]["cfg"].tokens
 
     # ---- device-resident timing, with per-kernel events and clock samples ----
@@ -361,7 +383,7 @@ def run_ours(args, layers, wl_name):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": wl_name,
+        "config": {"workload": wl_name, "layer": args.layer,
                    "layers": [f"{l['cfg'].d_in}->{l['cfg'].d_out}" for l in L],
                    "tokens_per_gpu": tokens_step_rank, "rank": L[0]["cfg"].rank, "bits": L[0]["cfg"].bits,
                    "group_size": L[0]["cfg"].group_size, "parallelism": f"dp{world}",
@@ -388,6 +410,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="llama7b_mlp", choices=sorted(workloads()))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layer", default="l4q", choices=["l4q", "lora", "qat_lora"],
+                    help="l4q = the benchmark; lora / qat_lora = the comparison layers (ours arm only)")
     args = ap.parse_args()
     layers = workloads()[args.workload]
     if args.impl == "reference":

@@ -127,6 +127,37 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The two layers L4Q is set against, on the same kernels, for measuring what the merged quantization
+ * costs per step (Sec. 3.1; the training-time remark of App. E).  `kind`:
+ *   L4Q_LORA_PLAIN  Y = X W0^T + gamma (X A^T) B^T                                          (Eq. 1)
+ *                   dA = gamma (dY B)^T X,   dB = gamma dY^T (X A^T)                        (Eq. 2)
+ *                   dX = dY W0 + gamma (dY B) A
+ *   L4Q_LORA_QAT    QAT-LoRA: the same with W0 replaced by Q(W0) = round(clamp((W0-b)/s)) s + b (Eq. 3),
+ *                   and ds, db = the LSQ gradients of that quantizer (Eq. 5-6, App. A.1) from the full
+ *                   weight gradient dY^T X; the LoRA factors and the quantizer do not see each other.
+ * Same layouts, dtypes and conventions as l4q_linear_fwd / l4q_linear_bwd; io_dtype must be L4Q_BF16
+ * and rank <= 64 (else L4Q_ERR_UNSUPPORTED).  s, b are read by L4Q_LORA_QAT only (NULL otherwise).
+ * X A^T and dY B are rounded to bf16, as are A and B where a tensor-core product reads them; every
+ * product accumulates in fp32.  The backward takes nothing from the forward (X A^T is recomputed).
+ * Backward outputs: dX may be NULL; dA and dB come together or not at all; ds and db likewise, and
+ * only for L4Q_LORA_QAT (rank 8, 16, 32 or 64) -- passing them with L4Q_LORA_PLAIN is
+ * L4Q_ERR_INVALID_ARG.  Outputs are overwritten.  Workspace: l4q_lora_workspace_bytes(desc, kind, op),
+ * op = L4Q_OP_FWD or L4Q_OP_BWD (0 if the problem is invalid or unsupported).
+ */
+enum { L4Q_LORA_PLAIN = 1, L4Q_LORA_QAT = 2 };
+
+size_t l4q_lora_workspace_bytes(const l4q_desc* desc, int kind, int op);
+
+l4q_status l4q_lora_linear_fwd(const l4q_desc* desc, int kind, const void* X, const void* W0,
+                               const float* A, const float* B, const float* s, const float* b,
+                               void* Y, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, const void* dY, const void* W0,
+                               const float* A, const float* B, const float* s, const float* b,
+                               void* dX, float* dA, float* dB, float* ds, float* db,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Inference with the fully quantized layer (Sec. 3.2, App. F): Y = X W_q^T, where the weight is rebuilt
  * on the fly from the export of l4q_pack_int,
  *     W_q[o, j] = u[o, j] * s_fp16[o, j / group_size] + b_fp16[o, j / group_size]     (Eq. 9, unsigned code u)
@@ -245,7 +276,8 @@ enum {
   L4Q_KERNEL_ERROR = 8,       /* E_quant, E_clip sums (Table 4)                             */
   L4Q_KERNEL_INFER = 9,       /* Y = X W_q^T from the packed export (App. F)                */
   L4Q_KERNEL_ADAMW = 10,      /* AdamW update of one parameter tensor (App. D)              */
-  L4Q_KERNEL_COUNT = 11
+  L4Q_KERNEL_LORA_SIDE = 11,  /* rank-side products of the LoRA / QAT-LoRA layers (Eq. 1-2) */
+  L4Q_KERNEL_COUNT = 12
 };
 l4q_status l4q_profile_enable(int enable);
 l4q_status l4q_profile_read(int kernel, uint64_t* launches, double* total_ms);

@@ -28,13 +28,16 @@ EXPORTED_SYMBOLS = (
     "l4q_check", "l4q_launch_count", "l4q_status_string",
     "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
     "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error", "l4q_linear_infer", "l4q_adamw_step",
+    "l4q_lora_workspace_bytes", "l4q_lora_linear_fwd", "l4q_lora_linear_bwd",
 )
+L4Q_LORA_PLAIN, L4Q_LORA_QAT = 1, 2
+LORA_KINDS = {"lora": L4Q_LORA_PLAIN, "qat_lora": L4Q_LORA_QAT}
 INIT_METHODS = {"lsq+": 0, "symm": 1, "asymm": 2, "l4q": 3}
 
 L4Q_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 KERNEL_IDS = {"dequant": 0, "pack": 1, "gemm_fwd": 2, "gemm_dgrad": 3, "gemm_wgrad": 4, "val_gemm": 5,
-              "val_wgrad": 6, "init": 7, "error": 8, "infer": 9, "adamw": 10}
+              "val_wgrad": 6, "init": 7, "error": 8, "infer": 9, "adamw": 10, "lora_side": 11}
 
 
 class L4QDesc(ctypes.Structure):
@@ -76,6 +79,12 @@ def lib() -> ctypes.CDLL:
         L.l4q_linear_fwd_static.argtypes = [dp, vp, vp, fp, fp, fp, fp, vp, vp]
         L.l4q_linear_bwd.restype = ctypes.c_int
         L.l4q_linear_bwd.argtypes = [dp, vp, vp, vp, fp, fp, fp, fp, vp, fp, fp, fp, fp, vp, sz, vp]
+        L.l4q_lora_workspace_bytes.restype = sz
+        L.l4q_lora_workspace_bytes.argtypes = [dp, ctypes.c_int, ctypes.c_int]
+        L.l4q_lora_linear_fwd.restype = ctypes.c_int
+        L.l4q_lora_linear_fwd.argtypes = [dp, ctypes.c_int, vp, vp, fp, fp, fp, fp, vp, vp, sz, vp]
+        L.l4q_lora_linear_bwd.restype = ctypes.c_int
+        L.l4q_lora_linear_bwd.argtypes = [dp, ctypes.c_int, vp, vp, vp, fp, fp, fp, fp, vp, fp, fp, fp, fp, vp, sz, vp]
         L.l4q_pack_int.restype = ctypes.c_int
         L.l4q_pack_int.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp, vp, vp, sz, vp]
         L.l4q_linear_infer.restype = ctypes.c_int
@@ -161,6 +170,33 @@ def l4q_linear_bwd(desc: L4QDesc, X, dY, W0, A, B, s, b, dX, dA, dB, ds, db, wor
                               _ptr(dX), _ptr(dA), _ptr(dB), _ptr(ds), _ptr(db),
                               _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream))
     _raise(st, "l4q_linear_bwd")
+
+
+def l4q_lora_workspace_bytes(desc: L4QDesc, kind: int, op: int) -> int:
+    return int(lib().l4q_lora_workspace_bytes(ctypes.byref(desc), int(kind), int(op)))
+
+
+def alloc_lora_workspace(desc: L4QDesc, kind: int, op: int, device="cuda") -> torch.Tensor:
+    n = max(l4q_lora_workspace_bytes(desc, kind, op), 256)
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def l4q_lora_linear_fwd(desc: L4QDesc, kind: int, X, W0, A, B, s, b, Y, workspace, stream=None) -> None:
+    """Forward of the LoRA (Eq. 1) or QAT-LoRA (Sec. 3.1) layer; kind = L4Q_LORA_PLAIN / L4Q_LORA_QAT."""
+    st = lib().l4q_lora_linear_fwd(ctypes.byref(desc), int(kind), _ptr(X), _ptr(W0), _ptr(A), _ptr(B), _ptr(s),
+                                   _ptr(b), _ptr(Y), _ptr(workspace),
+                                   workspace.numel() if workspace is not None else 0, _stream(stream))
+    _raise(st, "l4q_lora_linear_fwd")
+
+
+def l4q_lora_linear_bwd(desc: L4QDesc, kind: int, X, dY, W0, A, B, s, b, dX, dA, dB, ds, db, workspace,
+                        stream=None) -> None:
+    """Backward of the LoRA (Eq. 2) or QAT-LoRA layer; ds, db only for L4Q_LORA_QAT."""
+    st = lib().l4q_lora_linear_bwd(ctypes.byref(desc), int(kind), _ptr(X), _ptr(dY), _ptr(W0), _ptr(A), _ptr(B),
+                                   _ptr(s), _ptr(b), _ptr(dX), _ptr(dA), _ptr(dB), _ptr(ds), _ptr(db),
+                                   _ptr(workspace), workspace.numel() if workspace is not None else 0,
+                                   _stream(stream))
+    _raise(st, "l4q_lora_linear_bwd")
 
 
 def l4q_pack_int(desc: L4QDesc, W0, A, B, s, b, codes, s_fp16, b_fp16, workspace=None, stream=None) -> None:

@@ -14,6 +14,7 @@
 #include "l4q_gemm.cuh"
 #include "l4q_wtile.cuh"
 #include "l4q_infer.cuh"
+#include "l4q_variants.cuh"
 
 using namespace l4q;
 
@@ -149,6 +150,47 @@ l4q_status launch_pack(const Params& p, const void* W0, const float* A, const fl
   return launch_status();
 }
 
+// ---- LoRA and QAT-LoRA layers (Eq. 1-2, Sec. 3.1) ---------------------------------------------
+
+struct LoraWorkspace {
+  void* wq = nullptr;            // QAT-LoRA: Q(W0), bf16
+  __half* fac = nullptr;         // QAT-LoRA backward: STE factors
+  VariantScratch v{};
+  float* zero_B = nullptr;       // QAT-LoRA: a zero LoRA factor, so that the weight-tile kernel quantizes W0 alone
+  float *dA_unused = nullptr, *dB_unused = nullptr;   // QAT-LoRA backward: the merged-layer LoRA gradients, not wanted
+  size_t bytes = 0;
+};
+
+LoraWorkspace lora_workspace(const l4q_desc* d, const Params& p, int kind, int op, void* base) {
+  LoraWorkspace w;
+  unsigned char* c = static_cast<unsigned char*>(base);
+  size_t off = 0;
+  auto take = [&](size_t n) { unsigned char* q = c ? c + off : nullptr; off += align_up(n, 256); return q; };
+  if (kind == L4Q_LORA_QAT) {
+    w.wq = take(wq_scratch_bytes(d));
+    if (op == L4Q_OP_BWD) w.fac = reinterpret_cast<__half*>(take(factor_scratch_bytes(d)));
+  }
+  w.v = variant_scratch(p, c ? c + off : nullptr);
+  off += w.v.bytes;
+  if (kind == L4Q_LORA_QAT) {
+    w.zero_B = reinterpret_cast<float*>(take((size_t)p.d_out * p.rank * sizeof(float)));
+    if (op == L4Q_OP_BWD) {
+      w.dA_unused = reinterpret_cast<float*>(take((size_t)p.rank * p.d_in * sizeof(float)));
+      w.dB_unused = reinterpret_cast<float*>(take((size_t)p.d_out * p.rank * sizeof(float)));
+    }
+  }
+  w.bytes = off + 256;
+  return w;
+}
+
+l4q_status lora_check(const l4q_desc* desc, int kind, Params* p) {
+  l4q_status st = make_params(desc, p);
+  if (st != L4Q_OK) return st;
+  if (kind != L4Q_LORA_PLAIN && kind != L4Q_LORA_QAT) return L4Q_ERR_INVALID_ARG;
+  if (desc->io_dtype != L4Q_BF16 || p->rank > LORA_PAD) return L4Q_ERR_UNSUPPORTED;
+  return L4Q_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -264,6 +306,110 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
     KernelScope ks(L4Q_KERNEL_GEMM_WGRAD, stream);
     st = gemm_wgrad_bf16(p, X, dY, fac, A, B, dA, dB, ds, db, stream);
     if (st != L4Q_OK) return st;
+  }
+  return L4Q_OK;
+}
+
+size_t l4q_lora_workspace_bytes(const l4q_desc* desc, int kind, int op) {
+  Params p;
+  if (lora_check(desc, kind, &p) != L4Q_OK || (op != L4Q_OP_FWD && op != L4Q_OP_BWD)) return 0;
+  return lora_workspace(desc, p, kind, op, nullptr).bytes;
+}
+
+l4q_status l4q_lora_linear_fwd(const l4q_desc* desc, int kind, const void* X, const void* W0, const float* A,
+                               const float* B, const float* s, const float* b, void* Y, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream) {
+  Params p;
+  l4q_status st = lora_check(desc, kind, &p);
+  if (st != L4Q_OK) return st;
+  const bool qat = kind == L4Q_LORA_QAT;
+  if (!X || !W0 || !A || !B || !Y || (qat && (!s || !b))) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W0) || !aligned16(A) || !aligned16(B) || !aligned16(Y)) return L4Q_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < l4q_lora_workspace_bytes(desc, kind, L4Q_OP_FWD) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return L4Q_ERR_WORKSPACE;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const LoraWorkspace w = lora_workspace(desc, p, kind, L4Q_OP_FWD, workspace);
+  const void* W = W0;
+  if (qat) {
+    if (cudaMemsetAsync(w.zero_B, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+    if ((st = launch_dequant<true>(p, W0, A, w.zero_B, s, b, w.wq, nullptr, stream)) != L4Q_OK) return st;
+    W = w.wq;
+  }
+  {
+    KernelScope ks(L4Q_KERNEL_LORA_SIDE, stream);
+    if ((st = launch_lora_cast(p, A, B, w.v, stream)) != L4Q_OK) return st;
+  }
+  {
+    KernelScope ks(L4Q_KERNEL_LORA_SIDE, stream);
+    if ((st = gemm_lora_down_bf16(p, X, w.v, stream)) != L4Q_OK) return st;
+  }
+  KernelScope ks(L4Q_KERNEL_GEMM_FWD, stream);
+  return gemm_forward_lora_bf16(p, X, W, w.v, Y, stream);
+}
+
+l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, const void* dY, const void* W0,
+                               const float* A, const float* B, const float* s, const float* b, void* dX, float* dA,
+                               float* dB, float* ds, float* db, void* workspace, size_t workspace_bytes,
+                               void* cuda_stream) {
+  Params p;
+  l4q_status st = lora_check(desc, kind, &p);
+  if (st != L4Q_OK) return st;
+  const bool qat = kind == L4Q_LORA_QAT;
+  if (!X || !dY || !W0 || !A || !B || (qat && (!s || !b))) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(dY) || !aligned16(W0) || !aligned16(A) || !aligned16(B) || !aligned16(dX))
+    return L4Q_ERR_INVALID_ARG;
+  if ((dA != nullptr) != (dB != nullptr) || (ds != nullptr) != (db != nullptr)) return L4Q_ERR_INVALID_ARG;
+  if (!qat && ds) return L4Q_ERR_INVALID_ARG;                  // plain LoRA has no quantizer
+  if (qat && ds && !wgrad_rank_supported(p.rank)) return L4Q_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < l4q_lora_workspace_bytes(desc, kind, L4Q_OP_BWD) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return L4Q_ERR_WORKSPACE;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const LoraWorkspace w = lora_workspace(desc, p, kind, L4Q_OP_BWD, workspace);
+  const void* W = W0;
+  if (qat && (dX || ds)) {
+    if (cudaMemsetAsync(w.zero_B, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+    if ((st = launch_dequant<true>(p, W0, A, w.zero_B, s, b, w.wq, ds ? w.fac : nullptr, stream)) != L4Q_OK)
+      return st;
+    W = w.wq;
+  }
+  if (dX || dA) {
+    {
+      KernelScope ks(L4Q_KERNEL_LORA_SIDE, stream);
+      if ((st = launch_lora_cast(p, A, B, w.v, stream)) != L4Q_OK) return st;
+    }
+    KernelScope ks(L4Q_KERNEL_LORA_SIDE, stream);
+    if ((st = gemm_lora_up_t_bf16(p, dY, w.v, stream)) != L4Q_OK) return st;         // dYt = dY B
+  }
+  if (dX) {
+    KernelScope ks(L4Q_KERNEL_GEMM_DGRAD, stream);
+    if ((st = gemm_dgrad_lora_bf16(p, dY, W, w.v, dX, stream)) != L4Q_OK) return st;
+  }
+  if (dA) {
+    if (cudaMemsetAsync(dA, 0, (size_t)p.rank * p.d_in * sizeof(float), stream) != cudaSuccess ||
+        cudaMemsetAsync(dB, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+    {
+      KernelScope ks(L4Q_KERNEL_LORA_SIDE, stream);                                  // Xt = X A^T, recomputed
+      if ((st = gemm_lora_down_bf16(p, X, w.v, stream)) != L4Q_OK) return st;
+    }
+    {
+      KernelScope ks(L4Q_KERNEL_LORA_SIDE, stream);
+      if ((st = gemm_lora_da_bf16(p, X, w.v, dA, stream)) != L4Q_OK) return st;
+    }
+    KernelScope ks(L4Q_KERNEL_LORA_SIDE, stream);
+    if ((st = gemm_lora_db_bf16(p, dY, w.v, dB, stream)) != L4Q_OK) return st;
+  }
+  if (qat && ds) {
+    const size_t gsz = (size_t)p.d_out * p.ngroups * sizeof(float);
+    if (cudaMemsetAsync(ds, 0, gsz, stream) != cudaSuccess || cudaMemsetAsync(db, 0, gsz, stream) != cudaSuccess)
+      return L4Q_ERR_CUDA;
+    KernelScope ks(L4Q_KERNEL_GEMM_WGRAD, stream);
+    if ((st = gemm_wgrad_bf16(p, X, dY, w.fac, A, w.zero_B, w.dA_unused, w.dB_unused, ds, db, stream)) != L4Q_OK)
+      return st;
   }
   return L4Q_OK;
 }
@@ -482,6 +628,7 @@ const char* l4q_kernel_name(int kernel) {
     case L4Q_KERNEL_ERROR: return "k_weight_tile<error sums>";
     case L4Q_KERNEL_INFER: return "k_infer_bf16";
     case L4Q_KERNEL_ADAMW: return "k_adamw";
+    case L4Q_KERNEL_LORA_SIDE: return "k_gemm_bf16<rank side> / k_lora_cast";
     default: return "unknown kernel";
   }
 }

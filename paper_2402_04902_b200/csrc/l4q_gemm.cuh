@@ -6,6 +6,11 @@
 //   dgrad     dX = dY Wq     A = dY (K-major),   B = Wq (MN-major),  K = d_out
 //   wgrad     G  = dY^T X    A = dY (MN-major),  B = X  (MN-major),  K = tokens   (Eq. 11)
 //
+// The same template also runs the layers L4Q is compared with (Eq. 1-2, Sec. 3.1): a narrow N tile
+// (TN = 64) for the rank-side products X A^T and dY B, one extra K block taken from a second pair
+// of tensor maps (EXT) that adds the LoRA path gamma (X A^T) B^T to the main product inside the
+// accumulator, and an epilogue that adds a scaled fp32 tile into dA / dB (EPI_ADD_F32).
+//
 // The wgrad epilogue never writes G: each 128 x 256 tile of G is reduced from
 // tensor memory into ds, db (Eq. 5-6), dA and dB (Eq. 13-14).  The quantizer
 // state of the tile's weights (STE gate and dW_q/ds) is recomputed in the same
@@ -36,6 +41,7 @@ constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
 constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KB
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+__host__ __device__ constexpr int stage_bytes_for(int tn) { return A_STAGE_BYTES + tn * BK * 2; }
 constexpr int GEMM_THREADS = 384;
 constexpr int EPI_FIRST_WARP = 4;
 constexpr int EPI_GROUPS = 2;
@@ -44,13 +50,18 @@ constexpr int ACC_STAGES = 2;
 constexpr int TMEM_COLS = ACC_STAGES * BN;   // 512: all of tensor memory
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s at B200 clocks
 
-enum { EPI_STORE = 0, EPI_WGRAD = 1 };
+enum { EPI_STORE = 0, EPI_WGRAD = 1, EPI_ADD_F32 = 2 };
 
 struct GemmArgs {
   int M, N, K;                 // GEMM extents
   int tiles_m, tiles_n, num_kb;
+  int num_kb2;                 // EXT: K blocks taken from the second pair of tensor maps, after the first num_kb
   // EPI_STORE
   __nv_bfloat16* C;            // [M, N] row-major
+  // EPI_ADD_F32: C32[row * ldc + col] += scale * acc for row < M, col < N (atomic; C32 zero or partial on entry)
+  float* C32;
+  int ldc;
+  float scale;
   // EPI_WGRAD (M = d_out, N = d_in)
   Params p;
   const __half* F;             // [d_out, d_in] STE factors of the weights (ste_factor)
@@ -66,8 +77,8 @@ struct __align__(8) GemmBarriers {
   volatile uint32_t abort;
 };
 
-inline size_t gemm_smem_bytes(int stages, int epi_bytes) {
-  return 1024 /*alignment slack*/ + (size_t)stages * STAGE_BYTES + (size_t)epi_bytes + sizeof(GemmBarriers);
+inline size_t gemm_smem_bytes(int stages, int epi_bytes, int stage_bytes = STAGE_BYTES) {
+  return 1024 /*alignment slack*/ + (size_t)stages * stage_bytes + (size_t)epi_bytes + sizeof(GemmBarriers);
 }
 
 // Bounded mbarrier wait.  Returns immediately once the CTA's abort flag is set.
@@ -355,9 +366,14 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
   ptx::mbar_arrive(tmem_empty_bar);                    // accumulator stage (and its result columns) free
 }
 
-template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES>
+template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES, int TN = BN, bool EXT = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmArgs g) {
+k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+            const __grid_constant__ CUtensorMap tmap_a2, const __grid_constant__ CUtensorMap tmap_b2, const GemmArgs g) {
+  static_assert(TN == 64 || TN == BN, "tile width");
+  static_assert(EPI != EPI_WGRAD || (TN == BN && !EXT), "the weight-gradient epilogue works on 256-column tiles");
+  constexpr int STAGE_BYTES = stage_bytes_for(TN);           // shadows the 256-column figure
+  constexpr int TMEM_COLS = ACC_STAGES * TN;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
@@ -367,7 +383,8 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = g.tiles_m * g.tiles_n;
-  constexpr bool TAIL_SPLIT = (EPI == EPI_WGRAD);
+  constexpr bool TAIL_SPLIT = (EPI != EPI_STORE);            // reductions with atomics may be cut along K
+  const int total_kb = g.num_kb + (EXT ? g.num_kb2 : 0);
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&bars->full[i], 1); ptx::mbar_init(&bars->empty[i], 1); }
@@ -380,6 +397,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     ptx::fence_mbar_init();
     ptx::prefetch_tmap(&tmap_a);
     ptx::prefetch_tmap(&tmap_b);
+    if constexpr (EXT) { ptx::prefetch_tmap(&tmap_a2); ptx::prefetch_tmap(&tmap_b2); }
   }
   if (warp == 1) {
     ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -394,32 +412,36 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      WorkIter<TAIL_SPLIT> work(num_tiles, g.num_kb);
+      WorkIter<TAIL_SPLIT> work(num_tiles, total_kb);
       WorkUnit u;
       while (!bars->abort && work.next(u)) {
         int tm, tn;
         tile_coords(u.tile, g.tiles_m, g.tiles_n, tm, tn);
-        const int m0 = tm * BM, n0 = tn * BN;
+        const int m0 = tm * BM, n0 = tn * TN;
         for (int kb = u.kb0; kb < u.kb1 && !bars->abort; ++kb) {
           bounded_wait(&bars->empty[stage], phase ^ 1, bars);
           if (bars->abort) break;
           uint8_t* sa = stage_base + (size_t)stage * STAGE_BYTES;
           uint8_t* sb = sa + A_STAGE_BYTES;
           ptx::mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
-          const int k0 = kb * BK;
+          // K blocks past the first operand pair come from the second one (same box shapes)
+          const bool second = EXT && kb >= g.num_kb;
+          const CUtensorMap* ma = second ? &tmap_a2 : &tmap_a;
+          const CUtensorMap* mb = second ? &tmap_b2 : &tmap_b;
+          const int k0 = (second ? kb - g.num_kb : kb) * BK;
           if constexpr (!A_MN) {
-            ptx::tma_load_2d(sa, &tmap_a, &bars->full[stage], k0, m0);
+            ptx::tma_load_2d(sa, ma, &bars->full[stage], k0, m0);
           } else {
 #pragma unroll
             for (int h = 0; h < BM / 64; ++h)
-              ptx::tma_load_2d(sa + h * (64 * BK * 2), &tmap_a, &bars->full[stage], m0 + h * 64, k0);
+              ptx::tma_load_2d(sa + h * (64 * BK * 2), ma, &bars->full[stage], m0 + h * 64, k0);
           }
           if constexpr (!B_MN) {
-            ptx::tma_load_2d(sb, &tmap_b, &bars->full[stage], k0, n0);
+            ptx::tma_load_2d(sb, mb, &bars->full[stage], k0, n0);
           } else {
 #pragma unroll
-            for (int h = 0; h < BN / 64; ++h)
-              ptx::tma_load_2d(sb + h * (64 * BK * 2), &tmap_b, &bars->full[stage], n0 + h * 64, k0);
+            for (int h = 0; h < TN / 64; ++h)
+              ptx::tma_load_2d(sb + h * (64 * BK * 2), mb, &bars->full[stage], n0 + h * 64, k0);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -429,7 +451,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, BN, A_MN, B_MN);
+      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, TN, A_MN, B_MN);
       // K-major: 8-row groups of 128-byte rows are 1024 B apart; a K step of 16 elements is +32 B.
       // MN-major: 8 k-rows of 128 bytes (64 elements along M/N) are 1024 B apart, 64-element
       // blocks along M/N are one TMA box (BK rows x 128 B) apart; a K step of 16 is two row groups.
@@ -437,13 +459,13 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       constexpr uint32_t B_LBO = B_MN ? (BK * 128) : 16, B_SBO = 1024, B_KSTEP = B_MN ? 2048 : 32;
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
-      WorkIter<TAIL_SPLIT> work(num_tiles, g.num_kb);
+      WorkIter<TAIL_SPLIT> work(num_tiles, total_kb);
       WorkUnit u;
       while (!bars->abort && work.next(u)) {
         bounded_wait(&bars->tmem_empty[acc], acc_phase ^ 1, bars);
         if (bars->abort) break;
         ptx::tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TN);
         for (int kb = u.kb0; kb < u.kb1; ++kb) {
           bounded_wait(&bars->full[stage], phase, bars);
           if (bars->abort) break;
@@ -470,18 +492,40 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int eg = (warp - EPI_FIRST_WARP) >> 2;
     int acc = 0; uint32_t acc_phase = 0;
     [[maybe_unused]] uint32_t epi_phase = 0;
-    WorkIter<TAIL_SPLIT> work(num_tiles, g.num_kb);
+    WorkIter<TAIL_SPLIT> work(num_tiles, total_kb);
     WorkUnit u;
     while (work.next(u)) {
       int tm, tn;
       tile_coords(u.tile, g.tiles_m, g.tiles_n, tm, tn);
-      const int m0 = tm * BM, n0 = tn * BN;
-      const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
-      if constexpr (EPI == EPI_STORE) {
+      const int m0 = tm * BM, n0 = tn * TN;
+      const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * TN);
+      if constexpr (EPI == EPI_ADD_F32) {
         bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
         ptx::tc_fence_after_sync();
         const int row = m0 + quarter * 32 + lane;
-        constexpr int CHUNKS_PER_GROUP = (BN / 32) / EPI_GROUPS;
+        constexpr int CHUNKS_PER_GROUP = (TN / 32) / EPI_GROUPS;
+#pragma unroll 1
+        for (int cc = 0; cc < CHUNKS_PER_GROUP; ++cc) {
+          const int c = eg * CHUNKS_PER_GROUP + cc;
+          uint32_t raw[32];
+          ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), raw);
+          ptx::tmem_ld_wait();
+          if (cc == CHUNKS_PER_GROUP - 1) {
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&bars->tmem_empty[acc]);
+          }
+          if (row < g.M) {
+            float* dst = g.C32 + (size_t)row * g.ldc + n0 + c * 32;
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (n0 + c * 32 + e < g.N) atomicAdd(dst + e, g.scale * __uint_as_float(raw[e]));
+          }
+        }
+      } else if constexpr (EPI == EPI_STORE) {
+        bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
+        ptx::tc_fence_after_sync();
+        const int row = m0 + quarter * 32 + lane;
+        constexpr int CHUNKS_PER_GROUP = (TN / 32) / EPI_GROUPS;
 #pragma unroll 1
         for (int cc = 0; cc < CHUNKS_PER_GROUP; ++cc) {
           const int c = eg * CHUNKS_PER_GROUP + cc;
@@ -573,19 +617,23 @@ inline int sm_count() {
   return n;
 }
 
-template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES>
-l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g, cudaStream_t st) {
+// `ta2`, `tb2`: second operand pair of an EXT launch (g.num_kb2 K blocks); ignored otherwise.
+template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES, int TN = BN, bool EXT = false>
+l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g, cudaStream_t st,
+                       const CUtensorMap* ta2 = nullptr, const CUtensorMap* tb2 = nullptr) {
   g.tiles_m = ceil_div(g.M, BM);
-  g.tiles_n = ceil_div(g.N, BN);
+  g.tiles_n = ceil_div(g.N, TN);
   g.num_kb = ceil_div(g.K, BK);
-  auto kern = k_gemm_bf16<A_MN, B_MN, EPI, RANK, STAGES>;
-  const size_t smem = gemm_smem_bytes(STAGES, EPI == EPI_WGRAD ? wgrad_epi_smem_bytes(RANK) : 0);
+  if (!EXT) g.num_kb2 = 0;
+  if (EXT && (!ta2 || !tb2)) return L4Q_ERR_INVALID_ARG;
+  auto kern = k_gemm_bf16<A_MN, B_MN, EPI, RANK, STAGES, TN, EXT>;
+  const size_t smem = gemm_smem_bytes(STAGES, EPI == EPI_WGRAD ? wgrad_epi_smem_bytes(RANK) : 0, stage_bytes_for(TN));
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return L4Q_ERR_CUDA;
   const int tiles = g.tiles_m * g.tiles_n, sms = sm_count();
   int grid = std::min(tiles, sms);
-  if (EPI == EPI_WGRAD && tiles < sms) grid = tiles * std::min(sms / tiles, g.num_kb);   // K slices for the idle SMs
-  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, g);
+  if (EPI != EPI_STORE && tiles < sms) grid = tiles * std::min(sms / tiles, g.num_kb);   // K slices for the idle SMs
+  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, EXT ? *ta2 : ta, EXT ? *tb2 : tb, g);
   return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
 }
 

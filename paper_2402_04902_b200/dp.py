@@ -23,8 +23,11 @@ def token_shard(tokens: int, rank: int, world: int) -> slice:
 
 
 def allreduce_param_grads(grads: dict, group=None) -> None:
-    """In-place sum over ranks of dA, dB, ds, db (one all-reduce per tensor; a no-op for one rank)."""
+    """In-place sum over ranks of those of dA, dB, ds, db that `grads` holds (one all-reduce per tensor;
+    a no-op for one rank)."""
     if not dist.is_available() or not dist.is_initialized() or dist.get_world_size(group) == 1:
         return
     for k in PARAM_GRADS:
+        if k not in grads:
+            continue
         dist.all_reduce(grads[k], op=dist.ReduceOp.SUM, group=group)
