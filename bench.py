@@ -246,12 +246,40 @@ def run_ours(args, layers, wl_name):
         h2d += host["X"].numel() * 2 + host["dY"].numel() * 2
         d2h += sum(t.numel() * 4 for t in grads_host.values())
 
-    def step(e2e: bool):
-        for l in L:
-            d, o, pk = l["d"], l["outs"], l["pk"]
+    # End-to-end mode double-buffers the activations: while a layer computes on one pair of device
+    # buffers, a copy stream brings the next layer's (or next step's) X and dY from pinned host memory
+    # into the other pair.  Every step still copies all of its inputs inside the timed region.
+    copy_stream = torch.cuda.Stream(device=dev)
+    for l in L:
+        l["act"] = [{"X": l["d"]["X"], "dY": l["d"]["dY"]},
+                    {"X": torch.empty_like(l["d"]["X"]), "dY": torch.empty_like(l["d"]["dY"])}]
+        l["ready"] = [torch.cuda.Event(), torch.cuda.Event()]
+        l["free"] = [None, None]                     # recorded when the compute stream is done with the pair
+
+    def prefetch(l, par):
+        with torch.cuda.stream(copy_stream):
+            if l["free"][par] is not None:
+                copy_stream.wait_event(l["free"][par])
+            l["act"][par]["X"].copy_(l["host"]["X"], non_blocking=True)
+            l["act"][par]["dY"].copy_(l["host"]["dY"], non_blocking=True)
+            l["ready"][par].record(copy_stream)
+
+    e2e_units = {"n": 0}                             # steps run in end-to-end mode so far (buffer parity)
+
+    def step(e2e: bool, last: bool = True):
+        par = e2e_units["n"] % 2 if e2e else 0
+        for li, l in enumerate(L):
+            d, o, pk = dict(l["d"]), l["outs"], l["pk"]
             if e2e:
-                d["X"].copy_(l["host"]["X"], non_blocking=True)
-                d["dY"].copy_(l["host"]["dY"], non_blocking=True)
+                if li == 0 and not e2e_units.get("primed"):
+                    prefetch(l, par)                 # pipeline fill: nothing to overlap the first copy with
+                    e2e_units["primed"] = True
+                if li + 1 < len(L):
+                    prefetch(L[li + 1], par)
+                elif not last:
+                    prefetch(L[0], par ^ 1)
+                torch.cuda.current_stream().wait_event(l["ready"][par])
+                d["X"], d["dY"] = l["act"][par]["X"], l["act"][par]["dY"]
             if kind is None:
                 l4q.l4q_linear_fwd(l["desc"], d["X"], d["W0"], d["A"], d["B"], d["s"], d["b"], o["Y"], l["ws"])
                 l4q.l4q_linear_bwd(l["desc"], d["X"], d["dY"], d["W0"], d["A"], d["B"], d["s"], d["b"],
@@ -268,20 +296,27 @@ def run_ours(args, layers, wl_name):
             if world > 1:
                 dp.allreduce_param_grads({k: o[k] for k in grad_names} if kind else o)
             if e2e:
+                ev = torch.cuda.Event()
+                ev.record()
+                l["free"][par] = ev
                 for k in grad_names:
                     l["grads_host"][k].copy_(o[k], non_blocking=True)
+        if e2e:
+            e2e_units["n"] += 1
+            if last:
+                e2e_units["primed"] = False
 
     def timed(e2e: bool, steps: int, warmup: int):
-        for _ in range(warmup):
-            step(e2e)
+        for i in range(warmup):
+            step(e2e, last=(i == warmup - 1))
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
-        for _ in range(steps):
-            step(e2e)
+        for i in range(steps):
+            step(e2e, last=(i == steps - 1))
         ev1.record()
         torch.cuda.synchronize()
         if world > 1:
