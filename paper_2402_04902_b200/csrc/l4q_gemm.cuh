@@ -19,8 +19,8 @@
 // are two more tcgen05 MMAs per 128 columns, fed from a bf16 copy of G * m in
 // shared memory.
 //
-// Roles (384 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
-// owner, warps 4..11 = two epilogue groups of 128 threads (each group drains
+// Roles (384 threads): warp 0 = TMA producer of operand A, warp 2 = TMA producer
+// of operand B, warp 1 = MMA issuer and TMEM owner, warps 4..11 = two epilogue groups of 128 threads (each group drains
 // half of the tile's columns; a warp reads the TMEM lane quarter warp_id % 4).
 // Two accumulator stages of 256 TMEM columns let the epilogue of tile t overlap
 // the main loop of tile t + 1.
@@ -161,9 +161,16 @@ struct WorkIter {
 //   abf   4 x RN x 128 B   bf16 copy of A[:, n0 : n0+256], four K-major tiles of 64 columns
 //   btbf  2 x RN x 128 B   bf16 copy of B[m0 : m0+128, :]^T, two K-major tiles of 64 weight rows
 // RN = max(rank, 16) rows (the MMA's N), rows beyond the rank are zero.
+// Up to rank 16 the epilogue works on 64 columns at a time (Gm is one 128 x 64 tile, 16 KB): that leaves room
+// for a fourth pipeline stage, which the main loop needs more than the epilogue needs wide steps.
 constexpr int GM_BYTES = 128 * 128 * 2;
 __host__ __device__ constexpr int wgrad_rn(int rank) { return rank < 16 ? 16 : rank; }
-__host__ __device__ constexpr int wgrad_epi_smem_bytes(int rank) { return GM_BYTES + 6 * wgrad_rn(rank) * 128; }
+__host__ __device__ constexpr bool wgrad_quarters(int rank) { return wgrad_rn(rank) == 16; }
+__host__ __device__ constexpr int wgrad_gm_bytes(int rank) { return wgrad_quarters(rank) ? GM_BYTES / 2 : GM_BYTES; }
+__host__ __device__ constexpr int wgrad_epi_smem_bytes(int rank) {
+  return wgrad_gm_bytes(rank) + 6 * wgrad_rn(rank) * 128;
+}
+__host__ __device__ constexpr int wgrad_stages(int rank) { return wgrad_quarters(rank) ? 4 : 3; }
 
 template <int N>
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[N]) {
@@ -366,6 +373,185 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
   ptx::mbar_arrive(tmem_empty_bar);                    // accumulator stage (and its result columns) free
 }
 
+// The same reduction for ranks up to 16, 64 columns at a time (see wgrad_quarters).  Per quarter q the two
+// groups drain one 32-column chunk each into a 128 x 64 Gm tile; then
+//     dB[128 rows, r]   += Gm[128, 64] A[:, 64 cols]^T           M = 128, K-major Gm
+//     dA_q^T[64 cols, r] = Gm^T[64 cols, 128 rows] B[rows, :]    M = 64, MN-major view of the same bytes
+// An M = 64 accumulator keeps row j in TMEM lane 32 (j / 16) + j % 16, i.e. 16 rows in the lower half of each
+// warp's lane quarter.  Result columns inside the drained accumulator: dB at 0, dA_q at RN (1 + q); after
+// quarter q columns [0, 64 (q + 1)) have been read, and RN (2 + q) <= 64 (q + 1) for RN = 16.
+template <int RANK>
+__device__ __forceinline__ void wgrad_epilogue_tile_q(const GemmArgs& g, int m0, int n0, uint32_t tmem_acc, int quarter,
+                                                      int lane, int eg, uint8_t* epi_smem, GemmBarriers* bars,
+                                                      uint64_t* tmem_full_bar, uint32_t full_parity,
+                                                      uint64_t* tmem_empty_bar, uint32_t& epi_phase) {
+  constexpr int RN = wgrad_rn(RANK);
+  static_assert(RN == 16, "quarter path");
+  constexpr int GMQ = GM_BYTES / 2;
+  const Params& p = g.p;
+  uint8_t* gm = epi_smem;
+  uint8_t* abf = gm + GMQ;
+  uint8_t* btbf = abf + 4 * RN * 128;
+  const int t = quarter * 32 + lane;
+  const int t256 = eg * 128 + t;
+  const int o = m0 + t;
+  const bool row_ok = o < p.d_out;
+  const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+
+  // ---- bf16 copies of the tile's slices of A and B (as in wgrad_epilogue_tile) ----
+#pragma unroll
+  for (int u = 0; u < (RN * 32) / EPI_THREADS; ++u) {
+    const int q = t256 + u * EPI_THREADS;
+    const int k = q >> 5, jc = q & 31;
+    const int col = n0 + jc * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (k < RANK && col < p.d_in) {
+      const float4* src = reinterpret_cast<const float4*>(g.A + (size_t)k * p.d_in + col);
+      const float4 a0 = __ldg(src), a1 = __ldg(src + 1);
+      v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w);
+      v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
+    }
+    *reinterpret_cast<uint4*>(abf + (jc >> 3) * (RN * 128) + k * 128 + (((jc & 7) ^ (k & 7)) << 4)) = v;
+  }
+#pragma unroll
+  for (int u = 0; u < RN / 2; u += 4) {
+    const int n = eg * (RN / 2) + u;
+    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row_ok && n < RANK) bv = __ldg(reinterpret_cast<const float4*>(g.B + (size_t)o * RANK + n));
+    const float be[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int nn = n + e;
+      uint8_t* dst = btbf + (t >> 6) * (RN * 128) + nn * 128 + ((((t & 63) >> 3) ^ (nn & 7)) << 4) + (t & 7) * 2;
+      *reinterpret_cast<__nv_bfloat16*>(dst) = __float2bfloat16_rn(be[e]);
+    }
+  }
+  ptx::fence_proxy_async_smem();
+  ptx::named_bar_sync(3, EPI_THREADS);
+
+  bounded_wait(tmem_full_bar, full_parity, bars);
+  ptx::tc_fence_after_sync();
+
+  float ds_acc = 0.f, db_acc = 0.f;
+  int cur_grp = -1;
+
+#pragma unroll 1
+  for (int q = 0; q < 4; ++q) {
+    const int c = q * 2 + eg;                          // 32-column chunk of the tile
+    const int jc = n0 + c * 32;
+    uint4 fr[4];
+    int grp[4];
+#pragma unroll
+    for (int sub = 0; sub < 4; ++sub) {
+      const int j = jc + sub * 8;
+      const bool ok = row_ok && j < p.d_in;
+      grp[sub] = ok ? j / p.group : -1;
+      fr[sub] = ok ? __ldg(reinterpret_cast<const uint4*>(g.F + (size_t)o * p.d_in + j)) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    uint32_t raw[32];
+    ptx::tmem_ld_32x32(tmem_acc + lane_base + (uint32_t)(c * 32), raw);
+    ptx::tmem_ld_wait();
+    float G[32];
+#pragma unroll
+    for (int e = 0; e < 32; ++e) G[e] = __uint_as_float(raw[e]);
+#pragma unroll
+    for (int sub = 0; sub < 4; ++sub) {
+      if (grp[sub] >= 0) {
+        if (grp[sub] != cur_grp) {
+          if (cur_grp >= 0) {
+            atomicAdd(&g.ds[(size_t)o * p.ngroups + cur_grp], p.grad_scale * ds_acc);
+            atomicAdd(&g.db[(size_t)o * p.ngroups + cur_grp], p.grad_scale * db_acc);
+          }
+          cur_grp = grp[sub]; ds_acc = 0.f; db_acc = 0.f;
+        }
+        const __half2* fh = reinterpret_cast<const __half2*>(&fr[sub]);
+#pragma unroll
+        for (int e2 = 0; e2 < 4; ++e2) {
+          const float2 f2 = __half22float2(fh[e2]);
+          const float fe[2] = {f2.x, f2.y};
+#pragma unroll
+          for (int e1 = 0; e1 < 2; ++e1) {
+            const int idx = sub * 8 + e2 * 2 + e1;
+            const float f = fe[e1], Gv = G[idx];
+            const bool inr = fabsf(f) < 1.f;           // STE gate m
+            ds_acc = fmaf(Gv, inr ? f : (f < 0.f ? p.qn : p.qp), ds_acc);
+            db_acc += inr ? 0.f : Gv;
+            G[idx] = inr ? Gv : 0.f;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) G[sub * 8 + e] = 0.f;
+      }
+    }
+    // Gm chunk -> shared memory: row t, 16-byte pieces eg * 4 + v of the quarter's 64-column tile
+    uint8_t* grow = gm + t * 128;
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      uint4 o4;
+      o4.x = pack_bf16x2(G[v * 8 + 0], G[v * 8 + 1]); o4.y = pack_bf16x2(G[v * 8 + 2], G[v * 8 + 3]);
+      o4.z = pack_bf16x2(G[v * 8 + 4], G[v * 8 + 5]); o4.w = pack_bf16x2(G[v * 8 + 6], G[v * 8 + 7]);
+      *reinterpret_cast<uint4*>(grow + (((eg * 4 + v) ^ (t & 7)) << 4)) = o4;
+    }
+    ptx::fence_proxy_async_smem();
+    ptx::tc_fence_before_sync();
+    ptx::named_bar_sync(3, EPI_THREADS);
+    if (t256 == 0 && !bars->abort) {
+      ptx::tc_fence_after_sync();
+      constexpr uint32_t idesc_db = ptx::make_idesc_bf16(128, RN, false, false);
+      constexpr uint32_t idesc_da = ptx::make_idesc_bf16(64, RN, true, false);
+      const uint32_t gm_a = ptx::smem_u32(gm), abf_a = ptx::smem_u32(abf), bt_a = ptx::smem_u32(btbf);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint64_t da = ptx::make_smem_desc_sw128(gm_a + k * 32, 16, 1024);
+        const uint64_t db = ptx::make_smem_desc_sw128(abf_a + q * (RN * 128) + k * 32, 16, 1024);
+        ptx::mma_bf16_ss(tmem_acc, da, db, idesc_db, (q | k) != 0 ? 1u : 0u);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint64_t da = ptx::make_smem_desc_sw128(gm_a + k * 2048, GMQ, 1024);   // one 64-column block: LBO unused
+        const uint64_t db = ptx::make_smem_desc_sw128(bt_a + (k >> 2) * (RN * 128) + (k & 3) * 32, 16, 1024);
+        ptx::mma_bf16_ss(tmem_acc + (uint32_t)(RN * (1 + q)), da, db, idesc_da, k != 0 ? 1u : 0u);
+      }
+      ptx::mma_commit(&bars->epi_mma);
+    }
+    bounded_wait(&bars->epi_mma, epi_phase, bars);     // Gm reusable; after the last quarter, results complete
+    epi_phase ^= 1;
+    ptx::tc_fence_after_sync();
+  }
+
+  if (row_ok && cur_grp >= 0) {
+    atomicAdd(&g.ds[(size_t)o * p.ngroups + cur_grp], p.grad_scale * ds_acc);
+    atomicAdd(&g.db[(size_t)o * p.ngroups + cur_grp], p.grad_scale * db_acc);
+  }
+  {  // dB: lane = weight row; group eg takes half of the ranks
+    constexpr int NB = RN / 2;
+    uint32_t r[NB];
+    tmem_ld_cols<NB>(tmem_acc + lane_base + (uint32_t)(eg * NB), r);
+    ptx::tmem_ld_wait();
+    if (row_ok) {
+#pragma unroll
+      for (int k = 0; k < NB; ++k)
+        if (eg * NB + k < RANK) atomicAdd(&g.dB[(size_t)o * RANK + eg * NB + k], p.gamma * __uint_as_float(r[k]));
+    }
+  }
+#pragma unroll
+  for (int qq = 0; qq < 2; ++qq) {  // dA: group eg takes quarters 2 eg and 2 eg + 1; lanes 0..15 of a warp hold 16 columns
+    const int q = eg * 2 + qq;
+    uint32_t r[RN];
+    tmem_ld_cols<RN>(tmem_acc + lane_base + (uint32_t)(RN * (1 + q)), r);
+    ptx::tmem_ld_wait();
+    const int col = n0 + q * 64 + quarter * 16 + lane;
+    if (lane < 16 && col < p.d_in) {
+#pragma unroll
+      for (int k = 0; k < RN; ++k)
+        if (k < RANK) atomicAdd(&g.dA[(size_t)k * p.d_in + col], p.gamma * __uint_as_float(r[k]));
+    }
+  }
+  ptx::tc_fence_before_sync();
+  ptx::mbar_arrive(tmem_empty_bar);
+}
+
 template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES, int TN = BN, bool EXT = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -409,7 +595,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const uint32_t tmem_base = bars->tmem_base;
 
   if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
+    // ------------------------------ TMA producer, operand A --------------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       WorkIter<TAIL_SPLIT> work(num_tiles, total_kb);
@@ -422,12 +608,10 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           bounded_wait(&bars->empty[stage], phase ^ 1, bars);
           if (bars->abort) break;
           uint8_t* sa = stage_base + (size_t)stage * STAGE_BYTES;
-          uint8_t* sb = sa + A_STAGE_BYTES;
-          ptx::mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
+          ptx::mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);   // the bytes of both operands
           // K blocks past the first operand pair come from the second one (same box shapes)
           const bool second = EXT && kb >= g.num_kb;
           const CUtensorMap* ma = second ? &tmap_a2 : &tmap_a;
-          const CUtensorMap* mb = second ? &tmap_b2 : &tmap_b;
           const int k0 = (second ? kb - g.num_kb : kb) * BK;
           if constexpr (!A_MN) {
             ptx::tma_load_2d(sa, ma, &bars->full[stage], k0, m0);
@@ -436,6 +620,31 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             for (int h = 0; h < BM / 64; ++h)
               ptx::tma_load_2d(sa + h * (64 * BK * 2), ma, &bars->full[stage], m0 + h * 64, k0);
           }
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 2) {
+    // ------------------------------ TMA producer, operand B --------------------
+    // A second issuing thread: an MN-major operand takes one copy per 64 columns, and one thread issuing all of
+    // a stage's copies was measurably on the critical path.  Its bytes count towards the same full barrier; they
+    // may land before warp 0 has announced the stage's byte count, which the barrier's transaction count allows.
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      WorkIter<TAIL_SPLIT> work(num_tiles, total_kb);
+      WorkUnit u;
+      while (!bars->abort && work.next(u)) {
+        int tm, tn;
+        tile_coords(u.tile, g.tiles_m, g.tiles_n, tm, tn);
+        const int n0 = tn * TN;
+        for (int kb = u.kb0; kb < u.kb1 && !bars->abort; ++kb) {
+          bounded_wait(&bars->empty[stage], phase ^ 1, bars);
+          if (bars->abort) break;
+          uint8_t* sb = stage_base + (size_t)stage * STAGE_BYTES + A_STAGE_BYTES;
+          const bool second = EXT && kb >= g.num_kb;
+          const CUtensorMap* mb = second ? &tmap_b2 : &tmap_b;
+          const int k0 = (second ? kb - g.num_kb : kb) * BK;
           if constexpr (!B_MN) {
             ptx::tma_load_2d(sb, mb, &bars->full[stage], k0, n0);
           } else {
@@ -552,8 +761,12 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
         }
       } else {
-        wgrad_epilogue_tile<RANK>(g, m0, n0, tmem_acc, quarter, lane, eg, epi_smem, bars, &bars->tmem_full[acc],
-                                  acc_phase, &bars->tmem_empty[acc], epi_phase);
+        if constexpr (wgrad_quarters(RANK))
+          wgrad_epilogue_tile_q<RANK>(g, m0, n0, tmem_acc, quarter, lane, eg, epi_smem, bars, &bars->tmem_full[acc],
+                                      acc_phase, &bars->tmem_empty[acc], epi_phase);
+        else
+          wgrad_epilogue_tile<RANK>(g, m0, n0, tmem_acc, quarter, lane, eg, epi_smem, bars, &bars->tmem_full[acc],
+                                    acc_phase, &bars->tmem_empty[acc], epi_phase);
       }
       if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1; }
     }
@@ -672,8 +885,8 @@ inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY
   g.A = A; g.B = B;
   g.dA = dA; g.dB = dB; g.ds = ds; g.db = db;
   switch (p.rank) {
-    case 8: return launch_gemm<true, true, EPI_WGRAD, 8, 3>(ta, tb, g, st);
-    case 16: return launch_gemm<true, true, EPI_WGRAD, 16, 3>(ta, tb, g, st);
+    case 8: return launch_gemm<true, true, EPI_WGRAD, 8, wgrad_stages(8)>(ta, tb, g, st);
+    case 16: return launch_gemm<true, true, EPI_WGRAD, 16, wgrad_stages(16)>(ta, tb, g, st);
     case 32: return launch_gemm<true, true, EPI_WGRAD, 32, 3>(ta, tb, g, st);
     case 64: return launch_gemm<true, true, EPI_WGRAD, 64, 3>(ta, tb, g, st);
     default: return L4Q_ERR_UNSUPPORTED;
