@@ -248,6 +248,12 @@ l4q_status l4q_linear_fwd_static(const l4q_desc* desc, const void* X, const void
                                  const float* A, const float* B, const float* s, const float* b,
                                  void* Y, void* cuda_stream);
 
+/* Exercises the error path of the kernels' bounded waits without touching any data: launches one block that
+ * waits on a barrier nothing arrives on, with a limit of about a millisecond.  The wait gives up and the kernel
+ * ends normally; the next l4q_check() on the stream returns L4Q_ERR_TIMEOUT (and clears it), after which the
+ * library works as before.  No counterpart in the paper.  Returns L4Q_OK if the launch succeeded. */
+l4q_status l4q_selftest_timeout(void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the device status word
  * (L4Q_OK, or L4Q_ERR_TIMEOUT if a kernel gave up on a bounded wait), or
  * L4Q_ERR_CUDA if the stream reported an error. */

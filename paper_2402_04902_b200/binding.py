@@ -28,7 +28,7 @@ EXPORTED_SYMBOLS = (
     "l4q_check", "l4q_launch_count", "l4q_status_string",
     "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
     "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error", "l4q_linear_infer", "l4q_adamw_step",
-    "l4q_lora_workspace_bytes", "l4q_lora_linear_fwd", "l4q_lora_linear_bwd",
+    "l4q_lora_workspace_bytes", "l4q_lora_linear_fwd", "l4q_lora_linear_bwd", "l4q_selftest_timeout",
 )
 L4Q_LORA_PLAIN, L4Q_LORA_QAT = 1, 2
 LORA_KINDS = {"lora": L4Q_LORA_PLAIN, "qat_lora": L4Q_LORA_QAT}
@@ -96,6 +96,8 @@ def lib() -> ctypes.CDLL:
         L.l4q_init_params.argtypes = [dp, vp, ctypes.c_int, fp, fp, vp]
         L.l4q_quant_error.restype = ctypes.c_int
         L.l4q_quant_error.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp]
+        L.l4q_selftest_timeout.restype = ctypes.c_int
+        L.l4q_selftest_timeout.argtypes = [vp]
         L.l4q_check.restype = ctypes.c_int
         L.l4q_check.argtypes = [vp]
         L.l4q_launch_count.restype = ctypes.c_uint64
@@ -237,6 +239,11 @@ def l4q_quant_error(desc: L4QDesc, W0, A, B, s, b, errors, stream=None) -> None:
     st = lib().l4q_quant_error(ctypes.byref(desc), _ptr(W0), _ptr(A), _ptr(B), _ptr(s), _ptr(b), _ptr(errors),
                                _stream(stream))
     _raise(st, "l4q_quant_error")
+
+
+def l4q_selftest_timeout(stream=None) -> None:
+    """Make one bounded device-side wait expire (about a millisecond); the next l4q_check raises L4Q_ERR_TIMEOUT."""
+    _raise(lib().l4q_selftest_timeout(_stream(stream)), "l4q_selftest_timeout")
 
 
 def l4q_check(stream=None) -> None:

@@ -571,6 +571,12 @@ l4q_status l4q_linear_fwd_static(const l4q_desc* desc, const void* X, const void
   return gemm_forward_bf16(p, X, wq, Y, stream);
 }
 
+l4q_status l4q_selftest_timeout(void* cuda_stream) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  k_selftest_timeout<<<1, 32, 0, stream>>>();
+  return launch_status();
+}
+
 l4q_status l4q_check(void* cuda_stream) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (cudaStreamSynchronize(stream) != cudaSuccess) return L4Q_ERR_CUDA;

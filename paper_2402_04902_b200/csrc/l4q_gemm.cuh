@@ -83,20 +83,36 @@ inline size_t gemm_smem_bytes(int stages, int epi_bytes, int stage_bytes = STAGE
 
 // Bounded mbarrier wait.  Returns immediately once the CTA's abort flag is set.
 template <class Barriers>
-__device__ __forceinline__ void bounded_wait(uint64_t* bar, uint32_t parity, Barriers* bars) {
+__device__ __forceinline__ void bounded_wait(uint64_t* bar, uint32_t parity, Barriers* bars,
+                                             long long limit_cycles = WAIT_LIMIT_CYCLES) {
   if (ptx::mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!ptx::mbar_try_wait(bar, parity)) {
     if ((++spins & 0xFFu) == 0) {
       if (bars->abort) return;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (clock64() - t0 > limit_cycles) {
         bars->abort = 1;
         atomicExch(&g_l4q_status, (unsigned int)L4Q_ERR_TIMEOUT);
         return;
       }
     }
   }
+}
+
+// Self-test of the error path of bounded_wait: one block waits on a barrier that nothing ever arrives on, with
+// a limit of about a millisecond.  The wait gives up, records L4Q_ERR_TIMEOUT and the kernel returns normally.
+struct SelftestBarriers { uint64_t never; volatile uint32_t abort; };
+
+__global__ void k_selftest_timeout() {
+  __shared__ SelftestBarriers bars;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bars.never, 1);
+    bars.abort = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) bounded_wait(&bars.never, 0, &bars, 2000000LL);
 }
 
 // Tile order: bands of 16 tile-rows; inside a band the row index runs fastest, so
