@@ -12,17 +12,18 @@
 //     each fp32 factor split into a tf32 head and a tf32 tail (x = hi + lo, three products hi*hi + hi*lo +
 //     lo*hi), which keeps ~21 mantissa bits -- the codes must agree with fp64 arithmetic except within
 //     1e-6 of a rounding boundary, which a single tf32 or bf16 product does not give;
-//   * 16 epilogue warps (thread = one weight row x 32 columns) read the merge from tensor memory with
-//     tcgen05.ld, the W0 tile from shared memory in 16-byte pieces, and do the quantizer arithmetic.
+//   * 16 epilogue warps in four groups; a group owns every fourth tile of the CTA and one of the four
+//     accumulator stages, a thread one weight row of the group's tile.  It reads the merge from tensor memory
+//     with tcgen05.ld, the W0 tile from shared memory in 16-byte pieces, and does the quantizer arithmetic.
+//     The groups meet only through mbarriers, so four tiles are in flight per SM and the wait chain of one
+//     tile hides behind the arithmetic of the others.
 //
 // Roles (640 threads): warp 0 = TMA loads, warp 1 = MMA issuer + TMEM owner, warp 2 = TMA stores (one
-// thread each), warps 4..19 = epilogue (warp w: TMEM lane quarter w % 4, column slice (w - 4) / 4).  The
-// epilogue threads also prepare the MMA operands (split the tile's slices of A and B into tf32 head / tail,
-// swizzled K-major): with two operand buffers (rank <= 32) they load the factors of tile t + 3 and store
-// those of tile t + 2 while working on tile t, so the merge runs two tiles ahead; with one buffer (rank 64)
-// the operands of tile t + 1 are built once the MMAs of tile t have completed.  s and b of a tile are copied
-// to shared memory one tile ahead by one thread per weight row.  Every mbarrier wait is bounded (see
-// bounded_wait); the one block-level barrier per tile is reached unconditionally by all epilogue threads.
+// thread each), warps 4..19 = epilogue (warp w: TMEM lane quarter w % 4, group (w - 4) / 4).  A group also
+// prepares the MMA operands of its next tile (splits the tile's slices of A and B into tf32 head / tail,
+// swizzled K-major) once the MMAs that last read the operand buffer have completed (two buffers up to rank
+// 32, one at rank 64), and copies s and b of its next tile's rows to per-thread scratch in shared memory.
+// Every mbarrier wait is bounded (see bounded_wait); there is no block-level barrier after set-up.
 #pragma once
 
 #include "l4q_common.cuh"
@@ -35,6 +36,8 @@ constexpr int WT2_ROWS = 128, WT2_COLS = 128;
 constexpr int WT2_THREADS = 640;
 constexpr int WT2_FIRST_EPI_WARP = 4;
 constexpr int WT2_EPI_THREADS = 512;
+constexpr int WT2_GROUPS = 2;                       // epilogue warp groups; each owns every second tile of the CTA
+constexpr int WT2_GROUP_THREADS = WT2_EPI_THREADS / WT2_GROUPS;
 constexpr int WT2_ACC = 4;                          // accumulator stages of 128 TMEM columns
 constexpr int WT2_STAGE_BYTES = WT2_ROWS * WT2_COLS * 2;   // one bf16 tile: two 128 x 64 swizzled boxes
 constexpr int WT2_ATOM_BYTES = 128 * 128;           // 128 rows x 32 tf32 (one 128-byte swizzle atom along K)
@@ -52,7 +55,7 @@ struct WtileArgs {
   int out_bytes;           // bytes of one such buffer
   int atoms;               // swizzle atoms per operand row: ceil(2 rank / 32)
   int ngt;                 // upper bound of the quantization groups a 128-column tile intersects
-  int n_opbuf;             // MMA operand buffers ([A slice | B slice] each): 2 up to rank 32, else 1
+  int n_opbuf;             // MMA operand buffers ([A slice | B slice] each): 1 or 2
   int group_shift;         // log2(group size) if it is a power of two, else -1
 };
 
@@ -72,8 +75,9 @@ struct __align__(8) WtileBarriers {
   volatile uint32_t abort;
 };
 
-// s and b of a tile in shared memory: two buffers of [128 rows][s x ngt | b x ngt] floats (1 KB multiples).
-__host__ __device__ inline size_t wtile_sb_bytes(int ngt) { return 2 * (size_t)WT2_ROWS * 2 * ngt * sizeof(float); }
+// s and b in shared memory: per epilogue thread [s x ngt | b x ngt] floats of its weight row (1 KB multiples
+// in total); a thread reads and writes its own entry only.
+__host__ __device__ inline size_t wtile_sb_bytes(int ngt) { return (size_t)WT2_EPI_THREADS * 2 * ngt * sizeof(float); }
 
 inline size_t wtile_smem_bytes(const WtileArgs& a) {
   return 1024 + (size_t)a.n_stages * WT2_STAGE_BYTES + (size_t)a.n_out * a.out_bytes +
@@ -84,23 +88,26 @@ inline size_t wtile_smem_bytes(const WtileArgs& a) {
 // consecutive) goes to CTA t mod gridDim.x.  Coordinates advance without divisions.
 struct TileCursor {
   int t, total, tm, tn, tiles_m, dm, dn;
-  __device__ explicit TileCursor(const WtileArgs& a) {
+  int step;
+  // the CTA's tiles number first, first + stride, ... of its own sequence
+  __device__ explicit TileCursor(const WtileArgs& a, int first = 0, int stride = 1) {
     total = a.tiles_m * a.tiles_n;
     tiles_m = a.tiles_m;
-    t = blockIdx.x;
+    t = blockIdx.x + first * (int)gridDim.x;
     tn = t / tiles_m; tm = t - tn * tiles_m;
-    dn = (int)gridDim.x / tiles_m; dm = (int)gridDim.x - dn * tiles_m;
+    step = stride * (int)gridDim.x;
+    dn = step / tiles_m; dm = step - dn * tiles_m;
   }
   __device__ bool valid() const { return t < total; }
   __device__ void next() {
-    t += gridDim.x; tn += dn; tm += dm;
+    t += step; tn += dn; tm += dm;
     if (tm >= tiles_m) { tm -= tiles_m; ++tn; }
   }
   __device__ int m0() const { return tm * WT2_ROWS; }
   __device__ int n0() const { return tn * WT2_COLS; }
   // coordinates of this CTA's tile k (small) steps ahead; false beyond the end
   __device__ bool peek(int k, int& m0_, int& n0_) const {
-    if (t + k * (int)gridDim.x >= total) return false;
+    if (t + k * step >= total) return false;
     int m = tm + k * dm, n = tn + k * dn;
     while (m >= tiles_m) { m -= tiles_m; ++n; }
     m0_ = m * WT2_ROWS; n0_ = n * WT2_COLS;
@@ -118,9 +125,10 @@ __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
 // MMA operands of one tile in shared memory, K-major with the 128-byte swizzle:
 //   acat row n = column n0 + n of the weight:  [ hi(A[0..r, col]) | lo(A[0..r, col]) ]
 //   bcat row m = row m0 + m of the weight:      [ hi(B[row, 0..r]) | lo(B[row, 0..r]) ]
-// A work item is 4 consecutive ranks (kc) of one row of both slices (32 r items per tile); a warp takes 32
-// consecutive rows of the same ranks, so its reads of A are coalesced and its 16-byte shared-memory writes
-// are conflict-free.
+// A work item (32 r per tile) is 4 consecutive ranks of one row of each slice.  Item idx takes column
+// idx % 128, ranks 4 (idx / 128) of the A slice -- a warp reads 32 consecutive columns of one rank, coalesced --
+// and the idx-th 16 bytes of the B slice, which is one contiguous block of 128 r floats, so a warp reads 512
+// consecutive bytes.
 struct OperandItem { float av[4]; float4 bv; };
 
 __device__ __forceinline__ void operand_item_load(const WtileArgs& a, int m0, int n0, int idx, OperandItem& it) {
@@ -128,13 +136,17 @@ __device__ __forceinline__ void operand_item_load(const WtileArgs& a, int m0, in
   const int row = idx & 127, kc = idx >> 7, col = n0 + row;
 #pragma unroll
   for (int e = 0; e < 4; ++e) it.av[e] = (col < p.d_in) ? __ldg(a.A + (size_t)(4 * kc + e) * p.d_in + col) : 0.f;
-  it.bv = (m0 + row < p.d_out) ? __ldg(reinterpret_cast<const float4*>(a.B + (size_t)(m0 + row) * p.rank + 4 * kc))
-                               : make_float4(0.f, 0.f, 0.f, 0.f);
+  const int rq = p.rank >> 2;                        // 16-byte pieces per row of B
+  const int brow = idx / rq;
+  it.bv = (m0 + brow < p.d_out) ? __ldg(reinterpret_cast<const float4*>(a.B + (size_t)m0 * p.rank) + idx)
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 __device__ __forceinline__ void operand_item_store(const WtileArgs& a, int idx, const OperandItem& it, uint8_t* acat,
                                                    uint8_t* bcat) {
   const int row = idx & 127, kc = idx >> 7;
+  const int rq = a.p.rank >> 2;
+  const int brow = idx / rq, bkc = idx - brow * rq;
   const float bvv[4] = {it.bv.x, it.bv.y, it.bv.z, it.bv.w};
   float ah[4], al[4], bh[4], bl[4];
 #pragma unroll
@@ -147,15 +159,17 @@ __device__ __forceinline__ void operand_item_store(const WtileArgs& a, int idx, 
   const uint32_t off_l = (uint32_t)(cl >> 3) * WT2_ATOM_BYTES + row * 128 + (((cl & 7) ^ (row & 7)) << 4);
   *reinterpret_cast<float4*>(acat + off_h) = make_float4(ah[0], ah[1], ah[2], ah[3]);
   *reinterpret_cast<float4*>(acat + off_l) = make_float4(al[0], al[1], al[2], al[3]);
-  *reinterpret_cast<float4*>(bcat + off_h) = make_float4(bh[0], bh[1], bh[2], bh[3]);
-  *reinterpret_cast<float4*>(bcat + off_l) = make_float4(bl[0], bl[1], bl[2], bl[3]);
+  const int bch = bkc, bcl = rq + bkc;
+  const uint32_t boff_h = (uint32_t)(bch >> 3) * WT2_ATOM_BYTES + brow * 128 + (((bch & 7) ^ (brow & 7)) << 4);
+  const uint32_t boff_l = (uint32_t)(bcl >> 3) * WT2_ATOM_BYTES + brow * 128 + (((bcl & 7) ^ (brow & 7)) << 4);
+  *reinterpret_cast<float4*>(bcat + boff_h) = make_float4(bh[0], bh[1], bh[2], bh[3]);
+  *reinterpret_cast<float4*>(bcat + boff_l) = make_float4(bl[0], bl[1], bl[2], bl[3]);
 }
 
 // Adding and subtracting 1.5 * 2^23 rounds |x| < 2^22 to the nearest integer, ties to even, exactly like
 // rintf, on the FP32 add pipe; the low mantissa bits of the intermediate sum hold that integer.
 constexpr float kRoundMagic = 12582912.0f;
 constexpr int kRoundMagicBits = 0x4B400000;
-constexpr int WT2_CARRY = 2;                        // operand items a thread carries between tiles (rank <= 32)
 
 template <int MODE>
 __global__ void __launch_bounds__(WT2_THREADS, 1)
@@ -179,13 +193,13 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     for (int i = 0; i < WT2_MAX_STAGES; ++i) {
       ptx::mbar_init(&bars->full[i], 1);
       ptx::mbar_init(&bars->empty[i], 1);
-      ptx::mbar_init(&bars->written[i], WT2_EPI_THREADS);
+      ptx::mbar_init(&bars->written[i], WT2_GROUP_THREADS);
     }
     for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->out_empty[i], 1);
-    for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->prep_full[i], WT2_EPI_THREADS);
+    for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->prep_full[i], WT2_GROUP_THREADS);
     for (int i = 0; i < WT2_ACC; ++i) {
       ptx::mbar_init(&bars->tmem_full[i], 1);
-      ptx::mbar_init(&bars->tmem_empty[i], WT2_EPI_THREADS);
+      ptx::mbar_init(&bars->tmem_empty[i], WT2_GROUP_THREADS);
     }
     bars->abort = 0;
     ptx::fence_mbar_init();
@@ -287,55 +301,54 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     __syncwarp();
   } else if (warp >= WT2_FIRST_EPI_WARP) {
     // ------------------------------ epilogue ----------------------------------
+    // Two groups of eight warps; group grp owns the CTA's tiles i = grp, grp + 2, ... (accumulator stage i % 4,
+    // operand buffer i % 2).  A thread is one weight row (TMEM lane) and one 64-column half of its group's
+    // tile.  The groups meet only through the mbarriers.  While a group works on tile i the merge of its tile
+    // i + 2 runs into the group's other accumulator stage, and with four W0 stages two loads are in flight.
     const int quarter = warp & 3;
-    const int sl = (warp - WT2_FIRST_EPI_WARP) >> 2;            // 32-column slice of the tile
+    const int grp = (warp - WT2_FIRST_EPI_WARP) >> 3;
+    const int chalf = ((warp - WT2_FIRST_EPI_WARP) >> 2) & 1;   // column half of the tile
     const int row = quarter * 32 + lane;
-    const int et = (warp - WT2_FIRST_EPI_WARP) * 32 + lane;
+    const int tg = chalf * WT2_ROWS + row;                       // thread index within the group
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    int stage = 0; uint32_t phase = 0;
-    int acc = 0; uint32_t acc_phase = 0;
-    int ob = 0; uint32_t out_round = 0;                         // completed rounds over the staging buffers
     const int r = p.rank;
-    const int L = a.n_opbuf;
+    const int L = a.n_opbuf;                                    // 1 or 2
     const int n_items = 32 * r;                                 // (row, 4 ranks) operand items per tile
+    const int sbw = 2 * a.ngt;                                  // floats per thread: s x ngt | b x ngt
+    float* grp_sb = sb_base + (size_t)grp * 2 * WT2_ROWS * sbw;   // two buffers of [128 rows][s x ngt | b x ngt]
 
-    // ---- MMA operands.  Two buffers (rank <= 32): the factors of tile i + 2 are loaded one tile before they
-    //      are stored, so the merge runs two tiles ahead and no load latency is exposed.  One buffer: the
-    //      operands of tile i + 1 are loaded and stored once the MMAs of tile i have completed. ----
-    auto prep_now = [&](int m0_, int n0_, int buf) {
-      uint8_t* acat = op_base + (size_t)buf * 2 * op_half;
-      for (int idx = et; idx < n_items; idx += WT2_EPI_THREADS) {
+    // ---- MMA operands of tile j (CTA sequence number), built by the group that owns the tile.  With two
+    //      operand buffers the buffer of tile j was last read by the MMAs of tile j - 2, the group's own
+    //      previous tile, which the caller has already seen complete; with one buffer by those of tile j - 1. ----
+    auto prep_buffer_wait = [&](int j) {
+      if (L == 1 && j >= 1) {
+        bounded_wait(&bars->tmem_full[(j - 1) & 3], (uint32_t)(((j - 1) >> 2) & 1), bars);
+        ptx::tc_fence_after_sync();
+      }
+    };
+    auto prep = [&](int j, int m0_, int n0_) {
+      prep_buffer_wait(j);
+      uint8_t* acat = op_base + (size_t)(j & (L - 1)) * 2 * op_half;
+      for (int idx = tg; idx < n_items; idx += WT2_GROUP_THREADS) {
         OperandItem it_;
         operand_item_load(a, m0_, n0_, idx, it_);
         operand_item_store(a, idx, it_, acat, acat + op_half);
       }
-    };
-    OperandItem carry[WT2_CARRY];
-    auto carry_load = [&](int m0_, int n0_) {
-#pragma unroll
-      for (int j = 0; j < WT2_CARRY; ++j)
-        if (et + j * WT2_EPI_THREADS < n_items) operand_item_load(a, m0_, n0_, et + j * WT2_EPI_THREADS, carry[j]);
-    };
-    auto carry_store = [&](int buf) {
-      uint8_t* acat = op_base + (size_t)buf * 2 * op_half;
-#pragma unroll
-      for (int j = 0; j < WT2_CARRY; ++j)
-        if (et + j * WT2_EPI_THREADS < n_items)
-          operand_item_store(a, et + j * WT2_EPI_THREADS, carry[j], acat, acat + op_half);
+      ptx::fence_proxy_async_smem();
+      ptx::mbar_arrive(&bars->prep_full[j & (L - 1)]);
     };
 
-    // ---- s and b reach the arithmetic through shared memory: the four warps of column slice 0 (one thread
-    //      per weight row) copy the tile's values of their row, one tile ahead, with asynchronous 4-byte
-    //      copies; all epilogue threads meet at a barrier at the end of every tile.  (Loading them per thread
-    //      touches 32 different lines per instruction, sixteen times over, and starves the TMA loads.) ----
-    const int sbw = 2 * a.ngt;                                  // floats per row: s x ngt | b x ngt
+    // ---- s and b of the tile's rows for the quantization groups it intersects: the threads of column half 0
+    //      (one per weight row) copy them with asynchronous 4-byte copies into the group's buffer for its next
+    //      tile; the group meets at a named barrier when it starts that tile.  (Each row's values sit in a line
+    //      of their own, so every copy instruction touches 32 lines: the fewer of them the better.) ----
     auto stage_sb = [&](int m0_, int n0_, int buf) {
-      if (sl != 0) return;
-      float* dst = sb_base + ((size_t)buf * WT2_ROWS + row) * sbw;
+      if (chalf != 0) return;
+      float* dst = grp_sb + ((size_t)buf * WT2_ROWS + row) * sbw;
       const int o_ = m0_ + row;
-      const int g_first = group_of(a, n0_);
+      const int gf = group_of(a, n0_);
       for (int k = 0; k < a.ngt; ++k) {
-        const int g = g_first + k;
+        const int g = gf + k;
         if (o_ < p.d_out && g < p.ngroups) {
           ptx::cp_async_4(dst + k, a.s + (size_t)o_ * p.ngroups + g);
           ptx::cp_async_4(dst + a.ngt + k, a.b + (size_t)o_ * p.ngroups + g);
@@ -346,170 +359,134 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       ptx::cp_async_commit();
     };
 
-    // ---- quantization groups of the four 8-column pieces this thread owns (g % 8 == 0: one group each).
-    //      They depend on the tile's column only and are recomputed when it changes. ----
-    int gi[4] = {0, 0, 0, 0};                                   // group index relative to the tile's first group
-    uint32_t first_mask = 0, valid_mask = 0;                    // bit sub: first piece of its group / inside d_in
-    int g_first = 0, groups_n0 = -1;
-    auto set_groups = [&](int n0_) {
-      const int jc = n0_ + sl * 32;
-      g_first = group_of(a, n0_);
-      const int g0 = group_of(a, jc);
-      const int rem0 = jc - g0 * p.group;
-      first_mask = 0; valid_mask = 0;
-#pragma unroll
-      for (int sub = 0; sub < 4; ++sub) {
-        int rem = rem0 + sub * 8, g = g0;
-#pragma unroll
-        for (int c = 0; c < 3; ++c)
-          if (rem >= p.group) { rem -= p.group; ++g; }
-        gi[sub] = g - g_first;
-        if (rem == 0) first_mask |= 1u << sub;
-        if (jc + sub * 8 < p.d_in) valid_mask |= 1u << sub;
-      }
-      groups_n0 = n0_;
-    };
-
-    // ------------------------------ prologue ------------------------------
-    TileCursor cur(a);
-    {
-      int mb, nb;
-      if (cur.valid()) stage_sb(cur.m0(), cur.n0(), 0);
-      for (int k = 0; k < L; ++k) {
-        if (cur.peek(k, mb, nb)) {
-          prep_now(mb, nb, k);
-          ptx::fence_proxy_async_smem();
-          ptx::mbar_arrive(&bars->prep_full[k]);
-        }
-      }
-      if (L == 2 && cur.peek(2, mb, nb)) carry_load(mb, nb);
-      ptx::cp_async_wait_all();
+    TileCursor cur(a, grp, WT2_GROUPS);
+    if (cur.valid()) {
+      stage_sb(cur.m0(), cur.n0(), 0);
+      prep(grp, cur.m0(), cur.n0());
     }
-    ptx::named_bar_sync(1, WT2_EPI_THREADS);
+    int sb_buf = 0;
     const int qn_bits = kRoundMagicBits + (int)p.qn;
 
-    for (int i = 0; cur.valid(); cur.next(), ++i) {
+    for (int i = grp; cur.valid(); cur.next(), i += WT2_GROUPS) {
       const int m0 = cur.m0(), n0 = cur.n0();
       const int o = m0 + row;
       const bool row_ok = o < p.d_out;
-      if (n0 != groups_n0) set_groups(n0);
-      float sv[4], bv[4];
-      {
-        const float* src = sb_base + ((size_t)(i & 1) * WT2_ROWS + row) * sbw;
-#pragma unroll
-        for (int sub = 0; sub < 4; ++sub) {
-          const bool ok = row_ok && ((valid_mask >> sub) & 1u);
-          sv[sub] = ok ? src[gi[sub]] : 1.f;
-          bv[sub] = ok ? src[a.ngt + gi[sub]] : 0.f;
-        }
-      }
-      bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
+      const int stage = i % a.n_stages;
+      const uint32_t phase = (uint32_t)((i / a.n_stages) & 1);
+      const int acc = i & 3;
+      const int g_first = group_of(a, n0);
+      int m1 = 0, n1 = 0;
+      const bool has_next = cur.peek(1, m1, n1);
+      ptx::cp_async_wait_all();                                 // this thread's copies of the tile's s, b have landed
+      ptx::named_bar_sync(1 + grp, WT2_GROUP_THREADS);          // ... and so have the group's
+      const float* my_sb = grp_sb + ((size_t)sb_buf * WT2_ROWS + row) * sbw;
+      bounded_wait(&bars->tmem_full[acc], (uint32_t)((i >> 2) & 1), bars);
       ptx::tc_fence_after_sync();
-      {  // the MMAs of this tile have completed: its operand buffer is free for the tile L steps ahead
-        int m1, n1;
-        const int buf = i % L;
-        if (cur.peek(L, m1, n1)) {
-          if (L == 2) carry_store(buf); else prep_now(m1, n1, 0);
-          ptx::fence_proxy_async_smem();
-          ptx::mbar_arrive(&bars->prep_full[buf]);
-        }
-        if (L == 2 && cur.peek(3, m1, n1)) carry_load(m1, n1);
-        if (cur.peek(1, m1, n1)) stage_sb(m1, n1, (i + 1) & 1);
-      }
-
+      // the merge of this tile is complete: the operands of the group's next tile can take its buffer
+      if (has_next) prep(i + WT2_GROUPS, m1, n1);
       bounded_wait(&bars->full[stage], phase, bars);
+      int ob = 0;
       if constexpr (HAS_OUT1) {
-        if (out_round > 0) bounded_wait(&bars->out_empty[ob], (out_round - 1) & 1, bars);
+        ob = i % a.n_out;
+        if (i >= a.n_out) bounded_wait(&bars->out_empty[ob], (uint32_t)((i / a.n_out - 1) & 1), bars);
       }
-      uint8_t* wrow = stage_base + (size_t)stage * WT2_STAGE_BYTES + (sl >> 1) * (WT2_STAGE_BYTES / 2) + row * 128;
+      uint8_t* tile_rows = stage_base + (size_t)stage * WT2_STAGE_BYTES + row * 128;
       [[maybe_unused]] uint8_t* out1 = out_base + (size_t)ob * a.out_bytes;
-      [[maybe_unused]] uint32_t words[4] = {0u, 0u, 0u, 0u};    // WT2_PACK: this thread's 32 codes
-      float rs = 1.f;
+      float rs = 1.f, s_ = 1.f, b_ = 0.f;
+      int cur_g = -1;
+#pragma unroll 1
+      for (int bb = 0; bb < 2; ++bb) {                          // 32 columns
+        const int blk = chalf * 2 + bb;
+        [[maybe_unused]] uint32_t words[4] = {0u, 0u, 0u, 0u};  // WT2_PACK: the 32 codes of this block
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {                    // 16 columns at a time
-        uint32_t raw[16];
-        ptx::tmem_ld_32x16(tmem_base + lane_base + (uint32_t)(acc * WT2_COLS + sl * 32 + half * 16), raw);
-        ptx::tmem_ld_wait();
-        if (half == 1) {
-          ptx::tc_fence_before_sync();
-          ptx::mbar_arrive(&bars->tmem_empty[acc]);
-        }
+        for (int half = 0; half < 2; ++half) {                  // 16 columns at a time
+          uint32_t raw[16];
+          ptx::tmem_ld_32x16(tmem_base + lane_base + (uint32_t)(acc * WT2_COLS + blk * 32 + half * 16), raw);
+          ptx::tmem_ld_wait();
+          if (bb == 1 && half == 1) {
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&bars->tmem_empty[acc]);
+          }
 #pragma unroll
-        for (int s2 = 0; s2 < 2; ++s2) {
-          const int sub = half * 2 + s2;
-          const uint32_t chunk = (uint32_t)((((sl & 1) * 4 + sub) ^ (row & 7)) << 4);
-          const uint4 wr = *reinterpret_cast<const uint4*>(wrow + chunk);
-          const float w0[8] = {bf16_lo(wr.x), bf16_hi(wr.x), bf16_lo(wr.y), bf16_hi(wr.y),
-                               bf16_lo(wr.z), bf16_hi(wr.z), bf16_lo(wr.w), bf16_hi(wr.w)};
-          if (sub == 0 || ((first_mask >> sub) & 1u)) rs = 1.0f / sv[sub];        // one reciprocal per group
-          const float s_ = sv[sub], b_ = bv[sub];
-          float wq[8], fac[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            // Eq. 7-9 and the STE factor: the arithmetic of quantize_elem / ste_factor, with the rounding
-            // done by the magic-number add (exact for the clamped range)
-            const float wc = merge_elem(w0[e], __uint_as_float(raw[s2 * 8 + e]), p.gamma);
-            const float w = (wc - b_) * rs;
-            const float wcl = fminf(fmaxf(w, p.qn), p.qp);
-            const float y = wcl + kRoundMagic;
-            const float code = y - kRoundMagic;
-            wq[e] = fmaf(code, s_, b_);
-            if constexpr (MODE == WT2_DEQUANT_F) {
-              const float t = w - wcl;                                            // 0 inside [Q_N, Q_P]
-              const float sentinel = __uint_as_float((__float_as_uint(t) & 0x80000000u) | 0x40000000u);   // +-2
-              fac[e] = (fabsf(t) > kMaskGuard) ? sentinel : code - w;
+          for (int s2 = 0; s2 < 2; ++s2) {
+            const int sub = half * 2 + s2;
+            const int piece = blk * 4 + sub;                    // 8-column piece of the tile (g % 8 == 0: one group)
+            const int col = n0 + piece * 8;
+            const bool ok = row_ok && col < p.d_in;
+            const int g = group_of(a, col);
+            const bool group_start = (col - g * p.group) == 0;
+            if (g != cur_g) {                                   // one reciprocal per group
+              cur_g = g;
+              s_ = ok ? my_sb[g - g_first] : 1.f;
+              b_ = ok ? my_sb[a.ngt + g - g_first] : 0.f;
+              rs = 1.0f / s_;
             }
-            if constexpr (MODE == WT2_PACK) {                                     // code j of 32 at bit j * bits
-              const uint32_t u = (uint32_t)(__float_as_int(y) - qn_bits);
-              const int j = sub * 8 + e;
-              if (p.bits == 4) {
-                words[j >> 3] |= u << ((j & 7) * 4);
-              } else {
-                const int bit = j * 3, wd = bit >> 5, off = bit & 31;
-                words[wd] |= u << off;
-                if (off > 29) words[wd + 1] |= u >> (32 - off);
+            const uint32_t chunk = (uint32_t)((piece >> 3) * (WT2_STAGE_BYTES / 2) + (((piece & 7) ^ (row & 7)) << 4));
+            const uint4 wr = *reinterpret_cast<const uint4*>(tile_rows + chunk);
+            const float w0[8] = {bf16_lo(wr.x), bf16_hi(wr.x), bf16_lo(wr.y), bf16_hi(wr.y),
+                                 bf16_lo(wr.z), bf16_hi(wr.z), bf16_lo(wr.w), bf16_hi(wr.w)};
+            float wq[8], fac[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              // Eq. 7-9 and the STE factor: the arithmetic of quantize_elem / ste_factor, with the rounding
+              // done by the magic-number add (exact for the clamped range)
+              const float wc = merge_elem(w0[e], __uint_as_float(raw[s2 * 8 + e]), p.gamma);
+              const float w = (wc - b_) * rs;
+              const float wcl = fminf(fmaxf(w, p.qn), p.qp);
+              const float y = wcl + kRoundMagic;
+              const float code = y - kRoundMagic;
+              wq[e] = fmaf(code, s_, b_);
+              if constexpr (MODE == WT2_DEQUANT_F) {
+                const float t = w - wcl;                                            // 0 inside [Q_N, Q_P]
+                const float sentinel = __uint_as_float((__float_as_uint(t) & 0x80000000u) | 0x40000000u);   // +-2
+                fac[e] = (fabsf(t) > kMaskGuard) ? sentinel : code - w;
+              }
+              if constexpr (MODE == WT2_PACK) {                                     // code j of 32 at bit j * bits
+                const uint32_t u = (uint32_t)(__float_as_int(y) - qn_bits);
+                const int j = sub * 8 + e;
+                if (p.bits == 4) {
+                  words[j >> 3] |= u << ((j & 7) * 4);
+                } else {
+                  const int bit = j * 3, wd = bit >> 5, off = bit & 31;
+                  words[wd] |= u << off;
+                  if (off > 29) words[wd + 1] |= u >> (32 - off);
+                }
+              }
+            }
+            if constexpr (MODE != WT2_PACK) {
+              uint4 o4;
+              o4.x = pack_bf16x2(wq[0], wq[1]); o4.y = pack_bf16x2(wq[2], wq[3]);
+              o4.z = pack_bf16x2(wq[4], wq[5]); o4.w = pack_bf16x2(wq[6], wq[7]);
+              *reinterpret_cast<uint4*>(tile_rows + chunk) = o4;                    // in place, same swizzled position
+            }
+            if constexpr (MODE == WT2_DEQUANT_F) {
+              __half2 h[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) h[e] = __floats2half2_rn(fac[2 * e], fac[2 * e + 1]);
+              *reinterpret_cast<uint4*>(out1 + row * 128 + chunk) = *reinterpret_cast<const uint4*>(h);
+            }
+            if constexpr (MODE == WT2_PACK) {
+              if (ok && group_start) {                                              // first piece of its group
+                a.s16[(size_t)o * p.ngroups + g] = __float2half_rn(s_);
+                a.b16[(size_t)o * p.ngroups + g] = __float2half_rn(fmaf(s_, p.qn, b_));
               }
             }
           }
-          if constexpr (MODE != WT2_PACK) {
-            uint4 o4;
-            o4.x = pack_bf16x2(wq[0], wq[1]); o4.y = pack_bf16x2(wq[2], wq[3]);
-            o4.z = pack_bf16x2(wq[4], wq[5]); o4.w = pack_bf16x2(wq[6], wq[7]);
-            *reinterpret_cast<uint4*>(wrow + chunk) = o4;                         // in place, same swizzled position
-          }
-          if constexpr (MODE == WT2_DEQUANT_F) {
-            __half2 h[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) h[e] = __floats2half2_rn(fac[2 * e], fac[2 * e + 1]);
-            *reinterpret_cast<uint4*>(out1 + (sl >> 1) * (WT2_STAGE_BYTES / 2) + row * 128 + chunk) =
-                *reinterpret_cast<const uint4*>(h);
-          }
-          if constexpr (MODE == WT2_PACK) {
-            if (row_ok && ((valid_mask & first_mask) >> sub) & 1u) {              // first piece of its group
-              a.s16[(size_t)o * p.ngroups + g_first + gi[sub]] = __float2half_rn(s_);
-              a.b16[(size_t)o * p.ngroups + g_first + gi[sub]] = __float2half_rn(fmaf(s_, p.qn, b_));
-            }
-          }
         }
-      }
-      if constexpr (MODE == WT2_PACK) {
-        // staging row = the tile's 128 codes of this weight row; this thread owns 32 of them
-        if (p.bits == 4) {
-          *reinterpret_cast<uint4*>(out1 + row * 64 + sl * 16) = make_uint4(words[0], words[1], words[2], words[3]);
-        } else {
-          uint32_t* dst = reinterpret_cast<uint32_t*>(out1 + row * 48 + sl * 12);
-          dst[0] = words[0]; dst[1] = words[1]; dst[2] = words[2];
+        if constexpr (MODE == WT2_PACK) {
+          // staging row = the tile's 128 codes of this weight row; this block is 32 of them
+          if (p.bits == 4) {
+            *reinterpret_cast<uint4*>(out1 + row * 64 + blk * 16) = make_uint4(words[0], words[1], words[2], words[3]);
+          } else {
+            uint32_t* dst = reinterpret_cast<uint32_t*>(out1 + row * 48 + blk * 12);
+            dst[0] = words[0]; dst[1] = words[1]; dst[2] = words[2];
+          }
         }
       }
       ptx::fence_proxy_async_smem();                   // the stores above are read by TMA
       ptx::mbar_arrive(&bars->written[stage]);
-      ptx::cp_async_wait_all();                        // this thread's copies of the next tile's s, b have landed
-      ptx::named_bar_sync(1, WT2_EPI_THREADS);         // ... and so have everyone's
-      if (++stage == a.n_stages) { stage = 0; phase ^= 1; }
-      if (++acc == WT2_ACC) { acc = 0; acc_phase ^= 1; }
-      if constexpr (HAS_OUT1) {
-        if (++ob == a.n_out) { ob = 0; ++out_round; }
-      }
+      sb_buf ^= 1;
+      if (has_next) stage_sb(m1, n1, sb_buf);          // the other buffer: its readers passed this tile's barrier
     }
   }
 
@@ -543,29 +520,32 @@ inline bool make_tmap_words(CUtensorMap* m, const void* base, uint64_t rows, uin
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Shared-memory plan: LoRA operands first, then as many W0 stages as fit (a second staging buffer for
-// the extra output only if three stages still fit beside it).
+// Shared-memory plan.  A tile being worked on holds one W0 stage and, when there is a second output, one
+// staging buffer for it: two of each keep both epilogue groups busy, further stages let the loads run ahead.
+// Candidates in order of preference (a single operand buffer makes every merge wait for the previous one).
 inline bool wtile_plan(WtileArgs& a, int mode) {
   const Params& p = a.p;
   a.atoms = (2 * p.rank + 31) / 32;
   a.ngt = std::min(p.ngroups, (WT2_COLS - 1) / p.group + 2);
-  a.n_opbuf = (32 * p.rank <= WT2_CARRY * WT2_EPI_THREADS) ? 2 : 1;
   a.group_shift = -1;
   for (int sh = 3; sh < 31; ++sh)
     if ((1 << sh) == p.group) a.group_shift = sh;
   a.out_bytes = mode == WT2_DEQUANT_F ? WT2_STAGE_BYTES : mode == WT2_PACK ? WT2_ROWS * (WT2_COLS * p.bits / 8) : 0;
-  const long long budget = 227 * 1024 - 1024 - (long long)sizeof(WtileBarriers) -
-                           2LL * a.n_opbuf * a.atoms * WT2_ATOM_BYTES -
-                           (long long)wtile_sb_bytes(a.ngt);
-  a.n_out = a.out_bytes ? 2 : 0;
-  long long stages = (budget - (long long)a.n_out * a.out_bytes) / WT2_STAGE_BYTES;
-  if (a.n_out == 2 && stages < 3) {
-    a.n_out = 1;
-    stages = (budget - a.out_bytes) / WT2_STAGE_BYTES;
+  struct Cand { int opbuf, n_out, stages; };
+  static const Cand plain[] = {{2, 0, 4}, {1, 0, 4}, {2, 0, 3}, {1, 0, 3}, {2, 0, 2}, {1, 0, 2}};
+  static const Cand small_out[] = {{2, 2, 4}, {1, 2, 4}, {2, 2, 3},
+                                   {1, 2, 3}, {2, 2, 2}, {1, 2, 2}, {1, 1, 2}};
+  static const Cand big_out[] = {{2, 2, 3}, {1, 2, 3}, {2, 2, 2}, {1, 2, 2}, {2, 1, 3}, {1, 1, 3},
+                                 {2, 1, 2}, {1, 1, 2}};
+  const Cand* cands = mode == WT2_DEQUANT ? plain : mode == WT2_PACK ? small_out : big_out;
+  const int n_cands = mode == WT2_DEQUANT ? 6 : mode == WT2_PACK ? 7 : 8;
+  const int max_opbuf = p.rank <= 32 ? 2 : 1;       // rank 64: the split operands of one tile are already 128 KB
+  for (int c = 0; c < n_cands; ++c) {
+    if (cands[c].opbuf > max_opbuf) continue;
+    a.n_opbuf = cands[c].opbuf; a.n_out = cands[c].n_out; a.n_stages = cands[c].stages;
+    if (wtile_smem_bytes(a) <= 227 * 1024) return true;
   }
-  if (stages < 2) return false;
-  a.n_stages = (int)std::min<long long>(stages, WT2_MAX_STAGES);
-  return true;
+  return false;
 }
 
 // Whether the tensor-core weight-tile kernel covers this problem (otherwise the plain-ALU kernel runs).
