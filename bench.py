@@ -22,6 +22,10 @@ and the parameter gradients are all-reduced (sum) over NCCL each step.
 l4q_lora_linear_fwd / l4q_lora_linear_bwd, for the per-step cost comparison (no export step; the
 flop count is that layer's own).  The default, `--layer l4q`, is the benchmark proper.
 
+`--op extras` times the kernels outside the training step -- inference from the packed export (few tokens),
+quantizer initialisation, the error sums and the AdamW update -- each against the HBM roofline, and prints its
+own JSON line (not the benchmark line).
+
 `--impl reference` times the fp64 CPU oracle (oracle/), as it stands, on the
 host cores on a bounded slice of the same workload.
 """
@@ -438,6 +442,110 @@ def run_ours(args, layers, wl_name):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------
+# kernels outside the training step (--op extras)
+# --------------------------------------------------------------------------
+
+def run_extras(args):
+    """Device times (the library's per-launch CUDA events) of l4q_linear_infer, l4q_init_params, l4q_quant_error
+    and l4q_adamw_step on LLaMA-7B-shaped operands, with the bytes each must move.  Weights are rotated over
+    enough copies to exceed L2, as the layers of a model would."""
+    import torch
+
+    from paper_2402_04902_b200 import binding as l4q
+    from paper_2402_04902_b200 import build as l4q_build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    l4q_build.build()
+    l4q.lib()
+    pk_ = peaks()
+    dev = torch.device("cuda", 0)
+    reps = max(args.steps, 5)
+    out = {}
+
+    def timed(name_key, fn, n_calls):
+        for _ in range(args.warmup):
+            fn(0)
+        torch.cuda.synchronize()
+        l4q.l4q_profile_enable(False)
+        l4q.l4q_profile_enable(True)
+        for k in range(n_calls):
+            fn(k)
+        torch.cuda.synchronize()
+        n, ms = l4q.l4q_profile_read()[name_key]
+        l4q.l4q_profile_enable(False)
+        l4q.l4q_check()
+        return ms / max(n, 1) * 1e3                               # us per launch
+
+    L2_BYTES = 126e6
+    # ---- inference from the export (App. F): few tokens, weights streamed from HBM ----
+    for d_in, d_out in ((4096, 11008), (11008, 4096), (4096, 4096)):
+        cfg = synth.CONFIG3A.with_(name=f"infer_{d_in}x{d_out}", d_in=d_in, d_out=d_out, tokens=64)
+        arrays = synth.make_layer_inputs(cfg, seed=0, need_acts=False)
+        d = l4q.to_device(cfg, arrays, device=dev)
+        desc = l4q.make_desc(cfg)
+        pk = l4q.alloc_pack_outputs(cfg, device=dev)
+        l4q.l4q_pack_int(desc, d["W0"], d["A"], d["B"], d["s"], d["b"], pk["codes"], pk["s16"], pk["b16"])
+        wbytes = pk["codes"].numel() * 4 + pk["s16"].numel() * 4
+        copies = int(L2_BYTES * 1.5 // wbytes) + 1
+        ring = [{k: v.clone() for k, v in pk.items()} for _ in range(copies)]
+        for tokens in (1, 2, 16, 64):
+            dsc = l4q.make_desc(cfg, tokens=tokens)
+            X = torch.randn(tokens, d_in, device=dev).to(torch.bfloat16)
+            Y = torch.empty(tokens, d_out, dtype=torch.bfloat16, device=dev)
+
+            def call(k, dsc=dsc, X=X, Y=Y):
+                w = ring[k % copies]
+                l4q.l4q_linear_infer(dsc, X, w["codes"], w["s16"], w["b16"], Y)
+
+            us = timed("infer", call, reps * copies)
+            nbytes = wbytes + tokens * (d_in + d_out) * 2
+            out[f"infer_{d_in}x{d_out}_t{tokens}"] = {"us": us, "bytes": nbytes, "gbs": nbytes / us / 1e3,
+                                                       "frac_hbm": nbytes / us / 1e3 / pk_["hbm_gbs"],
+                                                       "dense_bf16_bytes": d_in * d_out * 2}
+        del ring
+
+    # ---- initialisation of s, b (App. B) and the error sums (Table 4): one pass over a bf16 weight ----
+    cfg = synth.CONFIG3A
+    arrays = synth.make_layer_inputs(cfg, seed=0, need_acts=False)
+    d = l4q.to_device(cfg, arrays, device=dev)
+    desc = l4q.make_desc(cfg)
+    wbytes = cfg.d_out * cfg.d_in * 2
+    copies = int(L2_BYTES * 1.5 // wbytes) + 1
+    Ws = [d["W0"].clone() for _ in range(copies)]
+    G = cfg.d_in // cfg.group_size
+    s_out = torch.empty(cfg.d_out, G, device=dev)
+    b_out = torch.empty(cfg.d_out, G, device=dev)
+    for method in ("lsq+", "symm", "asymm", "l4q"):
+        us = timed("init", lambda k, m=method: l4q.l4q_init_params(desc, Ws[k % copies], m, s_out, b_out), reps * copies)
+        nbytes = wbytes + 2 * s_out.numel() * 4
+        out[f"init_{method}_4096x11008"] = {"us": us, "bytes": nbytes, "gbs": nbytes / us / 1e3,
+                                            "frac_hbm": nbytes / us / 1e3 / pk_["hbm_gbs"]}
+    err = torch.zeros(2, dtype=torch.float64, device=dev)
+    us = timed("error", lambda k: l4q.l4q_quant_error(desc, Ws[k % copies], d["A"], d["B"], d["s"], d["b"], err),
+               reps * copies)
+    nbytes = wbytes + 2 * s_out.numel() * 4
+    out["quant_error_4096x11008"] = {"us": us, "bytes": nbytes, "gbs": nbytes / us / 1e3,
+                                     "frac_hbm": nbytes / us / 1e3 / pk_["hbm_gbs"]}
+    del Ws
+
+    # ---- AdamW (App. D): 4 reads + 3 writes of fp32 per element ----
+    n = 64 * 1024 * 1024
+    p_, g_, m_, v_ = (torch.randn(n, device=dev) for _ in range(4))
+    v_.abs_()
+    us = timed("adamw", lambda k: l4q.l4q_adamw_step(p_, g_, m_, v_, k + 1, 1e-4), reps)
+    out["adamw_64Mi"] = {"us": us, "bytes": 28 * n, "gbs": 28 * n / us / 1e3, "frac_hbm": 28 * n / us / 1e3 / pk_["hbm_gbs"]}
+    # the size the layer really has: A, B, s, b of the 4096 -> 11008 linear
+    n2 = cfg.rank * (cfg.d_in + cfg.d_out) + 2 * cfg.d_out * G
+    us = timed("adamw", lambda k: l4q.l4q_adamw_step(p_[:n2], g_[:n2], m_[:n2], v_[:n2], k + 1, 1e-4), reps * 8)
+    out["adamw_layer_params"] = {"us": us, "elements": n2, "bytes": 28 * n2}
+
+    print(json.dumps({"op": "extras", "unit": "us per launch (CUDA events around each launch)", "hbm_peak_gbs": pk_["hbm_gbs"],
+                      "peak_source": pk_["source"], "l2": "weights rotated over copies totalling 1.5x L2",
+                      "kernels": out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -447,7 +555,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layer", default="l4q", choices=["l4q", "lora", "qat_lora"],
                     help="l4q = the benchmark; lora / qat_lora = the comparison layers (ours arm only)")
+    ap.add_argument("--op", default="train", choices=["train", "extras"],
+                    help="train = the benchmark; extras = inference / initialisation / error sums / AdamW kernels")
     args = ap.parse_args()
+    if args.op == "extras":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_extras(args)
+        return
     layers = workloads()[args.workload]
     if args.impl == "reference":
         run_reference(args, layers, args.workload)

@@ -481,6 +481,18 @@ l4q_status l4q_init_params(const l4q_desc* desc, const void* W, int method, floa
   const int blocks = (int)std::min<long long>((groups + 7) / 8, (long long)sm_count() * 16);
   const bool signed_grid = (desc->flags & L4Q_FLAG_SIGNED_GRID) != 0;
   KernelScope ks(L4Q_KERNEL_INIT, stream);
+  int lanes_log2 = -1;                                   // group = 8 * 2^k elements with k <= 5: the coalesced kernel
+  for (int k = 0; k <= 5; ++k)
+    if (p.group == (8 << k)) lanes_log2 = k;
+  if (lanes_log2 >= 0) {
+    const long long pieces = (long long)p.d_out * p.d_in / 8;
+    const int vblocks = (int)std::min<long long>((pieces + 1023) / 1024, 1LL << 20);   // one sweep: blocks balance themselves
+    if (desc->io_dtype == L4Q_BF16)
+      k_init_params_vec<true><<<vblocks, 256, 0, stream>>>(p, method, signed_grid, lanes_log2, W, s, b);
+    else
+      k_init_params_vec<false><<<vblocks, 256, 0, stream>>>(p, method, signed_grid, lanes_log2, W, s, b);
+    return launch_status();
+  }
   if (desc->io_dtype == L4Q_BF16) k_init_params<true><<<blocks, 256, 0, stream>>>(p, method, signed_grid, W, s, b);
   else k_init_params<false><<<blocks, 256, 0, stream>>>(p, method, signed_grid, W, s, b);
   return launch_status();

@@ -233,6 +233,70 @@ k_init_params(Params p, int method, bool signed_grid, const void* __restrict__ W
   }
 }
 
+// The same initialisation for groups of 8, 16, ..., 256 elements (a power of two of 8-element pieces, at most
+// one warp wide): the weight is walked as one linear array of pieces, lane = piece, so every load of a warp is 512
+// contiguous bytes and four of them are in flight per thread; the lanes of a group reduce with shuffles, and the
+// variance of LSQ+ is taken from the values still in registers.
+template <bool IO_BF16>
+__global__ void __launch_bounds__(256)
+k_init_params_vec(Params p, int method, bool signed_grid, int lanes_log2, const void* __restrict__ W,
+                  float* __restrict__ s_out, float* __restrict__ b_out) {
+  constexpr int U = 4;
+  const int lane = threadIdx.x & 31;
+  const int lpg = 1 << lanes_log2;                         // lanes (pieces) per group
+  const long long total = (long long)p.d_out * p.d_in / 8;  // pieces; a multiple of lpg
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long nthreads = (long long)gridDim.x * blockDim.x;
+  const float qn_s = -(float)(1 << (p.bits - 1)), qp_s = (float)((1 << (p.bits - 1)) - 1);
+  const float inv_n = 1.f / (float)p.group;
+  for (long long w0 = tid - lane; w0 < total; w0 += nthreads * U) {
+    float v[U][8];
+    bool ok[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const long long q = w0 + (long long)u * nthreads + lane;
+      ok[u] = q < total;
+      if (ok[u]) load_w0_vec8<IO_BF16>(W, (size_t)q * 8, v[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      float lo = INFINITY, hi = -INFINITY, sum = 0.f;
+      if (ok[u]) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { lo = fminf(lo, v[u][j]); hi = fmaxf(hi, v[u][j]); sum += v[u][j]; }
+      }
+      for (int off = lpg >> 1; off > 0; off >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, off));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, off));
+        sum += __shfl_xor_sync(0xffffffffu, sum, off);
+      }
+      float sc = 0.f, bs = 0.f;
+      if (method == INIT_LSQ_PLUS) {
+        const float mu = sum * inv_n;
+        float ss = 0.f;
+        if (ok[u]) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) ss = fmaf(v[u][j] - mu, v[u][j] - mu, ss);
+        }
+        for (int off = lpg >> 1; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        const float sigma = sqrtf(ss * inv_n);
+        sc = fmaxf(fabsf(mu - 3.f * sigma), fabsf(mu + 3.f * sigma)) / (float)(1 << (p.bits - 1));
+      } else if (method == INIT_SYMM) {
+        sc = fmaxf(fabsf(lo), fabsf(hi)) / (float)(1 << (p.bits - 1));
+      } else if (method == INIT_ASYMM) {
+        sc = fmaxf((hi - lo) / (qp_s - qn_s), 1e-8f);
+        bs = signed_grid ? lo - sc * qn_s : lo;
+      } else {
+        sc = fmaxf(fabsf(lo / qn_s), fabsf(hi / qp_s));
+      }
+      sc = fmaxf(sc, 1e-8f);
+      if (!signed_grid && method != INIT_ASYMM) bs = sc * qn_s;
+      const long long q = w0 + (long long)u * nthreads + lane;
+      if (ok[u] && (lane & (lpg - 1)) == 0) { s_out[q >> lanes_log2] = sc; b_out[q >> lanes_log2] = bs; }
+    }
+  }
+}
+
 // One AdamW update of a parameter tensor (App. D: AdamW, decoupled weight decay), everything in one pass:
 //   p <- p - lr wd p;  m <- b1 m + (1 - b1) g;  v <- b2 v + (1 - b2) g^2;  p <- p - lr (m / c1) / (sqrt(v / c2) + eps)
 // with the bias corrections c1 = 1 - b1^t, c2 = 1 - b2^t computed on the host in double precision.

@@ -20,6 +20,13 @@ CASES = [
                       io_dtype="f32"),
     synth.LayerConfig("init_wide_group", tokens=8, d_in=1024, d_out=64, rank=8, alpha=16.0, bits=4,
                       group_size=512),
+    # the coalesced kernel at both ends of its range (1 and 32 lanes per group), with a ragged last warp,
+    # and more pieces than one sweep of the grid covers
+    synth.LayerConfig("init_group8", tokens=8, d_in=136, d_out=24, rank=8, alpha=16.0, bits=4, group_size=8,
+                      signed_grid=True),
+    synth.LayerConfig("init_group256", tokens=8, d_in=768, d_out=40, rank=8, alpha=16.0, bits=3, group_size=256),
+    synth.LayerConfig("init_many_pieces", tokens=8, d_in=4096, d_out=2048, rank=8, alpha=16.0, bits=4,
+                      group_size=64),
 ]
 
 
