@@ -62,6 +62,17 @@ def test_infer_llama7b_mlp_up_batch_16():
     _run(synth.CONFIG3A.with_(name="infer_cfg3a_b16", tokens=16), seed=0)
 
 
+@pytest.mark.parametrize("d_in,d_out,tokens,bits", [(4096, 1000, 1, 4), (4096, 1000, 4, 4), (11008, 520, 1, 4),
+                                                    (11008, 520, 2, 4), (14336, 264, 1, 4), (4096, 392, 2, 3),
+                                                    (11008, 392, 1, 3), (11008, 392, 3, 4)])
+def test_infer_matrix_vector_shapes(d_in, d_out, tokens, bits):
+    # one to four tokens on full-length rows (4096, 11008, 14336 values of k), output widths that leave a ragged
+    # last tile, both bit widths: the matrix-vector kernel up to two tokens, the tensor-core kernel beyond
+    cfg = synth.LayerConfig(f"infer_mv_{d_in}_{tokens}_{bits}", tokens=tokens, d_in=d_in, d_out=d_out, rank=8,
+                            alpha=16.0, bits=bits, group_size=128 if bits == 4 else 64)
+    _run(cfg, seed=5)
+
+
 def test_infer_rejects_what_it_does_not_cover():
     gh.ensure_built()
     cfg = synth.LayerConfig("infer_bad_group", tokens=4, d_in=1040, d_out=64, rank=8, alpha=16.0, bits=4,
