@@ -187,6 +187,8 @@ __host__ __device__ constexpr int wgrad_epi_smem_bytes(int rank) {
   return wgrad_gm_bytes(rank) + 6 * wgrad_rn(rank) * 128;
 }
 __host__ __device__ constexpr int wgrad_stages(int rank) { return wgrad_quarters(rank) ? 4 : 3; }
+constexpr int STORE_BOX_BYTES = 128 * 64 * 2;       // one staging box of the store epilogue: 128 rows x 64 columns bf16
+__host__ __device__ constexpr int store_epi_smem_bytes() { return EPI_GROUPS * STORE_BOX_BYTES; }
 
 template <int N>
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[N]) {
@@ -571,7 +573,8 @@ __device__ __forceinline__ void wgrad_epilogue_tile_q(const GemmArgs& g, int m0,
 template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES, int TN = BN, bool EXT = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-            const __grid_constant__ CUtensorMap tmap_a2, const __grid_constant__ CUtensorMap tmap_b2, const GemmArgs g) {
+            const __grid_constant__ CUtensorMap tmap_a2, const __grid_constant__ CUtensorMap tmap_b2,
+            const __grid_constant__ CUtensorMap tmap_c, const GemmArgs g) {
   static_assert(TN == 64 || TN == BN, "tile width");
   static_assert(EPI != EPI_WGRAD || (TN == BN && !EXT), "the weight-gradient epilogue works on 256-column tiles");
   constexpr int STAGE_BYTES = stage_bytes_for(TN);           // shadows the 256-column figure
@@ -579,7 +582,11 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
-  constexpr int EPI_SMEM = (EPI == EPI_WGRAD) ? wgrad_epi_smem_bytes(RANK) : 0;
+  // EPI_STORE on 256-column tiles leaves through shared memory and TMA stores: one 128 x 64 staging box per
+  // epilogue group.  (Stores from registers, one weight row per thread, touch 32 lines per instruction and cost
+  // the forward GEMM an eighth of its time.)
+  constexpr bool TMA_STORE = (EPI == EPI_STORE && TN == BN);
+  constexpr int EPI_SMEM = (EPI == EPI_WGRAD) ? wgrad_epi_smem_bytes(RANK) : TMA_STORE ? store_epi_smem_bytes() : 0;
   uint8_t* epi_smem = smem + (size_t)STAGES * STAGE_BYTES;
   GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + (size_t)STAGES * STAGE_BYTES + EPI_SMEM);
 
@@ -600,6 +607,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     ptx::prefetch_tmap(&tmap_a);
     ptx::prefetch_tmap(&tmap_b);
     if constexpr (EXT) { ptx::prefetch_tmap(&tmap_a2); ptx::prefetch_tmap(&tmap_b2); }
+    if constexpr (TMA_STORE) ptx::prefetch_tmap(&tmap_c);
   }
   if (warp == 1) {
     ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -746,6 +754,41 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
               if (n0 + c * 32 + e < g.N) atomicAdd(dst + e, g.scale * __uint_as_float(raw[e]));
           }
         }
+      } else if constexpr (EPI == EPI_STORE && TMA_STORE) {
+        bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
+        ptx::tc_fence_after_sync();
+        const int t = quarter * 32 + lane;                       // row in tile = TMEM lane = thread of the group
+        uint8_t* stg = epi_smem + eg * STORE_BOX_BYTES;
+#pragma unroll 1
+        for (int b = 0; b < 2; ++b) {                            // the group's 128 columns as two boxes of 64
+          uint32_t raw[2][32];
+          ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(eg * 128 + b * 64), raw[0]);
+          ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(eg * 128 + b * 64 + 32), raw[1]);
+          ptx::tmem_ld_wait();
+          if (b == 1) {
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&bars->tmem_empty[acc]);
+          }
+          if (t == 0) ptx::bulk_wait_group_read0();              // the previous store has read the staging box
+          ptx::named_bar_sync(1 + eg, 128);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {                          // 16-byte pieces of the row, 128-byte swizzle
+            const uint32_t* r = raw[j >> 2] + (j & 3) * 8;
+            uint4 o4;
+            o4.x = pack_bf16x2(__uint_as_float(r[0]), __uint_as_float(r[1]));
+            o4.y = pack_bf16x2(__uint_as_float(r[2]), __uint_as_float(r[3]));
+            o4.z = pack_bf16x2(__uint_as_float(r[4]), __uint_as_float(r[5]));
+            o4.w = pack_bf16x2(__uint_as_float(r[6]), __uint_as_float(r[7]));
+            *reinterpret_cast<uint4*>(stg + t * 128 + ((j ^ (t & 7)) << 4)) = o4;
+          }
+          ptx::fence_proxy_async_smem();
+          ptx::named_bar_sync(1 + eg, 128);
+          // rows and columns beyond C are clipped by the copy; a box that lies outside altogether is not issued
+          if (t == 0 && !bars->abort && n0 + eg * 128 + b * 64 < g.N && m0 < g.M) {
+            ptx::tma_store_2d(&tmap_c, stg, n0 + eg * 128 + b * 64, m0);
+            ptx::bulk_commit_group();
+          }
+        }
       } else if constexpr (EPI == EPI_STORE) {
         bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
         ptx::tc_fence_after_sync();
@@ -789,6 +832,9 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   }
 
   // ------------------------------ teardown ------------------------------------
+  if constexpr (TMA_STORE) {
+    if (warp >= EPI_FIRST_WARP && (warp & 3) == 0 && lane == 0) ptx::bulk_wait_group0();   // this thread's stores have landed
+  }
   if (bars->abort) {
     // give copies that are still in flight time to land before the block's shared memory is released
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
@@ -850,19 +896,23 @@ inline int sm_count() {
 template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES, int TN = BN, bool EXT = false>
 l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g, cudaStream_t st,
                        const CUtensorMap* ta2 = nullptr, const CUtensorMap* tb2 = nullptr) {
+  constexpr bool TMA_STORE = (EPI == EPI_STORE && TN == BN);
+  CUtensorMap tc = ta;                                  // placeholder where the epilogue does not store by TMA
+  if (TMA_STORE && !make_tmap_bf16(&tc, g.C, (uint64_t)g.M, (uint64_t)g.N, 128)) return L4Q_ERR_CUDA;
   g.tiles_m = ceil_div(g.M, BM);
   g.tiles_n = ceil_div(g.N, TN);
   g.num_kb = ceil_div(g.K, BK);
   if (!EXT) g.num_kb2 = 0;
   if (EXT && (!ta2 || !tb2)) return L4Q_ERR_INVALID_ARG;
   auto kern = k_gemm_bf16<A_MN, B_MN, EPI, RANK, STAGES, TN, EXT>;
-  const size_t smem = gemm_smem_bytes(STAGES, EPI == EPI_WGRAD ? wgrad_epi_smem_bytes(RANK) : 0, stage_bytes_for(TN));
+  const size_t smem = gemm_smem_bytes(STAGES, EPI == EPI_WGRAD ? wgrad_epi_smem_bytes(RANK)
+                                              : TMA_STORE ? store_epi_smem_bytes() : 0, stage_bytes_for(TN));
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return L4Q_ERR_CUDA;
   const int tiles = g.tiles_m * g.tiles_n, sms = sm_count();
   int grid = std::min(tiles, sms);
   if (EPI != EPI_STORE && tiles < sms) grid = tiles * std::min(sms / tiles, g.num_kb);   // K slices for the idle SMs
-  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, EXT ? *ta2 : ta, EXT ? *tb2 : tb, g);
+  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, EXT ? *ta2 : ta, EXT ? *tb2 : tb, tc, g);
   return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
 }
 
