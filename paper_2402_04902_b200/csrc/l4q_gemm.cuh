@@ -55,6 +55,7 @@ enum { EPI_STORE = 0, EPI_WGRAD = 1, EPI_ADD_F32 = 2 };
 struct GemmArgs {
   int M, N, K;                 // GEMM extents
   int tiles_m, tiles_n, num_kb;
+  int band;                    // tile rows per band of the tile order (see tile_coords)
   int num_kb2;                 // EXT: K blocks taken from the second pair of tensor maps, after the first num_kb
   // EPI_STORE
   __nv_bfloat16* C;            // [M, N] row-major
@@ -115,10 +116,10 @@ __global__ void k_selftest_timeout() {
   if (threadIdx.x == 0) bounded_wait(&bars.never, 0, &bars, 2000000LL);
 }
 
-// Tile order: bands of 16 tile-rows; inside a band the row index runs fastest, so
-// a wave of ~148 tiles touches ~16 row panels and ~9 column panels (L2 reuse).
-__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tm, int& tn) {
-  constexpr int GROUP = 16;
+// Tile order: bands of `GROUP` tile-rows; inside a band the row index runs fastest, so a wave of ~148 tiles
+// touches GROUP row panels and ~148 / GROUP column panels.  The A panels of a band stay in L2 while the B
+// panels stream past once per band, so the band is made as tall as L2 allows (tile_band_rows).
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int GROUP, int& tm, int& tn) {
   const int per_band = GROUP * tiles_n;
   const int band = t / per_band;
   const int first = band * GROUP;
@@ -626,7 +627,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       WorkUnit u;
       while (!bars->abort && work.next(u)) {
         int tm, tn;
-        tile_coords(u.tile, g.tiles_m, g.tiles_n, tm, tn);
+        tile_coords(u.tile, g.tiles_m, g.tiles_n, g.band, tm, tn);
         const int m0 = tm * BM, n0 = tn * TN;
         for (int kb = u.kb0; kb < u.kb1 && !bars->abort; ++kb) {
           bounded_wait(&bars->empty[stage], phase ^ 1, bars);
@@ -660,7 +661,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       WorkUnit u;
       while (!bars->abort && work.next(u)) {
         int tm, tn;
-        tile_coords(u.tile, g.tiles_m, g.tiles_n, tm, tn);
+        tile_coords(u.tile, g.tiles_m, g.tiles_n, g.band, tm, tn);
         const int n0 = tn * TN;
         for (int kb = u.kb0; kb < u.kb1 && !bars->abort; ++kb) {
           bounded_wait(&bars->empty[stage], phase ^ 1, bars);
@@ -729,7 +730,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     WorkUnit u;
     while (work.next(u)) {
       int tm, tn;
-      tile_coords(u.tile, g.tiles_m, g.tiles_n, tm, tn);
+      tile_coords(u.tile, g.tiles_m, g.tiles_n, g.band, tm, tn);
       const int m0 = tm * BM, n0 = tn * TN;
       const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * TN);
       if constexpr (EPI == EPI_ADD_F32) {
@@ -881,6 +882,22 @@ inline bool make_tmap_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tile rows per band: as many A panels (128 rows x K, bf16) as fit in half of L2, the rest being left to the
+// streamed operand and the output; at least 8, and split evenly so that the last band is not a sliver.
+inline int tile_band_rows(int tiles_m, size_t a_panel_bytes) {
+  static size_t l2 = 0;
+  if (!l2) {
+    int dev = 0, bytes = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&bytes, cudaDevAttrL2CacheSize, dev);
+    l2 = bytes > 0 ? (size_t)bytes : (size_t)96 << 20;
+  }
+  int rows = (int)std::max<size_t>(8, (l2 / 2) / std::max<size_t>(a_panel_bytes, 1));
+  rows = std::min(rows, tiles_m);
+  const int bands = ceil_div(tiles_m, rows);
+  return ceil_div(tiles_m, bands);
+}
+
 inline int sm_count() {
   static int n = 0;
   if (!n) {
@@ -902,6 +919,9 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
   g.tiles_m = ceil_div(g.M, BM);
   g.tiles_n = ceil_div(g.N, TN);
   g.num_kb = ceil_div(g.K, BK);
+  // measured: the taller band helps the GEMMs that write a large output; the weight-gradient GEMM, whose last
+  // wave is cut along K, is better off with 16 rows
+  g.band = EPI == EPI_STORE ? tile_band_rows(g.tiles_m, (size_t)BM * g.K * 2) : std::min(16, g.tiles_m);
   if (!EXT) g.num_kb2 = 0;
   if (EXT && (!ta2 || !tb2)) return L4Q_ERR_INVALID_ARG;
   auto kern = k_gemm_bf16<A_MN, B_MN, EPI, RANK, STAGES, TN, EXT>;
