@@ -102,7 +102,7 @@ size_t wq_scratch_bytes(const l4q_desc* d) {
 }
 
 size_t factor_scratch_bytes(const l4q_desc* d) {
-  return align_up((size_t)d->d_out * (size_t)d->d_in * sizeof(__half), 256);
+  return align_up(factor_elems((int)d->d_out, (int)d->d_in) * sizeof(__half), 256);
 }
 
 inline l4q_status launch_status() { return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA; }

@@ -74,4 +74,17 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Layout of the STE factor array that the weight-tile kernel hands to the weight-gradient kernel (internal, in the
+// workspace): tiles of 128 rows x 128 columns, each one contiguous block of 32 KB ordered [piece of 8 columns]
+// [row][8 values], tiles row-major over (row tile, column tile).  A thread that owns a weight row reads 16 bytes
+// per piece, and the 32 rows of a warp are then 512 contiguous bytes; the producer writes a tile as one bulk copy.
+constexpr int FACTOR_TILE_ELEMS = 128 * 128;
+__host__ __device__ inline int factor_tiles_n(int d_in) { return (d_in + 127) >> 7; }
+__host__ __device__ inline size_t factor_index(int o, int col, int tiles_n) {
+  return ((((size_t)(o >> 7) * tiles_n + (col >> 7)) * 16 + ((col & 127) >> 3)) * 128 + (o & 127)) * 8 + (col & 7);
+}
+__host__ __device__ inline size_t factor_elems(int d_out, int d_in) {
+  return (size_t)((d_out + 127) >> 7) * factor_tiles_n(d_in) * FACTOR_TILE_ELEMS;
+}
+
 }  // namespace l4q

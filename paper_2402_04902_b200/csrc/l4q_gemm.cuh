@@ -65,7 +65,8 @@ struct GemmArgs {
   float scale;
   // EPI_WGRAD (M = d_out, N = d_in)
   Params p;
-  const __half* F;             // [d_out, d_in] STE factors of the weights (ste_factor)
+  const __half* F;             // STE factors of the weights (ste_factor), in the factor_index layout
+  int f_tiles_n;               // column tiles of that layout
   const float *A, *B;
   float *dA, *dB, *ds, *db;
 };
@@ -279,7 +280,7 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
         const int j = jc + sub * 8;
         const bool ok = row_ok && j < p.d_in;
         grp[sub] = ok ? j / p.group : -1;
-        fr[sub] = ok ? __ldg(reinterpret_cast<const uint4*>(g.F + (size_t)o * p.d_in + j)) : make_uint4(0u, 0u, 0u, 0u);
+        fr[sub] = ok ? __ldg(reinterpret_cast<const uint4*>(g.F + factor_index(o, j, g.f_tiles_n))) : make_uint4(0u, 0u, 0u, 0u);
       }
       uint32_t raw[32];
       ptx::tmem_ld_32x32(tmem_acc + lane_base + (uint32_t)(c * 32), raw);
@@ -465,7 +466,7 @@ __device__ __forceinline__ void wgrad_epilogue_tile_q(const GemmArgs& g, int m0,
       const int j = jc + sub * 8;
       const bool ok = row_ok && j < p.d_in;
       grp[sub] = ok ? j / p.group : -1;
-      fr[sub] = ok ? __ldg(reinterpret_cast<const uint4*>(g.F + (size_t)o * p.d_in + j)) : make_uint4(0u, 0u, 0u, 0u);
+      fr[sub] = ok ? __ldg(reinterpret_cast<const uint4*>(g.F + factor_index(o, j, g.f_tiles_n))) : make_uint4(0u, 0u, 0u, 0u);
     }
     uint32_t raw[32];
     ptx::tmem_ld_32x32(tmem_acc + lane_base + (uint32_t)(c * 32), raw);
@@ -968,6 +969,7 @@ inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY
   g.M = p.d_out; g.N = p.d_in; g.K = p.tokens;
   g.p = p;
   g.F = reinterpret_cast<const __half*>(F);
+  g.f_tiles_n = factor_tiles_n(p.d_in);
   g.A = A; g.B = B;
   g.dA = dA; g.dB = dB; g.ds = ds; g.db = db;
   switch (p.rank) {

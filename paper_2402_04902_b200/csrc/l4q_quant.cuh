@@ -121,7 +121,7 @@ k_weight_tile(Params p, const void* __restrict__ W0, const float* __restrict__ A
           __half2 h[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) h[j] = __floats2half2_rn(fac[2 * j], fac[2 * j + 1]);
-          *reinterpret_cast<uint4*>(f_out + (size_t)o * p.d_in + col) = *reinterpret_cast<const uint4*>(h);
+          *reinterpret_cast<uint4*>(f_out + factor_index(o, col, factor_tiles_n(p.d_in))) = *reinterpret_cast<const uint4*>(h);
         }
         if constexpr (IO_BF16) {
           uint4 out;

@@ -49,6 +49,7 @@ struct WtileArgs {
   Params p;
   const float *A, *B, *s, *b;
   __half *s16, *b16;       // WT2_PACK
+  __half* F;               // WT2_DEQUANT_F: the factor array (factor_index layout)
   int tiles_m, tiles_n;
   int n_stages;            // W0 stages in shared memory (2..4)
   int n_out;               // staging buffers for the second output (F or codes): 0, 1 or 2
@@ -283,8 +284,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
           if (second_box) ptx::tma_store_2d(&tmap_out0, src + WT2_STAGE_BYTES / 2, n0 + 64, m0);
         }
         if constexpr (MODE == WT2_DEQUANT_F) {
-          ptx::tma_store_2d(&tmap_out1, src1, n0, m0);
-          if (second_box) ptx::tma_store_2d(&tmap_out1, src1 + WT2_STAGE_BYTES / 2, n0 + 64, m0);
+          // the staging buffer is the tile's block of the factor array as it stands: one contiguous copy
+          ptx::bulk_store(a.F + ((size_t)cur.tm * a.tiles_n + cur.tn) * FACTOR_TILE_ELEMS, src1, WT2_STAGE_BYTES);
         }
         if constexpr (MODE == WT2_PACK) ptx::tma_store_2d(&tmap_out0, src1, (n0 * p.bits) >> 5, m0);
         ptx::bulk_commit_group();
@@ -463,7 +464,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
               __half2 h[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) h[e] = __floats2half2_rn(fac[2 * e], fac[2 * e + 1]);
-              *reinterpret_cast<uint4*>(out1 + row * 128 + chunk) = *reinterpret_cast<const uint4*>(h);
+              *reinterpret_cast<uint4*>(out1 + (piece * WT2_ROWS + row) * 16) = *reinterpret_cast<const uint4*>(h);
             }
             if constexpr (MODE == WT2_PACK) {
               if (ok && group_start) {                                              // first piece of its group
@@ -578,7 +579,7 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
       return L4Q_ERR_CUDA;
   } else {
     if (!make_tmap_bf16(&t_o0, out0, p.d_out, p.d_in, WT2_ROWS)) return L4Q_ERR_CUDA;
-    if (mode == WT2_DEQUANT_F && !make_tmap_bf16(&t_o1, out1, p.d_out, p.d_in, WT2_ROWS)) return L4Q_ERR_CUDA;
+    a.F = reinterpret_cast<__half*>(out1);
   }
   const size_t smem = wtile_smem_bytes(a);
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
