@@ -692,6 +692,14 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       // blocks along M/N are one TMA box (BK rows x 128 B) apart; a K step of 16 is two row groups.
       constexpr uint32_t A_LBO = A_MN ? (BK * 128) : 16, A_SBO = 1024, A_KSTEP = A_MN ? 2048 : 32;
       constexpr uint32_t B_LBO = B_MN ? (BK * 128) : 16, B_SBO = 1024, B_KSTEP = B_MN ? 2048 : 32;
+      // This thread shares its scheduler with two epilogue warps, so every instruction here waits its turn: the
+      // loop is kept to a barrier poll, one add per descriptor and the MMAs.  A descriptor's low word is the start
+      // address (in 16-byte units, below 2^14) plus the leading-dimension offset, the high word is constant;
+      // stages and K steps are plain increments of the low word.
+      constexpr uint32_t DESC_HI = ((1024u >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);   // SBO, version 1, 128-byte swizzle
+      const uint32_t a_lo0 = ((ptx::smem_u32(stage_base) >> 4) & 0x3FFFu) | (((A_LBO >> 4) & 0x3FFFu) << 16);
+      const uint32_t b_lo0 = (((ptx::smem_u32(stage_base) + A_STAGE_BYTES) >> 4) & 0x3FFFu) | (((B_LBO >> 4) & 0x3FFFu) << 16);
+      static_assert(A_SBO == 1024 && B_SBO == 1024, "descriptor high word");
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       WorkIter<TAIL_SPLIT> work(num_tiles, total_kb);
@@ -701,17 +709,17 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         if (bars->abort) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TN);
+        uint32_t accumulate = 0;
         for (int kb = u.kb0; kb < u.kb1; ++kb) {
-          bounded_wait(&bars->full[stage], phase, bars);
-          if (bars->abort) break;
+          bounded_wait(&bars->full[stage], phase, bars);   // on a time-out the wait returns and the abort flag ends the tile loop
           ptx::tc_fence_after_sync();
-          const uint32_t sa = ptx::smem_u32(stage_base + (size_t)stage * STAGE_BYTES);
-          const uint32_t sb = sa + A_STAGE_BYTES;
+          const uint32_t al = a_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4), bl = b_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t da = ptx::make_smem_desc_sw128(sa + k * A_KSTEP, A_LBO, A_SBO);
-            const uint64_t db = ptx::make_smem_desc_sw128(sb + k * B_KSTEP, B_LBO, B_SBO);
-            ptx::mma_bf16_ss(d_tmem, da, db, idesc, (kb != u.kb0 || k != 0) ? 1u : 0u);
+            const uint64_t da = ((uint64_t)DESC_HI << 32) | (al + k * (A_KSTEP >> 4));
+            const uint64_t db = ((uint64_t)DESC_HI << 32) | (bl + k * (B_KSTEP >> 4));
+            ptx::mma_bf16_ss(d_tmem, da, db, idesc, accumulate);
+            accumulate = 1;
           }
           ptx::mma_commit(&bars->empty[stage]);       // smem stage reusable once these MMAs retire
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
