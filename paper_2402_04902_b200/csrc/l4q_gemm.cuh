@@ -630,9 +630,10 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         int tm, tn;
         tile_coords(u.tile, g.tiles_m, g.tiles_n, g.band, tm, tn);
         const int m0 = tm * BM, n0 = tn * TN;
-        for (int kb = u.kb0; kb < u.kb1 && !bars->abort; ++kb) {
+        // (no flag check in this loop: it would be a shared-memory load on the critical path of a thread that shares
+        // its scheduler with two epilogue warps; a wait that times out returns, and the abort flag ends the tile loop)
+        for (int kb = u.kb0; kb < u.kb1; ++kb) {
           bounded_wait(&bars->empty[stage], phase ^ 1, bars);
-          if (bars->abort) break;
           uint8_t* sa = stage_base + (size_t)stage * STAGE_BYTES;
           ptx::mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);   // the bytes of both operands
           // K blocks past the first operand pair come from the second one (same box shapes)
@@ -664,9 +665,10 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         int tm, tn;
         tile_coords(u.tile, g.tiles_m, g.tiles_n, g.band, tm, tn);
         const int n0 = tn * TN;
-        for (int kb = u.kb0; kb < u.kb1 && !bars->abort; ++kb) {
+        // (no flag check in this loop: it would be a shared-memory load on the critical path of a thread that shares
+        // its scheduler with two epilogue warps; a wait that times out returns, and the abort flag ends the tile loop)
+        for (int kb = u.kb0; kb < u.kb1; ++kb) {
           bounded_wait(&bars->empty[stage], phase ^ 1, bars);
-          if (bars->abort) break;
           uint8_t* sb = stage_base + (size_t)stage * STAGE_BYTES + A_STAGE_BYTES;
           const bool second = EXT && kb >= g.num_kb;
           const CUtensorMap* mb = second ? &tmap_b2 : &tmap_b;
