@@ -135,9 +135,8 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
       int stage = 0; uint32_t phase = 0;
       for (int t = blockIdx.x; t < num_tiles && !bars->abort; t += gridDim.x) {
         const int m0 = (t / a.tiles_n) * INF_M;
-        for (int kb = 0; kb < a.num_kb && !bars->abort; ++kb) {
+        for (int kb = 0; kb < a.num_kb; ++kb) {      // no flag loads here: see the GEMM producers
           bounded_wait(&bars->empty_op[stage], phase ^ 1, bars);
-          if (bars->abort) break;
           // only the rows that hold tokens are copied; the other rows of the operand are never stored
           // from (an MMA output row depends on its own input row only)
           ptx::mbar_arrive_expect_tx(&bars->full_x[stage], (uint32_t)(2 * a.x_rows * 128));
@@ -154,9 +153,8 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
       int cs = 0; uint32_t cphase = 0;
       for (int t = blockIdx.x; t < num_tiles && !bars->abort; t += gridDim.x) {
         const int n0 = (t % a.tiles_n) * N;
-        for (int kb = 0; kb < a.num_kb && !bars->abort; ++kb) {
+        for (int kb = 0; kb < a.num_kb; ++kb) {      // no flag loads here: see the GEMM producers
           bounded_wait(&bars->empty_c[cs], cphase ^ 1, bars);
-          if (bars->abort) break;
           ptx::mbar_arrive_expect_tx(&bars->full_c[cs], (uint32_t)(N * CW * 4));
           ptx::tma_load_2d(c_tile(cs), &tmap_c, &bars->full_c[cs], kb * CW, n0);
           if (++cs == INF_C_STAGES) { cs = 0; cphase ^= 1; }
@@ -178,7 +176,6 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
         for (int kb = 0; kb < a.num_kb; ++kb) {
           bounded_wait(&bars->full_x[stage], phase, bars);
           bounded_wait(&bars->full_w[stage], phase, bars);
-          if (bars->abort) break;
           ptx::tc_fence_after_sync();
           const uint32_t xa = ptx::smem_u32(x_tile(stage)), wa = ptx::smem_u32(w_tile(stage));
 #pragma unroll
