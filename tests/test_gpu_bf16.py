@@ -60,6 +60,17 @@ def test_bf16_ragged_tails(rank, bits, group, signed):
     check_layer(cfg, arrays, gh.run_layer(cfg, arrays, do_pack=True, grad_scale=0.25), grad_scale=0.25)
 
 
+@pytest.mark.parametrize("tokens", [1, 8, 100, 129])
+@pytest.mark.parametrize("d_out", [64, 392])
+def test_bf16_few_tokens_and_narrow_output(tokens, d_out):
+    # fewer rows than one tile (the TMA boxes of X, dY, Y and dX are then taller than the tensors) and fewer
+    # output columns than one tile
+    cfg = synth.LayerConfig(f"bf16_tok{tokens}_o{d_out}", tokens=tokens, d_in=320, d_out=d_out, rank=16, alpha=32.0,
+                            bits=4, group_size=64)
+    arrays = synth.make_layer_inputs(cfg, seed=3)
+    check_layer(cfg, arrays, gh.run_layer(cfg, arrays, do_pack=True))
+
+
 def test_bf16_many_tiles_more_than_sms():
     # 3 x 56 = 168 forward tiles > 148 SMs: exercises the persistent loop, both accumulator stages and phase flips
     cfg = synth.LayerConfig("bf16_persistent", tokens=384, d_in=320, d_out=14336, rank=16, alpha=32.0, bits=4,
