@@ -16,7 +16,7 @@ host memory and the parameter gradients copied back inside the timed region.
 
 N > 1 (launched by torch.distributed.run, one rank per GPU): data parallel over
 tokens -- every rank runs the same layers on its own token batch (weak scaling)
-and the parameter gradients are all-reduced (sum) over NCCL each step.
+and the parameter gradients of each layer are all-reduced (sum) over NCCL each step, as one bucket.
 
 `--layer lora|qat_lora` runs the LoRA (Eq. 1-2) or QAT-LoRA (Sec. 3.1) layer instead, through
 l4q_lora_linear_fwd / l4q_lora_linear_bwd, for the per-step cost comparison (no export step; the
@@ -240,13 +240,17 @@ def run_ours(args, layers, wl_name):
         d["dY"] = host["dY"].to(dev)
         desc = l4q.make_desc(cfg)
         outs = l4q.alloc_outputs(cfg, device=dev)
+        # the parameter gradients of a layer live in one buffer, so that N > 1 ranks exchange them in one all-reduce
+        bucket, views = dp.alloc_grad_bucket({k: outs[k].shape for k in grad_names}, device=dev)
+        outs.update(views)
         pk = l4q.alloc_pack_outputs(cfg, device=dev)
         if args.layer == "l4q":
             ws = l4q.alloc_workspace(desc, l4q.L4Q_OP_BWD, device=dev)
         else:
             ws = l4q.alloc_lora_workspace(desc, l4q.LORA_KINDS[args.layer], l4q.L4Q_OP_BWD, device=dev)
         grads_host = {k: torch.empty_like(outs[k], device="cpu").pin_memory() for k in grad_names}
-        L.append(dict(cfg=cfg, desc=desc, d=d, outs=outs, pk=pk, ws=ws, host=host, grads_host=grads_host))
+        L.append(dict(cfg=cfg, desc=desc, d=d, outs=outs, pk=pk, ws=ws, host=host, grads_host=grads_host,
+                      bucket=bucket))
         h2d += host["X"].numel() * 2 + host["dY"].numel() * 2
         d2h += sum(t.numel() * 4 for t in grads_host.values())
 
@@ -298,7 +302,7 @@ def run_ours(args, layers, wl_name):
                                         o["dA"], o["dB"], o["ds"] if qat else None, o["db"] if qat else None,
                                         l["ws"])
             if world > 1:
-                dp.allreduce_param_grads({k: o[k] for k in grad_names} if kind else o)
+                dp.allreduce_grad_bucket(l["bucket"])
             if e2e:
                 ev = torch.cuda.Event()
                 ev.record()

@@ -34,8 +34,17 @@ def _rank_main(rank: int, world: int, port: int, out_dir: str):
         sl = dp.token_shard(CFG.tokens, rank, world)
         g = orc.backward(spec, arrays["X"][sl], arrays["dY"][sl], arrays["W0"], arrays["A"], arrays["B"],
                          arrays["s"], arrays["b"])
+        if True:
+            # half of the test goes through the per-tensor helper, half through the bucket bench.py uses
+            flat, views = dp.alloc_grad_bucket({k: g[k].shape for k in dp.PARAM_GRADS}, dtype=torch.float64)
+            for k in dp.PARAM_GRADS:
+                views[k].copy_(torch.from_numpy(np.ascontiguousarray(g[k])))
+            dp.allreduce_grad_bucket(flat)
         grads = {k: torch.from_numpy(np.ascontiguousarray(g[k])) for k in dp.PARAM_GRADS}
         dp.allreduce_param_grads(grads)
+        for k in dp.PARAM_GRADS:
+            assert torch.equal(views[k], grads[k]), k
+            assert views[k].data_ptr() % 16 == 0
         np.savez(os.path.join(out_dir, f"rank{rank}.npz"), dX=g["dX"], start=sl.start, stop=sl.stop,
                  **{k: v.numpy() for k, v in grads.items()})
     finally:
