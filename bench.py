@@ -293,7 +293,7 @@ def run_ours(args, layers, wl_name):
                 l4q.l4q_linear_bwd(l["desc"], d["X"], d["dY"], d["W0"], d["A"], d["B"], d["s"], d["b"],
                                    o["dX"], o["dA"], o["dB"], o["ds"], o["db"], l["ws"])
                 l4q.l4q_pack_int(l["desc"], d["W0"], d["A"], d["B"], d["s"], d["b"], pk["codes"], pk["s16"],
-                                 pk["b16"])
+                                 pk["b16"], l["ws"])
             else:
                 qat = args.layer == "qat_lora"
                 sq, bq = (d["s"], d["b"]) if qat else (None, None)

@@ -119,7 +119,9 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
  *   s_fp16 = fp16(s), b_fp16 = fp16(b + s*Q_N) as IEEE binary16 bit patterns
  *   [d_out, d_in/group_size], so that W_q ~= u * s_fp16 + b_fp16.
  * Codes are taken with the fp32 s and b (they equal the forward's codes).
- * bits must be 3 or 4 and d_in*bits a multiple of 32.  Needs no workspace.
+ * bits must be 3 or 4 and d_in*bits a multiple of 32.  The workspace is optional: NULL works; given
+ * l4q_workspace_bytes(desc, L4Q_OP_PACK) bytes of 256-byte aligned device scratch the bf16 path is faster
+ * (the split LoRA operands of the merge are then built once per call instead of once per tile).
  */
 l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, const float* B,
                         const float* s, const float* b,

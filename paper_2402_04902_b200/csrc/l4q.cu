@@ -101,6 +101,11 @@ size_t wq_scratch_bytes(const l4q_desc* d) {
   return align_up((size_t)d->d_out * (size_t)d->d_in * esz, 256);
 }
 
+// Scratch of the split LoRA operands of the tensor-core weight-tile kernel (bf16 mode).
+size_t operand_image_bytes(const l4q_desc* d, const Params& p) {
+  return d->io_dtype == L4Q_BF16 && wtile_tc_supported(p, WT2_DEQUANT) ? align_up(wtile_image_bytes(p), 256) : 0;
+}
+
 size_t factor_scratch_bytes(const l4q_desc* d) {
   return align_up(factor_elems((int)d->d_out, (int)d->d_in) * sizeof(__half), 256);
 }
@@ -111,12 +116,13 @@ inline l4q_status launch_status() { return cudaGetLastError() == cudaSuccess ? L
 // `fac` (optional, bf16 mode only) also receives the fp16 STE factors the weight-gradient kernel reads.
 template <bool IO_BF16>
 l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const float* B, const float* s,
-                          const float* b, void* wq, __half* fac, cudaStream_t st) {
+                          const float* b, void* wq, __half* fac, cudaStream_t st, void* op_img = nullptr) {
   if constexpr (IO_BF16) {
     const int mode = fac ? WT2_DEQUANT_F : WT2_DEQUANT;
     if (wtile_tc_supported(p, mode)) {               // tensor-core merge, TMA in and out
-      KernelScope ks(L4Q_KERNEL_DEQUANT, st);
-      return launch_wtile_tc(mode, p, W0, A, B, s, b, wq, fac, nullptr, nullptr, st);
+      KernelScope ks(L4Q_KERNEL_DEQUANT, st);   // covers the operand split too, which is one more launch
+      if (op_img) g_launches.fetch_add(1, std::memory_order_relaxed);
+      return launch_wtile_tc(mode, p, W0, A, B, s, b, wq, fac, nullptr, nullptr, st, op_img);
     }
   }
   const size_t smem = weight_tile_smem_bytes(p.rank);
@@ -132,11 +138,13 @@ l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const
 
 template <bool IO_BF16>
 l4q_status launch_pack(const Params& p, const void* W0, const float* A, const float* B, const float* s,
-                       const float* b, uint32_t* codes, __half* s16, __half* b16, cudaStream_t st) {
+                       const float* b, uint32_t* codes, __half* s16, __half* b16, cudaStream_t st,
+                       void* op_img = nullptr) {
   if constexpr (IO_BF16) {
     if (wtile_tc_supported(p, WT2_PACK)) {
-      KernelScope ks(L4Q_KERNEL_PACK, st);
-      return launch_wtile_tc(WT2_PACK, p, W0, A, B, s, b, codes, nullptr, s16, b16, st);
+      KernelScope ks(L4Q_KERNEL_PACK, st);      // covers the operand split too, which is one more launch
+      if (op_img) g_launches.fetch_add(1, std::memory_order_relaxed);
+      return launch_wtile_tc(WT2_PACK, p, W0, A, B, s, b, codes, nullptr, s16, b16, st, op_img);
     }
   }
   const size_t smem = weight_tile_smem_bytes(p.rank);
@@ -200,10 +208,12 @@ size_t l4q_workspace_bytes(const l4q_desc* desc, int op) {
   if (make_params(desc, &p) != L4Q_OK) return 0;
   switch (op) {
     case L4Q_OP_FWD:
-      return wq_scratch_bytes(desc) + 256;
+      return wq_scratch_bytes(desc) + operand_image_bytes(desc, p) + 256;
     case L4Q_OP_BWD:   // W_q for the input gradient, and in bf16 mode the fp16 STE factors for the weight gradient
-      return wq_scratch_bytes(desc) + (desc->io_dtype == L4Q_BF16 ? factor_scratch_bytes(desc) : 0) + 256;
-    case L4Q_OP_PACK:
+      return wq_scratch_bytes(desc) + (desc->io_dtype == L4Q_BF16 ? factor_scratch_bytes(desc) : 0) +
+             operand_image_bytes(desc, p) + 256;
+    case L4Q_OP_PACK:   // optional (see l4q_pack_int)
+      return operand_image_bytes(desc, p);
     default:
       return 0;
   }
@@ -234,7 +244,9 @@ l4q_status l4q_linear_fwd(const l4q_desc* desc, const void* X, const void* W0, c
     k_val_gemm<<<grid, V_THREADS, 0, stream>>>(g, reinterpret_cast<float*>(Y));
     return launch_status();
   }
-  st = launch_dequant<true>(p, W0, A, B, s, b, wq, nullptr, stream);
+  // the split operands of the merge follow W_q in the workspace
+  void* op_img = operand_image_bytes(desc, p) ? static_cast<unsigned char*>(workspace) + wq_scratch_bytes(desc) : nullptr;
+  st = launch_dequant<true>(p, W0, A, B, s, b, wq, nullptr, stream, op_img);
   if (st != L4Q_OK) return st;
   KernelScope ks(L4Q_KERNEL_GEMM_FWD, stream);
   return gemm_forward_bf16(p, X, wq, Y, stream);
@@ -273,7 +285,11 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
                     : nullptr;
   if (dX || fac) {
     st = f32 ? launch_dequant<false>(p, W0, A, B, s, b, wq, nullptr, stream)
-             : launch_dequant<true>(p, W0, A, B, s, b, wq, fac, stream);
+             : launch_dequant<true>(p, W0, A, B, s, b, wq, fac, stream,
+                                    operand_image_bytes(desc, p)
+                                        ? static_cast<unsigned char*>(workspace) + wq_scratch_bytes(desc) +
+                                              factor_scratch_bytes(desc)
+                                        : nullptr);
     if (st != L4Q_OK) return st;
   }
   if (f32) {
@@ -417,7 +433,6 @@ l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, co
 l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, const float* B, const float* s,
                         const float* b, uint32_t* codes, uint16_t* s_fp16, uint16_t* b_fp16, void* workspace,
                         size_t workspace_bytes, void* cuda_stream) {
-  (void)workspace; (void)workspace_bytes;
   Params p;
   l4q_status st = make_params(desc, &p);
   if (st != L4Q_OK) return st;
@@ -428,7 +443,11 @@ l4q_status l4q_pack_int(const l4q_desc* desc, const void* W0, const float* A, co
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   __half* s16 = reinterpret_cast<__half*>(s_fp16);
   __half* b16 = reinterpret_cast<__half*>(b_fp16);
-  return desc->io_dtype == L4Q_BF16 ? launch_pack<true>(p, W0, A, B, s, b, codes, s16, b16, stream)
+  // the workspace is optional: with it the split operands of the merge are built once instead of tile by tile
+  const size_t img = operand_image_bytes(desc, p);
+  void* op_img = (workspace && img && workspace_bytes >= img && !(reinterpret_cast<uintptr_t>(workspace) & 255u))
+                     ? workspace : nullptr;
+  return desc->io_dtype == L4Q_BF16 ? launch_pack<true>(p, W0, A, B, s, b, codes, s16, b16, stream, op_img)
                                     : launch_pack<false>(p, W0, A, B, s, b, codes, s16, b16, stream);
 }
 

@@ -85,6 +85,13 @@ __device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uin
                ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes)
                : "memory");
 }
+// Untiled bulk load global -> shared, completing `bytes` on an mbarrier of this CTA: both addresses 16-byte
+// aligned, size a multiple of 16 bytes.
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // All of this thread's committed bulk stores have finished READING shared memory.
 __device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }

@@ -50,6 +50,7 @@ struct WtileArgs {
   const float *A, *B, *s, *b;
   __half *s16, *b16;       // WT2_PACK
   __half* F;               // WT2_DEQUANT_F: the factor array (factor_index layout)
+  const uint8_t* op_img;   // optional: the split MMA operands of every panel, ready made (see k_split_operands)
   int tiles_m, tiles_n;
   int n_stages;            // W0 stages in shared memory (2..4)
   int n_out;               // staging buffers for the second output (F or codes): 0, 1 or 2
@@ -132,39 +133,81 @@ __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
 // consecutive bytes.
 struct OperandItem { float av[4]; float4 bv; };
 
-__device__ __forceinline__ void operand_item_load(const WtileArgs& a, int m0, int n0, int idx, OperandItem& it) {
+__device__ __forceinline__ void operand_a_load(const WtileArgs& a, int n0, int idx, float (&av)[4]) {
   const Params& p = a.p;
   const int row = idx & 127, kc = idx >> 7, col = n0 + row;
 #pragma unroll
-  for (int e = 0; e < 4; ++e) it.av[e] = (col < p.d_in) ? __ldg(a.A + (size_t)(4 * kc + e) * p.d_in + col) : 0.f;
-  const int rq = p.rank >> 2;                        // 16-byte pieces per row of B
-  const int brow = idx / rq;
-  it.bv = (m0 + brow < p.d_out) ? __ldg(reinterpret_cast<const float4*>(a.B + (size_t)m0 * p.rank) + idx)
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int e = 0; e < 4; ++e) av[e] = (col < p.d_in) ? __ldg(a.A + (size_t)(4 * kc + e) * p.d_in + col) : 0.f;
 }
 
-__device__ __forceinline__ void operand_item_store(const WtileArgs& a, int idx, const OperandItem& it, uint8_t* acat,
-                                                   uint8_t* bcat) {
+__device__ __forceinline__ void operand_b_load(const WtileArgs& a, int m0, int idx, float4& bv) {
+  const Params& p = a.p;
+  const int rq = p.rank >> 2;                        // 16-byte pieces per row of B
+  const int brow = idx / rq;
+  bv = (m0 + brow < p.d_out) ? __ldg(reinterpret_cast<const float4*>(a.B + (size_t)m0 * p.rank) + idx)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+__device__ __forceinline__ void operand_a_store(const WtileArgs& a, int idx, const float (&av)[4], uint8_t* acat) {
   const int row = idx & 127, kc = idx >> 7;
-  const int rq = a.p.rank >> 2;
-  const int brow = idx / rq, bkc = idx - brow * rq;
-  const float bvv[4] = {it.bv.x, it.bv.y, it.bv.z, it.bv.w};
-  float ah[4], al[4], bh[4], bl[4];
+  float ah[4], al[4];
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    split_tf32(it.av[e], ah[e], al[e]);
-    split_tf32(bvv[e], bh[e], bl[e]);
-  }
+  for (int e = 0; e < 4; ++e) split_tf32(av[e], ah[e], al[e]);
   const int ch = kc, cl = (a.p.rank >> 2) + kc;      // 16-byte chunk index of the head / tail within the row
   const uint32_t off_h = (uint32_t)(ch >> 3) * WT2_ATOM_BYTES + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
   const uint32_t off_l = (uint32_t)(cl >> 3) * WT2_ATOM_BYTES + row * 128 + (((cl & 7) ^ (row & 7)) << 4);
   *reinterpret_cast<float4*>(acat + off_h) = make_float4(ah[0], ah[1], ah[2], ah[3]);
   *reinterpret_cast<float4*>(acat + off_l) = make_float4(al[0], al[1], al[2], al[3]);
+}
+
+__device__ __forceinline__ void operand_b_store(const WtileArgs& a, int idx, const float4& bv, uint8_t* bcat) {
+  const int rq = a.p.rank >> 2;
+  const int brow = idx / rq, bkc = idx - brow * rq;
+  const float bvv[4] = {bv.x, bv.y, bv.z, bv.w};
+  float bh[4], bl[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) split_tf32(bvv[e], bh[e], bl[e]);
   const int bch = bkc, bcl = rq + bkc;
   const uint32_t boff_h = (uint32_t)(bch >> 3) * WT2_ATOM_BYTES + brow * 128 + (((bch & 7) ^ (brow & 7)) << 4);
   const uint32_t boff_l = (uint32_t)(bcl >> 3) * WT2_ATOM_BYTES + brow * 128 + (((bcl & 7) ^ (brow & 7)) << 4);
   *reinterpret_cast<float4*>(bcat + boff_h) = make_float4(bh[0], bh[1], bh[2], bh[3]);
   *reinterpret_cast<float4*>(bcat + boff_l) = make_float4(bl[0], bl[1], bl[2], bl[3]);
+}
+
+__device__ __forceinline__ void operand_item_load(const WtileArgs& a, int m0, int n0, int idx, OperandItem& it) {
+  operand_a_load(a, n0, idx, it.av);
+  operand_b_load(a, m0, idx, it.bv);
+}
+
+__device__ __forceinline__ void operand_item_store(const WtileArgs& a, int idx, const OperandItem& it, uint8_t* acat,
+                                                   uint8_t* bcat) {
+  operand_a_store(a, idx, it.av, acat);
+  operand_b_store(a, idx, it.bv, bcat);
+}
+
+// The operand images of all panels, written once per launch of the weight-tile kernel so that its epilogue warps
+// need not build them tile by tile: image tn (tn < tiles_n) is the acat block of column panel tn, image
+// tiles_n + tm the bcat block of row panel tm, each exactly as it stands in shared memory (op_half bytes), so
+// that one bulk copy brings it in.  One block per panel.
+__global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8_t* __restrict__ img) {
+  const uint32_t op_half = (uint32_t)a.atoms * WT2_ATOM_BYTES;
+  const int panel = blockIdx.x;
+  uint8_t* dst = img + (size_t)panel * op_half;
+  const int n_items = 32 * a.p.rank;
+  // chunks of an atom row beyond 2 rank values are never read by the MMAs; the image leaves them as they are
+  if (panel < a.tiles_n) {
+    for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
+      float av[4];
+      operand_a_load(a, panel * WT2_COLS, idx, av);
+      operand_a_store(a, idx, av, dst);
+    }
+  } else {
+    for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
+      float4 bv;
+      operand_b_load(a, (panel - a.tiles_n) * WT2_ROWS, idx, bv);
+      operand_b_store(a, idx, bv, dst);
+    }
+  }
 }
 
 // Adding and subtracting 1.5 * 2^23 rounds |x| < 2^22 to the nearest integer, ties to even, exactly like
@@ -197,7 +240,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       ptx::mbar_init(&bars->written[i], WT2_GROUP_THREADS);
     }
     for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->out_empty[i], 1);
-    for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->prep_full[i], WT2_GROUP_THREADS);
+    for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->prep_full[i], a.op_img ? 1 : WT2_GROUP_THREADS);
     for (int i = 0; i < WT2_ACC; ++i) {
       ptx::mbar_init(&bars->tmem_full[i], 1);
       ptx::mbar_init(&bars->tmem_empty[i], WT2_GROUP_THREADS);
@@ -300,6 +343,25 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       ptx::bulk_wait_group0();
     }
     __syncwarp();
+  } else if (warp == 3) {
+    // ------------------------------ MMA operands from the ready-made images ----
+    if (lane == 0 && a.op_img) {
+      const int L = a.n_opbuf;
+      int j = 0;
+      for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next(), ++j) {
+        const int buf = j & (L - 1);
+        if (j >= L) {      // the MMAs of tile j - L, the last readers of this buffer, have completed
+          bounded_wait(&bars->tmem_full[(j - L) & 3], (uint32_t)(((j - L) >> 2) & 1), bars);
+          if (bars->abort) break;
+        }
+        uint8_t* acat = op_base + (size_t)buf * 2 * op_half;
+        ptx::mbar_arrive_expect_tx(&bars->prep_full[buf], 2 * op_half);
+        ptx::bulk_load(acat, a.op_img + (size_t)cur.tn * op_half, op_half, &bars->prep_full[buf]);
+        ptx::bulk_load(acat + op_half, a.op_img + (size_t)(a.tiles_n + cur.tm) * op_half, op_half,
+                       &bars->prep_full[buf]);
+      }
+    }
+    __syncwarp();
   } else if (warp >= WT2_FIRST_EPI_WARP) {
     // ------------------------------ epilogue ----------------------------------
     // Two groups of eight warps; group grp owns the CTA's tiles i = grp, grp + 2, ... (accumulator stage i % 4,
@@ -328,6 +390,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
     };
     auto prep = [&](int j, int m0_, int n0_) {
+      if (a.op_img) return;                                     // warp 3 brings the operands in
       prep_buffer_wait(j);
       uint8_t* acat = op_base + (size_t)(j & (L - 1)) * 2 * op_half;
       for (int idx = tg; idx < n_items; idx += WT2_GROUP_THREADS) {
@@ -368,12 +431,12 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     int sb_buf = 0;
     const int qn_bits = kRoundMagicBits + (int)p.qn;
 
+    int stage = grp;                                            // W0 stage of tile i and its phase, kept without divisions
+    uint32_t phase = 0;                                         // (n_stages >= 2 = WT2_GROUPS)
     for (int i = grp; cur.valid(); cur.next(), i += WT2_GROUPS) {
       const int m0 = cur.m0(), n0 = cur.n0();
       const int o = m0 + row;
       const bool row_ok = o < p.d_out;
-      const int stage = i % a.n_stages;
-      const uint32_t phase = (uint32_t)((i / a.n_stages) & 1);
       const int acc = i & 3;
       const int g_first = group_of(a, n0);
       int m1 = 0, n1 = 0;
@@ -388,8 +451,9 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       bounded_wait(&bars->full[stage], phase, bars);
       int ob = 0;
       if constexpr (HAS_OUT1) {
-        ob = i % a.n_out;
-        if (i >= a.n_out) bounded_wait(&bars->out_empty[ob], (uint32_t)((i / a.n_out - 1) & 1), bars);
+        const int uses = a.n_out == 2 ? (i >> 1) : i;           // earlier tiles that went through this buffer
+        ob = a.n_out == 2 ? (i & 1) : 0;
+        if (uses >= 1) bounded_wait(&bars->out_empty[ob], (uint32_t)((uses - 1) & 1), bars);
       }
       uint8_t* tile_rows = stage_base + (size_t)stage * WT2_STAGE_BYTES + row * 128;
       [[maybe_unused]] uint8_t* out1 = out_base + (size_t)ob * a.out_bytes;
@@ -488,6 +552,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       ptx::mbar_arrive(&bars->written[stage]);
       sb_buf ^= 1;
       if (has_next) stage_sb(m1, n1, sb_buf);          // the other buffer: its readers passed this tile's barrier
+      stage += WT2_GROUPS;
+      if (stage >= a.n_stages) { stage -= a.n_stages; phase ^= 1; }
     }
   }
 
@@ -563,9 +629,18 @@ inline bool wtile_tc_supported(const Params& p, int mode) {
 }
 
 // mode WT2_DEQUANT: out0 = W_q.  WT2_DEQUANT_F: out0 = W_q, out1 = STE factors.  WT2_PACK: out0 = codes.
+// Bytes of the operand images of a problem (see k_split_operands).
+inline size_t wtile_image_bytes(const Params& p) {
+  const size_t atoms = (2 * (size_t)p.rank + 31) / 32;
+  return ((size_t)ceil_div(p.d_out, WT2_ROWS) + (size_t)ceil_div(p.d_in, WT2_COLS)) * atoms * WT2_ATOM_BYTES;
+}
+
+// `op_img` (optional, wtile_image_bytes(p) bytes of device scratch, 16-byte aligned): with it the MMA operands are
+// split once by a launch of k_split_operands and reach the tiles by bulk copies; without it the epilogue warps
+// build them tile by tile.
 inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, const float* A, const float* B,
                                   const float* s, const float* b, void* out0, void* out1, __half* s16, __half* b16,
-                                  cudaStream_t st) {
+                                  cudaStream_t st, void* op_img = nullptr) {
   WtileArgs a{};
   a.p = p; a.A = A; a.B = B; a.s = s; a.b = b; a.s16 = s16; a.b16 = b16;
   a.tiles_m = ceil_div(p.d_out, WT2_ROWS);
@@ -583,6 +658,11 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   }
   const size_t smem = wtile_smem_bytes(a);
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
+  if (op_img) {
+    k_split_operands<<<a.tiles_n + a.tiles_m, 256, 0, st>>>(a, static_cast<uint8_t*>(op_img));
+    if (cudaGetLastError() != cudaSuccess) return L4Q_ERR_CUDA;
+    a.op_img = static_cast<const uint8_t*>(op_img);
+  }
   auto launch = [&](auto kern) -> l4q_status {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return L4Q_ERR_CUDA;

@@ -61,8 +61,10 @@ def run_layer(cfg, arrays, do_fwd=True, do_bwd=True, do_pack=False, grad_scale=1
         guards["codes"] = Guarded((cfg.d_out, cfg.d_in * cfg.bits // 32), torch.int32)
         guards["s16"] = Guarded((cfg.d_out, G), torch.float16)
         guards["b16"] = Guarded((cfg.d_out, G), torch.float16)
+        # with the optional scratch (the split operands are then built once); the calls elsewhere in the
+        # tests pass none and cover the other path
         l4q.l4q_pack_int(desc, dev["W0"], dev["A"], dev["B"], dev["s"], dev["b"], guards["codes"].view,
-                         guards["s16"].view, guards["b16"].view)
+                         guards["s16"].view, guards["b16"].view, l4q.alloc_workspace(desc, l4q.L4Q_OP_PACK))
     l4q.l4q_check()
     for k, g in guards.items():
         assert g.intact(), f"out-of-bounds write around {k}"

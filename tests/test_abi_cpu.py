@@ -45,7 +45,9 @@ def test_status_strings(lib):
 def test_workspace_query_and_rejections(lib):
     d = l4q.make_desc(CONFIG2)
     assert l4q.l4q_workspace_bytes(d, l4q.L4Q_OP_FWD) >= CONFIG2.d_in * CONFIG2.d_out * 2
-    assert l4q.l4q_workspace_bytes(d, l4q.L4Q_OP_PACK) == 0
+    # optional scratch of the export: one split-operand block of 16 KiB per 128-wide panel of A and of B at rank 16
+    assert l4q.l4q_workspace_bytes(d, l4q.L4Q_OP_PACK) == (CONFIG2.d_in // 128 + CONFIG2.d_out // 128) * 16384
+    assert l4q.l4q_workspace_bytes(l4q.make_desc(CONFIG2.with_(io_dtype="f32")), l4q.L4Q_OP_PACK) == 0
     bad = l4q.make_desc(CONFIG2.with_(group_size=100))        # d_in % group_size != 0
     assert l4q.l4q_workspace_bytes(bad, l4q.L4Q_OP_FWD) == 0
 
