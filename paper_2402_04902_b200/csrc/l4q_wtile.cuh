@@ -59,6 +59,8 @@ struct WtileArgs {
   int ngt;                 // upper bound of the quantization groups a 128-column tile intersects
   int n_opbuf;             // MMA operand buffers ([A slice | B slice] each): 1 or 2
   int group_shift;         // log2(group size) if it is a power of two, else -1
+  int sb_box;              // groups per row of the s / b boxes that TMA brings in with the W0 tile; 0: the epilogue
+                           // warps stage s and b themselves
 };
 
 // column / group size without a division in the common power-of-two case
@@ -81,9 +83,13 @@ struct __align__(8) WtileBarriers {
 // in total); a thread reads and writes its own entry only.
 __host__ __device__ inline size_t wtile_sb_bytes(int ngt) { return (size_t)WT2_EPI_THREADS * 2 * ngt * sizeof(float); }
 
+// With sb_box: per W0 stage one box [128 rows][sb_box] of s and one of b.
+__host__ __device__ inline size_t wtile_sb_region_bytes(const WtileArgs& a) {
+  return a.sb_box ? (size_t)a.n_stages * 2 * WT2_ROWS * a.sb_box * sizeof(float) : wtile_sb_bytes(a.ngt);
+}
 inline size_t wtile_smem_bytes(const WtileArgs& a) {
   return 1024 + (size_t)a.n_stages * WT2_STAGE_BYTES + (size_t)a.n_out * a.out_bytes +
-         2 * (size_t)a.n_opbuf * a.atoms * WT2_ATOM_BYTES + wtile_sb_bytes(a.ngt) + sizeof(WtileBarriers);
+         2 * (size_t)a.n_opbuf * a.atoms * WT2_ATOM_BYTES + wtile_sb_region_bytes(a) + sizeof(WtileBarriers);
 }
 
 // The tiles of one CTA: tile t of the column-panel-major sequence (row tiles of one column panel are
@@ -220,6 +226,8 @@ __global__ void __launch_bounds__(WT2_THREADS, 1)
 k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out, d_in] bf16, box 64 x 128, swizzled
            const __grid_constant__ CUtensorMap tmap_out0,   // store: W_q (same geometry) | codes (uint32 words)
            const __grid_constant__ CUtensorMap tmap_out1,   // store: STE factors (same geometry as W0) | unused
+           const __grid_constant__ CUtensorMap tmap_s,      // load:  s [d_out, ngroups] fp32, box sb_box x 128 (if sb_box)
+           const __grid_constant__ CUtensorMap tmap_b,      // load:  b, likewise
            const WtileArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -228,7 +236,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
   uint8_t* op_base = out_base + (size_t)a.n_out * a.out_bytes;          // operand buffer b: [acat | bcat]
   const uint32_t op_half = (uint32_t)a.atoms * WT2_ATOM_BYTES;           // bytes of one acat or bcat
   float* sb_base = reinterpret_cast<float*>(op_base + (size_t)a.n_opbuf * 2 * op_half);
-  WtileBarriers* bars = reinterpret_cast<WtileBarriers*>(reinterpret_cast<uint8_t*>(sb_base) + wtile_sb_bytes(a.ngt));
+  WtileBarriers* bars = reinterpret_cast<WtileBarriers*>(reinterpret_cast<uint8_t*>(sb_base) + wtile_sb_region_bytes(a));
   const Params& p = a.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr bool HAS_OUT1 = (MODE != WT2_DEQUANT);
@@ -250,6 +258,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     ptx::prefetch_tmap(&tmap_w0);
     ptx::prefetch_tmap(&tmap_out0);
     if (MODE == WT2_DEQUANT_F) ptx::prefetch_tmap(&tmap_out1);
+    if (a.sb_box) { ptx::prefetch_tmap(&tmap_s); ptx::prefetch_tmap(&tmap_b); }
   }
   if (warp == 1) {
     ptx::tmem_alloc(&bars->tmem_base, WT2_ACC * WT2_COLS);
@@ -269,9 +278,17 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
         bounded_wait(&bars->empty[stage], phase ^ 1, bars);
         if (bars->abort) break;
         uint8_t* dst = stage_base + (size_t)stage * WT2_STAGE_BYTES;
-        ptx::mbar_arrive_expect_tx(&bars->full[stage], WT2_STAGE_BYTES);
+        const uint32_t sb_box_bytes = (uint32_t)(WT2_ROWS * a.sb_box * sizeof(float));
+        ptx::mbar_arrive_expect_tx(&bars->full[stage], WT2_STAGE_BYTES + 2 * sb_box_bytes);
         ptx::tma_load_2d(dst, &tmap_w0, &bars->full[stage], n0, m0);
         ptx::tma_load_2d(dst + WT2_STAGE_BYTES / 2, &tmap_w0, &bars->full[stage], n0 + 64, m0);
+        if (a.sb_box) {
+          // s and b of the tile's rows, from the group column rounded down to a 16-byte boundary
+          uint8_t* sdst = reinterpret_cast<uint8_t*>(sb_base) + (size_t)stage * 2 * sb_box_bytes;
+          const int x0 = group_of(a, n0) & ~3;
+          ptx::tma_load_2d(sdst, &tmap_s, &bars->full[stage], x0, m0);
+          ptx::tma_load_2d(sdst + sb_box_bytes, &tmap_b, &bars->full[stage], x0, m0);
+        }
         if (++stage == a.n_stages) { stage = 0; phase ^= 1; }
       }
     }
@@ -407,7 +424,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     //      tile; the group meets at a named barrier when it starts that tile.  (Each row's values sit in a line
     //      of their own, so every copy instruction touches 32 lines: the fewer of them the better.) ----
     auto stage_sb = [&](int m0_, int n0_, int buf) {
-      if (chalf != 0) return;
+      if (chalf != 0 || a.sb_box) return;
       float* dst = grp_sb + ((size_t)buf * WT2_ROWS + row) * sbw;
       const int o_ = m0_ + row;
       const int gf = group_of(a, n0_);
@@ -441,9 +458,19 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       const int g_first = group_of(a, n0);
       int m1 = 0, n1 = 0;
       const bool has_next = cur.peek(1, m1, n1);
-      ptx::cp_async_wait_all();                                 // this thread's copies of the tile's s, b have landed
-      ptx::named_bar_sync(1 + grp, WT2_GROUP_THREADS);          // ... and so have the group's
-      const float* my_sb = grp_sb + ((size_t)sb_buf * WT2_ROWS + row) * sbw;
+      const float *my_s, *my_b;                                 // s and b of this row, from group sb_first on
+      int sb_first;
+      if (a.sb_box) {                                           // they arrive with the W0 tile (full[stage] below)
+        my_s = sb_base + ((size_t)stage * 2 * WT2_ROWS + row) * a.sb_box;
+        my_b = my_s + WT2_ROWS * a.sb_box;
+        sb_first = g_first & ~3;
+      } else {
+        ptx::cp_async_wait_all();                               // this thread's copies of the tile's s, b have landed
+        ptx::named_bar_sync(1 + grp, WT2_GROUP_THREADS);        // ... and so have the group's
+        my_s = grp_sb + ((size_t)sb_buf * WT2_ROWS + row) * sbw;
+        my_b = my_s + a.ngt;
+        sb_first = g_first;
+      }
       bounded_wait(&bars->tmem_full[acc], (uint32_t)((i >> 2) & 1), bars);
       ptx::tc_fence_after_sync();
       // the merge of this tile is complete: the operands of the group's next tile can take its buffer
@@ -482,8 +509,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
             const bool group_start = (col - g * p.group) == 0;
             if (g != cur_g) {                                   // one reciprocal per group
               cur_g = g;
-              s_ = ok ? my_sb[g - g_first] : 1.f;
-              b_ = ok ? my_sb[a.ngt + g - g_first] : 0.f;
+              s_ = ok ? my_s[g - sb_first] : 1.f;
+              b_ = ok ? my_b[g - sb_first] : 0.f;
               rs = 1.0f / s_;
             }
             const uint32_t chunk = (uint32_t)((piece >> 3) * (WT2_STAGE_BYTES / 2) + (((piece & 7) ^ (row & 7)) << 4));
@@ -590,10 +617,15 @@ inline bool make_tmap_words(CUtensorMap* m, const void* base, uint64_t rows, uin
 // Shared-memory plan.  A tile being worked on holds one W0 stage and, when there is a second output, one
 // staging buffer for it: two of each keep both epilogue groups busy, further stages let the loads run ahead.
 // Candidates in order of preference (a single operand buffer makes every merge wait for the previous one).
-inline bool wtile_plan(WtileArgs& a, int mode) {
+// `sb_by_tma`: s and b may come in by TMA (the caller has checked their alignment); the shape must allow it too.
+inline bool wtile_plan(WtileArgs& a, int mode, bool sb_by_tma = true) {
   const Params& p = a.p;
   a.atoms = (2 * p.rank + 31) / 32;
   a.ngt = std::min(p.ngroups, (WT2_COLS - 1) / p.group + 2);
+  // a box starts at a group column that is a multiple of 4 (16 bytes) at or below the tile's first group, so it
+  // is up to 3 groups wider than the tile; the row pitch of s and b must be a multiple of 16 bytes
+  const int box = (a.ngt + 3 + 3) / 4 * 4;
+  a.sb_box = (sb_by_tma && p.ngroups % 4 == 0 && p.ngroups >= box && box <= 256) ? box : 0;
   a.group_shift = -1;
   for (int sh = 3; sh < 31; ++sh)
     if ((1 << sh) == p.group) a.group_shift = sh;
@@ -645,8 +677,9 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   a.p = p; a.A = A; a.B = B; a.s = s; a.b = b; a.s16 = s16; a.b16 = b16;
   a.tiles_m = ceil_div(p.d_out, WT2_ROWS);
   a.tiles_n = ceil_div(p.d_in, WT2_COLS);
-  if (!wtile_plan(a, mode)) return L4Q_ERR_UNSUPPORTED;
-  CUtensorMap t_w0, t_o0, t_o1;
+  const bool sb_aligned = ((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(b)) & 15u) == 0;
+  if (!wtile_plan(a, mode, sb_aligned)) return L4Q_ERR_UNSUPPORTED;
+  CUtensorMap t_w0, t_o0, t_o1, t_s, t_b;
   if (!make_tmap_bf16(&t_w0, W0, p.d_out, p.d_in, WT2_ROWS)) return L4Q_ERR_CUDA;
   t_o1 = t_w0;
   if (mode == WT2_PACK) {
@@ -655,6 +688,11 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   } else {
     if (!make_tmap_bf16(&t_o0, out0, p.d_out, p.d_in, WT2_ROWS)) return L4Q_ERR_CUDA;
     a.F = reinterpret_cast<__half*>(out1);
+  }
+  t_s = t_w0; t_b = t_w0;                          // placeholders when unused
+  if (a.sb_box) {                                   // fp32 moved as 32-bit words
+    if (!make_tmap_words(&t_s, s, p.d_out, p.ngroups, a.sb_box) || !make_tmap_words(&t_b, b, p.d_out, p.ngroups, a.sb_box))
+      return L4Q_ERR_CUDA;
   }
   const size_t smem = wtile_smem_bytes(a);
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
@@ -666,7 +704,7 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   auto launch = [&](auto kern) -> l4q_status {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return L4Q_ERR_CUDA;
-    kern<<<grid, WT2_THREADS, smem, st>>>(t_w0, t_o0, t_o1, a);
+    kern<<<grid, WT2_THREADS, smem, st>>>(t_w0, t_o0, t_o1, t_s, t_b, a);
     return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
   };
   switch (mode) {
