@@ -165,6 +165,7 @@ struct LoraWorkspace {
   __half* fac = nullptr;         // QAT-LoRA backward: STE factors
   VariantScratch v{};
   float* zero_B = nullptr;       // QAT-LoRA: a zero LoRA factor, so that the weight-tile kernel quantizes W0 alone
+  void* op_img = nullptr;        // QAT-LoRA: the split operands of that kernel's merge (operand_image_bytes)
   float *dA_unused = nullptr, *dB_unused = nullptr;   // QAT-LoRA backward: the merged-layer LoRA gradients, not wanted
   size_t bytes = 0;
 };
@@ -182,6 +183,7 @@ LoraWorkspace lora_workspace(const l4q_desc* d, const Params& p, int kind, int o
   off += w.v.bytes;
   if (kind == L4Q_LORA_QAT) {
     w.zero_B = reinterpret_cast<float*>(take((size_t)p.d_out * p.rank * sizeof(float)));
+    if (operand_image_bytes(d, p)) w.op_img = take(operand_image_bytes(d, p));
     if (op == L4Q_OP_BWD) {
       w.dA_unused = reinterpret_cast<float*>(take((size_t)p.rank * p.d_in * sizeof(float)));
       w.dB_unused = reinterpret_cast<float*>(take((size_t)p.d_out * p.rank * sizeof(float)));
@@ -350,7 +352,7 @@ l4q_status l4q_lora_linear_fwd(const l4q_desc* desc, int kind, const void* X, co
   if (qat) {
     if (cudaMemsetAsync(w.zero_B, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess)
       return L4Q_ERR_CUDA;
-    if ((st = launch_dequant<true>(p, W0, A, w.zero_B, s, b, w.wq, nullptr, stream)) != L4Q_OK) return st;
+    if ((st = launch_dequant<true>(p, W0, A, w.zero_B, s, b, w.wq, nullptr, stream, w.op_img)) != L4Q_OK) return st;
     W = w.wq;
   }
   {
@@ -388,7 +390,7 @@ l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, co
   if (qat && (dX || ds)) {
     if (cudaMemsetAsync(w.zero_B, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess)
       return L4Q_ERR_CUDA;
-    if ((st = launch_dequant<true>(p, W0, A, w.zero_B, s, b, w.wq, ds ? w.fac : nullptr, stream)) != L4Q_OK)
+    if ((st = launch_dequant<true>(p, W0, A, w.zero_B, s, b, w.wq, ds ? w.fac : nullptr, stream, w.op_img)) != L4Q_OK)
       return st;
     W = w.wq;
   }

@@ -12,17 +12,23 @@
 //     each fp32 factor split into a tf32 head and a tf32 tail (x = hi + lo, three products hi*hi + hi*lo +
 //     lo*hi), which keeps ~21 mantissa bits -- the codes must agree with fp64 arithmetic except within
 //     1e-6 of a rounding boundary, which a single tf32 or bf16 product does not give;
-//   * 16 epilogue warps in four groups; a group owns every fourth tile of the CTA and one of the four
-//     accumulator stages, a thread one weight row of the group's tile.  It reads the merge from tensor memory
-//     with tcgen05.ld, the W0 tile from shared memory in 16-byte pieces, and does the quantizer arithmetic.
-//     The groups meet only through mbarriers, so four tiles are in flight per SM and the wait chain of one
-//     tile hides behind the arithmetic of the others.
+//   * 16 epilogue warps in two groups of eight; a group owns every second tile of the CTA and two of the four
+//     accumulator stages, a thread one weight row and one 64-column half of the group's tile.  It reads the
+//     merge from tensor memory with tcgen05.ld, the W0 tile from shared memory in 16-byte pieces, and does
+//     the quantizer arithmetic.  The groups meet only through mbarriers, so two tiles are worked on per SM
+//     while the loads, merges and stores of their neighbours are in flight;
+//   * nothing but that arithmetic is left to the epilogue warps where the caller provides scratch: the MMA
+//     operands of the merge (the tile's slices of A and B, each value split into tf32 head / tail, K-major
+//     with the 128-byte swizzle) are written once per launch for every row and column panel by
+//     k_split_operands, laid out as they stand in shared memory, and come in by two bulk copies per tile;
+//     s and b of the tile's rows come in by TMA with the W0 tile (where their row pitch allows).
 //
-// Roles (640 threads): warp 0 = TMA loads, warp 1 = MMA issuer + TMEM owner, warp 2 = TMA stores (one
-// thread each), warps 4..19 = epilogue (warp w: TMEM lane quarter w % 4, group (w - 4) / 4).  A group also
-// prepares the MMA operands of its next tile (splits the tile's slices of A and B into tf32 head / tail,
-// swizzled K-major) once the MMAs that last read the operand buffer have completed (two buffers up to rank
-// 32, one at rank 64), and copies s and b of its next tile's rows to per-thread scratch in shared memory.
+// Roles (640 threads): warp 0 = TMA loads (W0, s, b), warp 1 = MMA issuer + TMEM owner, warp 2 = TMA stores,
+// warp 3 = bulk copies of the operand images (one thread each), warps 4..19 = epilogue (warp w: TMEM lane
+// quarter w % 4, group (w - 4) / 8, column half ((w - 4) / 4) % 2).  Without operand images a group builds
+// the operands of its next tile itself once the MMAs that last read the operand buffer have completed (two
+// buffers up to rank 32, one at rank 64); without TMA boxes of s and b it copies those of its next tile's rows
+// to scratch in shared memory and meets at a named barrier per tile.
 // Every mbarrier wait is bounded (see bounded_wait); there is no block-level barrier after set-up.
 #pragma once
 
