@@ -524,30 +524,45 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
             const float w0[8] = {bf16_lo(wr.x), bf16_hi(wr.x), bf16_lo(wr.y), bf16_hi(wr.y),
                                  bf16_lo(wr.z), bf16_hi(wr.z), bf16_lo(wr.w), bf16_hi(wr.w)};
             float wq[8], fac[8];
+            // Eq. 7-9 and the STE factor: the arithmetic of quantize_elem / ste_factor, with the rounding done
+            // by the magic-number add (exact for the clamped range).  Two columns at a time on the packed fp32
+            // pipe: every packed operation is the same IEEE operation per lane as its scalar form.
+            const float2 gamma2 = make_float2(p.gamma, p.gamma), nb2 = make_float2(-b_, -b_), rs2 = make_float2(rs, rs);
+            const float2 s2v = make_float2(s_, s_), b2v = make_float2(b_, b_);
+            const float2 magic2 = make_float2(kRoundMagic, kRoundMagic), nmagic2 = make_float2(-kRoundMagic, -kRoundMagic);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              // Eq. 7-9 and the STE factor: the arithmetic of quantize_elem / ste_factor, with the rounding
-              // done by the magic-number add (exact for the clamped range)
-              const float wc = merge_elem(w0[e], __uint_as_float(raw[s2 * 8 + e]), p.gamma);
-              const float w = (wc - b_) * rs;
-              const float wcl = fminf(fmaxf(w, p.qn), p.qp);
-              const float y = wcl + kRoundMagic;
-              const float code = y - kRoundMagic;
-              wq[e] = fmaf(code, s_, b_);
+            for (int e = 0; e < 8; e += 2) {
+              const float2 acc2 = make_float2(__uint_as_float(raw[s2 * 8 + e]), __uint_as_float(raw[s2 * 8 + e + 1]));
+              const float2 wc = __ffma2_rn(gamma2, acc2, make_float2(w0[e], w0[e + 1]));      // merge_elem
+              const float2 w = __fmul2_rn(__fadd2_rn(wc, nb2), rs2);                         // (wc - b) * rs
+              const float2 wcl = make_float2(fminf(fmaxf(w.x, p.qn), p.qp), fminf(fmaxf(w.y, p.qn), p.qp));
+              const float2 y = __fadd2_rn(wcl, magic2);
+              const float2 code = __fadd2_rn(y, nmagic2);
+              const float2 q = __ffma2_rn(code, s2v, b2v);
+              wq[e] = q.x; wq[e + 1] = q.y;
               if constexpr (MODE == WT2_DEQUANT_F) {
-                const float t = w - wcl;                                            // 0 inside [Q_N, Q_P]
-                const float sentinel = __uint_as_float((__float_as_uint(t) & 0x80000000u) | 0x40000000u);   // +-2
-                fac[e] = (fabsf(t) > kMaskGuard) ? sentinel : code - w;
+                const float2 t2 = __fadd2_rn(w, make_float2(-wcl.x, -wcl.y));                 // 0 inside [Q_N, Q_P]
+                const float2 inr = __fadd2_rn(code, make_float2(-w.x, -w.y));                 // code - w
+                const float tt[2] = {t2.x, t2.y}, ii[2] = {inr.x, inr.y};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                  const float sentinel = __uint_as_float((__float_as_uint(tt[h]) & 0x80000000u) | 0x40000000u);   // +-2
+                  fac[e + h] = (fabsf(tt[h]) > kMaskGuard) ? sentinel : ii[h];
+                }
               }
               if constexpr (MODE == WT2_PACK) {                                     // code j of 32 at bit j * bits
-                const uint32_t u = (uint32_t)(__float_as_int(y) - qn_bits);
-                const int j = sub * 8 + e;
-                if (p.bits == 4) {
-                  words[j >> 3] |= u << ((j & 7) * 4);
-                } else {
-                  const int bit = j * 3, wd = bit >> 5, off = bit & 31;
-                  words[wd] |= u << off;
-                  if (off > 29) words[wd + 1] |= u >> (32 - off);
+                const float yy[2] = {y.x, y.y};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                  const uint32_t u = (uint32_t)(__float_as_int(yy[h]) - qn_bits);
+                  const int j = sub * 8 + e + h;
+                  if (p.bits == 4) {
+                    words[j >> 3] |= u << ((j & 7) * 4);
+                  } else {
+                    const int bit = j * 3, wd = bit >> 5, off = bit & 31;
+                    words[wd] |= u << off;
+                    if (off > 29) words[wd + 1] |= u >> (32 - off);
+                  }
                 }
               }
             }
