@@ -60,6 +60,22 @@ def test_bf16_ragged_tails(rank, bits, group, signed):
     check_layer(cfg, arrays, gh.run_layer(cfg, arrays, do_pack=True, grad_scale=0.25), grad_scale=0.25)
 
 
+@pytest.mark.parametrize("d_in,group,rank,bits,signed", [
+    (1216, 16, 16, 4, False),    # 76 groups, 9.5 column tiles: boxes of 12 groups, the last one past the end of the row
+    (1280, 64, 8, 3, True),      # 20 groups, 2 per tile: the box starts up to 2 groups left of the tile
+    (1536, 128, 32, 4, False),   # 12 groups, 1 per tile: offsets 0..3 inside the box
+    (2048, 32, 64, 4, False)])   # rank 64 (one operand buffer; plain-ALU kernel for the factor output)
+def test_bf16_wide_rows_scale_and_offset_by_tma(d_in, group, rank, bits, signed):
+    # rows with at least one box of groups and a pitch that is a multiple of 16 bytes: s and b reach the weight-tile
+    # kernel by TMA with the W0 tile (narrower rows, as in the cases above, are staged by the epilogue warps);
+    # d_out and the tokens leave partial tiles
+    cfg = synth.LayerConfig(f"bf16_wide_g{group}", tokens=200, d_in=d_in, d_out=200, rank=rank, alpha=32.0,
+                            bits=bits, group_size=group, signed_grid=signed)
+    arrays = synth.make_layer_inputs(cfg, seed=13)
+    arrays["s"] = (arrays["s"] * 0.9).astype(np.float32)          # some weights clip: db and the bound terms matter
+    check_layer(cfg, arrays, gh.run_layer(cfg, arrays, do_pack=True, grad_scale=0.5), grad_scale=0.5)
+
+
 @pytest.mark.parametrize("tokens", [1, 8, 100, 129])
 @pytest.mark.parametrize("d_out", [64, 392])
 def test_bf16_few_tokens_and_narrow_output(tokens, d_out):
