@@ -123,6 +123,15 @@ def test_qat_lora_with_clipped_weights():
     check_variant(cfg, arrays, l4q.L4Q_LORA_QAT)
 
 
+def test_qat_lora_wide_rows():
+    # 20 groups per row: s and b reach the weight-tile kernel by TMA (the narrower cases above stage them by hand)
+    cfg = synth.LayerConfig("variant_wide", tokens=200, d_in=1280, d_out=200, rank=16, alpha=32.0, bits=4,
+                            group_size=64)
+    arrays = _inputs(cfg, 15)
+    arrays["s"] = (arrays["s"] * 0.9).astype(np.float32)
+    check_variant(cfg, arrays, l4q.L4Q_LORA_QAT, grad_scale=0.5)
+
+
 def test_plain_lora_takes_any_rank_up_to_64():
     cfg = synth.LayerConfig("variant_r12", tokens=200, d_in=320, d_out=264, rank=12, alpha=24.0, bits=4,
                             group_size=64)
