@@ -116,13 +116,14 @@ inline l4q_status launch_status() { return cudaGetLastError() == cudaSuccess ? L
 // `fac` (optional, bf16 mode only) also receives the fp16 STE factors the weight-gradient kernel reads.
 template <bool IO_BF16>
 l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const float* B, const float* s,
-                          const float* b, void* wq, __half* fac, cudaStream_t st, void* op_img = nullptr) {
+                          const float* b, void* wq, __half* fac, cudaStream_t st, void* op_img = nullptr,
+                          const ZeroList* zero = nullptr, bool* zeroed = nullptr) {
   if constexpr (IO_BF16) {
     const int mode = fac ? WT2_DEQUANT_F : WT2_DEQUANT;
     if (wtile_tc_supported(p, mode)) {               // tensor-core merge, TMA in and out
       KernelScope ks(L4Q_KERNEL_DEQUANT, st);   // covers the operand split too, which is one more launch
       if (op_img) g_launches.fetch_add(1, std::memory_order_relaxed);
-      return launch_wtile_tc(mode, p, W0, A, B, s, b, wq, fac, nullptr, nullptr, st, op_img);
+      return launch_wtile_tc(mode, p, W0, A, B, s, b, wq, fac, nullptr, nullptr, st, op_img, zero, zeroed);
     }
   }
   const size_t smem = weight_tile_smem_bytes(p.rank);
@@ -273,14 +274,11 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   void* wq = workspace;
 
-  if (n_param_out == 4) {
-    // the reductions below accumulate with fp32 atomics: start from zero
-    const size_t gsz = (size_t)p.d_out * p.ngroups * sizeof(float);
-    if (cudaMemsetAsync(dA, 0, (size_t)p.rank * p.d_in * sizeof(float), stream) != cudaSuccess ||
-        cudaMemsetAsync(dB, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess ||
-        cudaMemsetAsync(ds, 0, gsz, stream) != cudaSuccess || cudaMemsetAsync(db, 0, gsz, stream) != cudaSuccess)
-      return L4Q_ERR_CUDA;
-  }
+  // the reductions below accumulate with fp32 atomics: dA, dB, ds, db start from zero.  The operand split of the
+  // recompute step clears them where it runs; otherwise four memsets do.
+  const size_t gn = (size_t)p.d_out * p.ngroups;
+  const ZeroList grads{{dA, dB, ds, db}, {(size_t)p.rank * p.d_in, (size_t)p.d_out * p.rank, gn, gn}};
+  bool zeroed = false;
   // recompute step (App. E.2): W_q for dX and, on the tensor-core path, the STE factors for the weight gradient
   __half* fac = (!f32 && n_param_out == 4)
                     ? reinterpret_cast<__half*>(static_cast<unsigned char*>(workspace) + wq_scratch_bytes(desc))
@@ -291,8 +289,16 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
                                     operand_image_bytes(desc, p)
                                         ? static_cast<unsigned char*>(workspace) + wq_scratch_bytes(desc) +
                                               factor_scratch_bytes(desc)
-                                        : nullptr);
+                                        : nullptr,
+                                    n_param_out == 4 ? &grads : nullptr, &zeroed);
     if (st != L4Q_OK) return st;
+  }
+  if (n_param_out == 4 && !zeroed) {
+    if (cudaMemsetAsync(dA, 0, grads.n[0] * sizeof(float), stream) != cudaSuccess ||
+        cudaMemsetAsync(dB, 0, grads.n[1] * sizeof(float), stream) != cudaSuccess ||
+        cudaMemsetAsync(ds, 0, grads.n[2] * sizeof(float), stream) != cudaSuccess ||
+        cudaMemsetAsync(db, 0, grads.n[3] * sizeof(float), stream) != cudaSuccess)
+      return L4Q_ERR_CUDA;
   }
   if (f32) {
     if (dX) {

@@ -201,7 +201,17 @@ __device__ __forceinline__ void operand_item_store(const WtileArgs& a, int idx, 
 // need not build them tile by tile: image tn (tn < tiles_n) is the acat block of column panel tn, image
 // tiles_n + tm the bcat block of row panel tm, each exactly as it stands in shared memory (op_half bytes), so
 // that one bulk copy brings it in.  One block per panel.
-__global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8_t* __restrict__ img) {
+// Output buffers of the caller that must start from zero (they are accumulated into with atomics later on the
+// stream): cleared by the same launch, which saves one memset launch per buffer.
+struct ZeroList { float* ptr[4]; size_t n[4]; };
+
+__global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8_t* __restrict__ img, const ZeroList zl) {
+  {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+      for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < zl.n[b]; e += stride) zl.ptr[b][e] = 0.f;
+  }
   const uint32_t op_half = (uint32_t)a.atoms * WT2_ATOM_BYTES;
   const int panel = blockIdx.x;
   uint8_t* dst = img + (size_t)panel * op_half;
@@ -690,10 +700,11 @@ inline size_t wtile_image_bytes(const Params& p) {
 
 // `op_img` (optional, wtile_image_bytes(p) bytes of device scratch, 16-byte aligned): with it the MMA operands are
 // split once by a launch of k_split_operands and reach the tiles by bulk copies; without it the epilogue warps
-// build them tile by tile.
+// build them tile by tile.  `zero` (optional): buffers that launch also clears; *zeroed is set when it did.
 inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, const float* A, const float* B,
                                   const float* s, const float* b, void* out0, void* out1, __half* s16, __half* b16,
-                                  cudaStream_t st, void* op_img = nullptr) {
+                                  cudaStream_t st, void* op_img = nullptr, const ZeroList* zero = nullptr,
+                                  bool* zeroed = nullptr) {
   WtileArgs a{};
   a.p = p; a.A = A; a.B = B; a.s = s; a.b = b; a.s16 = s16; a.b16 = b16;
   a.tiles_m = ceil_div(p.d_out, WT2_ROWS);
@@ -718,8 +729,11 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   const size_t smem = wtile_smem_bytes(a);
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
   if (op_img) {
-    k_split_operands<<<a.tiles_n + a.tiles_m, 256, 0, st>>>(a, static_cast<uint8_t*>(op_img));
+    ZeroList zl{};
+    if (zero) zl = *zero;
+    k_split_operands<<<a.tiles_n + a.tiles_m, 256, 0, st>>>(a, static_cast<uint8_t*>(op_img), zl);
     if (cudaGetLastError() != cudaSuccess) return L4Q_ERR_CUDA;
+    if (zero && zeroed) *zeroed = true;
     a.op_img = static_cast<const uint8_t*>(op_img);
   }
   auto launch = [&](auto kern) -> l4q_status {
