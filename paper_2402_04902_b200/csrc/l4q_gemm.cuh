@@ -83,23 +83,25 @@ inline size_t gemm_smem_bytes(int stages, int epi_bytes, int stage_bytes = STAGE
   return 1024 /*alignment slack*/ + (size_t)stages * stage_bytes + (size_t)epi_bytes + sizeof(GemmBarriers);
 }
 
-// Bounded mbarrier wait.  Returns immediately once the CTA's abort flag is set.
+// Bounded mbarrier wait.  Returns true once the phase has completed; false when it gave up because the time limit
+// ran out (it then sets the CTA's abort flag and the device status word) or because the abort flag was already set.
 template <class Barriers>
-__device__ __forceinline__ void bounded_wait(uint64_t* bar, uint32_t parity, Barriers* bars,
+__device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Barriers* bars,
                                              long long limit_cycles = WAIT_LIMIT_CYCLES) {
-  if (ptx::mbar_try_wait(bar, parity)) return;
+  if (ptx::mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!ptx::mbar_try_wait(bar, parity)) {
     if ((++spins & 0xFFu) == 0) {
-      if (bars->abort) return;
+      if (bars->abort) return false;
       if (clock64() - t0 > limit_cycles) {
         bars->abort = 1;
         atomicExch(&g_l4q_status, (unsigned int)L4Q_ERR_TIMEOUT);
-        return;
+        return false;
       }
     }
   }
+  return true;
 }
 
 // Self-test of the error path of bounded_wait: one block waits on a barrier that nothing ever arrives on, with

@@ -2,33 +2,35 @@
 // 128 x 128 tiles, streaming W0 once from HBM, and write one of
 //   WT2_DEQUANT    W_q (bf16)                      -- the recompute step of forward and backward (App. E.2)
 //   WT2_DEQUANT_F  W_q (bf16) + STE factors (fp16) -- backward: input gradient + weight-gradient reduction
+//                  (the factors leave from registers, 16 bytes per thread and 8-column piece, coalesced)
 //   WT2_PACK       bit-packed codes + fp16 s, b    -- export (Sec. 3.2)
 //
-// HBM-bound by design (2 bytes in, 2-4 bytes out per weight), so everything else is arranged to stay out
+// HBM-bound by design (2 bytes in, 0.4-4 bytes out per weight), so everything else is arranged to stay out
 // of the way of the copies:
-//   * W0 tiles arrive by TMA into 128-byte-swizzled shared memory (2-4 stages in flight); W_q is written
+//   * W0 tiles arrive by TMA into 128-byte-swizzled shared memory (up to 5 stages in flight); W_q is written
 //     back IN PLACE into the same stage and leaves by a TMA store, so every global access is a full line;
 //   * the rank-r merge B A is a tensor-core contraction: tcgen05.mma kind::tf32 into tensor memory, with
 //     each fp32 factor split into a tf32 head and a tf32 tail (x = hi + lo, three products hi*hi + hi*lo +
 //     lo*hi), which keeps ~21 mantissa bits -- the codes must agree with fp64 arithmetic except within
 //     1e-6 of a rounding boundary, which a single tf32 or bf16 product does not give;
-//   * 16 epilogue warps in two groups of eight; a group owns every second tile of the CTA and two of the four
-//     accumulator stages, a thread one weight row and one 64-column half of the group's tile.  It reads the
+//   * the MMA operands of the merge (the tile's slices of A and B, each value split into head / tail, K-major
+//     with the 128-byte swizzle) are written once per launch for every column and row panel by
+//     k_split_operands, laid out as they stand in shared memory.  A CTA works on a contiguous run of the
+//     column-panel-major tile sequence, so the A image of its column panel stays resident (reloaded at a panel
+//     change) and only the B image of the tile's row panel streams in, 16 KB (one swizzle atom of K) at a
+//     time through a ring of chunks, each released by the MMAs that read it;
+//   * 24 epilogue warps in three groups of eight; a group owns every third tile of the CTA (accumulator stage
+//     tile % 4), a thread one weight row and one 64-column half of the group's tile.  It reads the
 //     merge from tensor memory with tcgen05.ld, the W0 tile from shared memory in 16-byte pieces, and does
-//     the quantizer arithmetic.  The groups meet only through mbarriers, so two tiles are worked on per SM
-//     while the loads, merges and stores of their neighbours are in flight;
-//   * nothing but that arithmetic is left to the epilogue warps where the caller provides scratch: the MMA
-//     operands of the merge (the tile's slices of A and B, each value split into tf32 head / tail, K-major
-//     with the 128-byte swizzle) are written once per launch for every row and column panel by
-//     k_split_operands, laid out as they stand in shared memory, and come in by two bulk copies per tile;
-//     s and b of the tile's rows come in by TMA with the W0 tile (where their row pitch allows).
+//     the quantizer arithmetic.  Interior tiles whose half rows lie in one quantization
+//     group take wtile_half_row_fast (no per-element bounds or group logic; s and b come straight from
+//     global memory, one pair per thread and tile, fetched a tile ahead); every other tile takes the
+//     general loop.
 //
-// Roles (640 threads): warp 0 = TMA loads (W0, s, b), warp 1 = MMA issuer + TMEM owner, warp 2 = TMA stores,
-// warp 3 = bulk copies of the operand images (one thread each), warps 4..19 = epilogue (warp w: TMEM lane
-// quarter w % 4, group (w - 4) / 8, column half ((w - 4) / 4) % 2).  Without operand images a group builds
-// the operands of its next tile itself once the MMAs that last read the operand buffer have completed (two
-// buffers up to rank 32, one at rank 64); without TMA boxes of s and b it copies those of its next tile's rows
-// to scratch in shared memory and meets at a named barrier per tile.
+// Roles (896 threads): warp 0 = TMA loads (W0; s, b boxes where used), warp 1 = MMA issuer + TMEM owner,
+// warp 2 = TMA stores, warp 3 = operand loader (one thread issuing bulk copies of the ready-made images, or,
+// without images, the whole warp building the operands from A and B), warps 4..27 = epilogue (warp w: TMEM
+// lane quarter w % 4, group (w - 4) / 8, column half ((w - 4) / 4) % 2).
 // Every mbarrier wait is bounded (see bounded_wait); there is no block-level barrier after set-up.
 #pragma once
 
@@ -39,15 +41,20 @@
 namespace l4q {
 
 constexpr int WT2_ROWS = 128, WT2_COLS = 128;
-constexpr int WT2_THREADS = 640;
+#ifndef WT2_NGROUPS
+#define WT2_NGROUPS 2
+#endif
+constexpr int WT2_THREADS = 128 + 256 * WT2_NGROUPS;
 constexpr int WT2_FIRST_EPI_WARP = 4;
-constexpr int WT2_EPI_THREADS = 512;
-constexpr int WT2_GROUPS = 2;                       // epilogue warp groups; each owns every second tile of the CTA
+constexpr int WT2_EPI_THREADS = 256 * WT2_NGROUPS;
+constexpr int WT2_GROUPS = WT2_NGROUPS;                       // epilogue warp groups; each owns every third tile of the CTA
 constexpr int WT2_GROUP_THREADS = WT2_EPI_THREADS / WT2_GROUPS;
 constexpr int WT2_ACC = 4;                          // accumulator stages of 128 TMEM columns
 constexpr int WT2_STAGE_BYTES = WT2_ROWS * WT2_COLS * 2;   // one bf16 tile: two 128 x 64 swizzled boxes
 constexpr int WT2_ATOM_BYTES = 128 * 128;           // 128 rows x 32 tf32 (one 128-byte swizzle atom along K)
-constexpr int WT2_MAX_STAGES = 4;
+constexpr int WT2_MAX_STAGES = 6;
+constexpr int WT2_MAX_BSLOTS = 8;
+constexpr int WT2_MAX_ATOMS = 4;                    // rank <= 64
 
 enum { WT2_DEQUANT = 0, WT2_DEQUANT_F = 1, WT2_PACK = 2 };
 
@@ -58,15 +65,17 @@ struct WtileArgs {
   __half* F;               // WT2_DEQUANT_F: the factor array (factor_index layout)
   const uint8_t* op_img;   // optional: the split MMA operands of every panel, ready made (see k_split_operands)
   int tiles_m, tiles_n;
-  int n_stages;            // W0 stages in shared memory (2..4)
-  int n_out;               // staging buffers for the second output (F or codes): 0, 1 or 2
+  int n_stages;            // W0 stages in shared memory (2..5)
+  int n_out;               // staging buffers for the code words of the export: 0 (other modes) .. 3
   int out_bytes;           // bytes of one such buffer
   int atoms;               // swizzle atoms per operand row: ceil(2 rank / 32)
   int ngt;                 // upper bound of the quantization groups a 128-column tile intersects
-  int n_opbuf;             // MMA operand buffers ([A slice | B slice] each): 1 or 2
+  int n_abuf;              // buffers for the A image of a column panel (atoms x 16 KB each): 1 or 2
+  int n_bslot;             // ring of 16 KB chunks of the B images
   int group_shift;         // log2(group size) if it is a power of two, else -1
-  int sb_box;              // groups per row of the s / b boxes that TMA brings in with the W0 tile; 0: the epilogue
-                           // warps stage s and b themselves
+  int fast;                // interior tiles take wtile_half_row_fast (group a multiple of 64); s and b are then read
+                           // from global memory and no copy of them is staged in shared memory
+  int sb_box;              // groups per row of the s / b boxes that TMA brings in with the W0 tile; 0: none
 };
 
 // column / group size without a division in the common power-of-two case
@@ -78,51 +87,54 @@ struct __align__(8) WtileBarriers {
   uint64_t full[WT2_MAX_STAGES];      // W0 tile has landed in the stage
   uint64_t empty[WT2_MAX_STAGES];     // the stage may be overwritten (its store has read it)
   uint64_t written[WT2_MAX_STAGES];   // the epilogue has written the stage's outputs
-  uint64_t out_empty[2];              // second-output staging buffer may be overwritten
-  uint64_t prep_full[2];              // split LoRA operands are complete in operand buffer b
+  uint64_t out_empty[3];              // staging buffer of the code words may be overwritten
+  uint64_t afull[2], aempty[2];       // A image of a column panel: complete in buffer b / no longer read by any MMA
+  uint64_t bfull[WT2_MAX_BSLOTS], bempty[WT2_MAX_BSLOTS];   // one chunk of a B image, likewise
   uint64_t tmem_full[WT2_ACC], tmem_empty[WT2_ACC];
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
 
-// s and b in shared memory: per epilogue thread [s x ngt | b x ngt] floats of its weight row (1 KB multiples
-// in total); a thread reads and writes its own entry only.
+// s and b staged in shared memory by the epilogue warps (general path without TMA boxes): per epilogue thread
+// [s x ngt | b x ngt] floats of its weight row; a thread reads and writes its own entry only.
 __host__ __device__ inline size_t wtile_sb_bytes(int ngt) { return (size_t)WT2_EPI_THREADS * 2 * ngt * sizeof(float); }
 
-// With sb_box: per W0 stage one box [128 rows][sb_box] of s and one of b.
+// With sb_box: per W0 stage one box [128 rows][sb_box] of s and one of b.  On the fast path: nothing.
 __host__ __device__ inline size_t wtile_sb_region_bytes(const WtileArgs& a) {
+  if (a.fast) return 0;
   return a.sb_box ? (size_t)a.n_stages * 2 * WT2_ROWS * a.sb_box * sizeof(float) : wtile_sb_bytes(a.ngt);
 }
 inline size_t wtile_smem_bytes(const WtileArgs& a) {
   return 1024 + (size_t)a.n_stages * WT2_STAGE_BYTES + (size_t)a.n_out * a.out_bytes +
-         2 * (size_t)a.n_opbuf * a.atoms * WT2_ATOM_BYTES + wtile_sb_region_bytes(a) + sizeof(WtileBarriers);
+         ((size_t)a.n_abuf * a.atoms + a.n_bslot) * WT2_ATOM_BYTES + wtile_sb_region_bytes(a) + sizeof(WtileBarriers);
 }
 
-// The tiles of one CTA: tile t of the column-panel-major sequence (row tiles of one column panel are
-// consecutive) goes to CTA t mod gridDim.x.  Coordinates advance without divisions.
+// The tiles of one CTA: a contiguous run [t0, t1) of the column-panel-major sequence (row tiles of one column
+// panel are consecutive), runs of equal length up to one tile, so that the A image of a column panel is loaded
+// once or twice per CTA.  (Handing tiles out strided by the grid size, neighbouring CTAs on neighbouring row
+// tiles, was measured and made no difference to the memory system.)  Coordinates advance without divisions.
 struct TileCursor {
-  int t, total, tm, tn, tiles_m, dm, dn;
-  int step;
-  // the CTA's tiles number first, first + stride, ... of its own sequence
+  int t, t1, tm, tn, tiles_m, step;
+  // the run's tiles number first, first + stride, ...
   __device__ explicit TileCursor(const WtileArgs& a, int first = 0, int stride = 1) {
-    total = a.tiles_m * a.tiles_n;
+    const long long total = (long long)a.tiles_m * a.tiles_n;
     tiles_m = a.tiles_m;
-    t = blockIdx.x + first * (int)gridDim.x;
+    t = (int)(total * blockIdx.x / gridDim.x) + first;
+    t1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
     tn = t / tiles_m; tm = t - tn * tiles_m;
-    step = stride * (int)gridDim.x;
-    dn = step / tiles_m; dm = step - dn * tiles_m;
+    step = stride;
   }
-  __device__ bool valid() const { return t < total; }
+  __device__ bool valid() const { return t < t1; }
   __device__ void next() {
-    t += step; tn += dn; tm += dm;
-    if (tm >= tiles_m) { tm -= tiles_m; ++tn; }
+    t += step; tm += step;
+    while (tm >= tiles_m) { tm -= tiles_m; ++tn; }
   }
   __device__ int m0() const { return tm * WT2_ROWS; }
   __device__ int n0() const { return tn * WT2_COLS; }
-  // coordinates of this CTA's tile k (small) steps ahead; false beyond the end
+  // coordinates of the run's tile k (small) steps ahead; false beyond the end
   __device__ bool peek(int k, int& m0_, int& n0_) const {
-    if (t + k * step >= total) return false;
-    int m = tm + k * dm, n = tn + k * dn;
+    if (t + k * step >= t1) return false;
+    int m = tm + k * step, n = tn;
     while (m >= tiles_m) { m -= tiles_m; ++n; }
     m0_ = m * WT2_ROWS; n0_ = n * WT2_COLS;
     return true;
@@ -136,99 +148,73 @@ __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
   lo = __uint_as_float(__float_as_uint(x - hi) & 0xFFFFE000u);
 }
 
-// MMA operands of one tile in shared memory, K-major with the 128-byte swizzle:
-//   acat row n = column n0 + n of the weight:  [ hi(A[0..r, col]) | lo(A[0..r, col]) ]
-//   bcat row m = row m0 + m of the weight:      [ hi(B[row, 0..r]) | lo(B[row, 0..r]) ]
-// A work item (32 r per tile) is 4 consecutive ranks of one row of each slice.  Item idx takes column
-// idx % 128, ranks 4 (idx / 128) of the A slice -- a warp reads 32 consecutive columns of one rank, coalesced --
-// and the idx-th 16 bytes of the B slice, which is one contiguous block of 128 r floats, so a warp reads 512
-// consecutive bytes.
-struct OperandItem { float av[4]; float4 bv; };
-
-__device__ __forceinline__ void operand_a_load(const WtileArgs& a, int n0, int idx, float (&av)[4]) {
+// MMA operands of one tile, K-major with the 128-byte swizzle, one atom (32 values of K, 16 KB) at a time:
+//   A image, row n = column n0 + n of the weight:  [ hi(A[0..r, col]) | lo(A[0..r, col]) ]
+//   B image, row m = row m0 + m of the weight:      [ hi(B[row, 0..r]) | lo(B[row, 0..r]) ]
+// Atom c holds values 32 c .. 32 c + 31 of that concatenation (beyond 2 r: zero).  A work item is one 16-byte
+// piece (4 values) of one row: item it -> row it % 128, piece it / 128, so that a warp reads 32 consecutive
+// columns of A (coalesced) or 32 rows of B.  `dst`: the atom, in shared or global memory.
+__device__ __forceinline__ void build_atom_a(const WtileArgs& a, int n0, int c, uint8_t* dst, int tid, int nthreads) {
   const Params& p = a.p;
-  const int row = idx & 127, kc = idx >> 7, col = n0 + row;
+  for (int it = tid; it < 1024; it += nthreads) {
+    const int row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j, col = n0 + row;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (e0 < 2 * p.rank && col < p.d_in) {
+      const bool tail = e0 >= p.rank;
+      const int k = tail ? e0 - p.rank : e0;
+      float x[4], h[4], l[4];
 #pragma unroll
-  for (int e = 0; e < 4; ++e) av[e] = (col < p.d_in) ? __ldg(a.A + (size_t)(4 * kc + e) * p.d_in + col) : 0.f;
+      for (int e = 0; e < 4; ++e) {
+        x[e] = __ldg(a.A + (size_t)(k + e) * p.d_in + col);
+        split_tf32(x[e], h[e], l[e]);
+      }
+      v = tail ? make_float4(l[0], l[1], l[2], l[3]) : make_float4(h[0], h[1], h[2], h[3]);
+    }
+    *reinterpret_cast<float4*>(dst + row * 128 + ((j ^ (row & 7)) << 4)) = v;
+  }
 }
 
-__device__ __forceinline__ void operand_b_load(const WtileArgs& a, int m0, int idx, float4& bv) {
+__device__ __forceinline__ void build_atom_b(const WtileArgs& a, int m0, int c, uint8_t* dst, int tid, int nthreads) {
   const Params& p = a.p;
-  const int rq = p.rank >> 2;                        // 16-byte pieces per row of B
-  const int brow = idx / rq;
-  bv = (m0 + brow < p.d_out) ? __ldg(reinterpret_cast<const float4*>(a.B + (size_t)m0 * p.rank) + idx)
-                             : make_float4(0.f, 0.f, 0.f, 0.f);
-}
-
-__device__ __forceinline__ void operand_a_store(const WtileArgs& a, int idx, const float (&av)[4], uint8_t* acat) {
-  const int row = idx & 127, kc = idx >> 7;
-  float ah[4], al[4];
+  for (int it = tid; it < 1024; it += nthreads) {
+    const int row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j, o = m0 + row;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (e0 < 2 * p.rank && o < p.d_out) {
+      const bool tail = e0 >= p.rank;
+      const int k = tail ? e0 - p.rank : e0;
+      const float4 bv = __ldg(reinterpret_cast<const float4*>(a.B + (size_t)o * p.rank + k));
+      const float x[4] = {bv.x, bv.y, bv.z, bv.w};
+      float h[4], l[4];
 #pragma unroll
-  for (int e = 0; e < 4; ++e) split_tf32(av[e], ah[e], al[e]);
-  const int ch = kc, cl = (a.p.rank >> 2) + kc;      // 16-byte chunk index of the head / tail within the row
-  const uint32_t off_h = (uint32_t)(ch >> 3) * WT2_ATOM_BYTES + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
-  const uint32_t off_l = (uint32_t)(cl >> 3) * WT2_ATOM_BYTES + row * 128 + (((cl & 7) ^ (row & 7)) << 4);
-  *reinterpret_cast<float4*>(acat + off_h) = make_float4(ah[0], ah[1], ah[2], ah[3]);
-  *reinterpret_cast<float4*>(acat + off_l) = make_float4(al[0], al[1], al[2], al[3]);
+      for (int e = 0; e < 4; ++e) split_tf32(x[e], h[e], l[e]);
+      v = tail ? make_float4(l[0], l[1], l[2], l[3]) : make_float4(h[0], h[1], h[2], h[3]);
+    }
+    *reinterpret_cast<float4*>(dst + row * 128 + ((j ^ (row & 7)) << 4)) = v;
+  }
 }
 
-__device__ __forceinline__ void operand_b_store(const WtileArgs& a, int idx, const float4& bv, uint8_t* bcat) {
-  const int rq = a.p.rank >> 2;
-  const int brow = idx / rq, bkc = idx - brow * rq;
-  const float bvv[4] = {bv.x, bv.y, bv.z, bv.w};
-  float bh[4], bl[4];
-#pragma unroll
-  for (int e = 0; e < 4; ++e) split_tf32(bvv[e], bh[e], bl[e]);
-  const int bch = bkc, bcl = rq + bkc;
-  const uint32_t boff_h = (uint32_t)(bch >> 3) * WT2_ATOM_BYTES + brow * 128 + (((bch & 7) ^ (brow & 7)) << 4);
-  const uint32_t boff_l = (uint32_t)(bcl >> 3) * WT2_ATOM_BYTES + brow * 128 + (((bcl & 7) ^ (brow & 7)) << 4);
-  *reinterpret_cast<float4*>(bcat + boff_h) = make_float4(bh[0], bh[1], bh[2], bh[3]);
-  *reinterpret_cast<float4*>(bcat + boff_l) = make_float4(bl[0], bl[1], bl[2], bl[3]);
-}
-
-__device__ __forceinline__ void operand_item_load(const WtileArgs& a, int m0, int n0, int idx, OperandItem& it) {
-  operand_a_load(a, n0, idx, it.av);
-  operand_b_load(a, m0, idx, it.bv);
-}
-
-__device__ __forceinline__ void operand_item_store(const WtileArgs& a, int idx, const OperandItem& it, uint8_t* acat,
-                                                   uint8_t* bcat) {
-  operand_a_store(a, idx, it.av, acat);
-  operand_b_store(a, idx, it.bv, bcat);
-}
-
-// The operand images of all panels, written once per launch of the weight-tile kernel so that its epilogue warps
-// need not build them tile by tile: image tn (tn < tiles_n) is the acat block of column panel tn, image
-// tiles_n + tm the bcat block of row panel tm, each exactly as it stands in shared memory (op_half bytes), so
-// that one bulk copy brings it in.  One block per panel.
+// The operand images of all panels, written once per launch of the weight-tile kernel: image tn (tn < tiles_n)
+// is the A image of column panel tn, image tiles_n + tm the B image of row panel tm, each `atoms` atoms exactly
+// as they stand in shared memory, so that bulk copies bring them in.  One block per panel.
 // Output buffers of the caller that must start from zero (they are accumulated into with atomics later on the
 // stream): cleared by the same launch, which saves one memset launch per buffer.
 struct ZeroList { float* ptr[4]; size_t n[4]; };
 
 __global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8_t* __restrict__ img, const ZeroList zl) {
+  // the weight-tile kernel that follows may start now: it loads W0 tiles while the images are being written and
+  // waits for this grid (griddep_wait) only before it copies the first image
+  ptx::griddep_launch_dependents();
   {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
 #pragma unroll
     for (int b = 0; b < 4; ++b)
       for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < zl.n[b]; e += stride) zl.ptr[b][e] = 0.f;
   }
-  const uint32_t op_half = (uint32_t)a.atoms * WT2_ATOM_BYTES;
   const int panel = blockIdx.x;
-  uint8_t* dst = img + (size_t)panel * op_half;
-  const int n_items = 32 * a.p.rank;
-  // chunks of an atom row beyond 2 rank values are never read by the MMAs; the image leaves them as they are
-  if (panel < a.tiles_n) {
-    for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
-      float av[4];
-      operand_a_load(a, panel * WT2_COLS, idx, av);
-      operand_a_store(a, idx, av, dst);
-    }
-  } else {
-    for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
-      float4 bv;
-      operand_b_load(a, (panel - a.tiles_n) * WT2_ROWS, idx, bv);
-      operand_b_store(a, idx, bv, dst);
-    }
+  uint8_t* dst = img + (size_t)panel * a.atoms * WT2_ATOM_BYTES;
+  for (int c = 0; c < a.atoms; ++c) {
+    if (panel < a.tiles_n) build_atom_a(a, panel * WT2_COLS, c, dst + (size_t)c * WT2_ATOM_BYTES, threadIdx.x, blockDim.x);
+    else build_atom_b(a, (panel - a.tiles_n) * WT2_ROWS, c, dst + (size_t)c * WT2_ATOM_BYTES, threadIdx.x, blockDim.x);
   }
 }
 
@@ -236,6 +222,208 @@ __global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8
 // rintf, on the FP32 add pipe; the low mantissa bits of the intermediate sum hold that integer.
 constexpr float kRoundMagic = 12582912.0f;
 constexpr int kRoundMagicBits = 0x4B400000;
+
+// The merge MMAs of one B chunk (atom c of the tile's B image, at shared address `bchunk`) against the resident
+// A image at `acat`:  B A = Bhi Ahi + Bhi Alo + Blo Ahi  (the tail x tail product is below fp32 resolution of
+// the sum).  A K step is 8 values (32 bytes); a head step of B meets the head and the tail of A, a tail step
+// the head of A.  `first` : the tile's first MMA overwrites the accumulator.  With R known at compile time the
+// whole sequence is straight-line code: the issuing thread shares its scheduler with four epilogue warps, and
+// every instruction of a data-dependent address computation costs it several cycles.
+__device__ __forceinline__ uint64_t wt_desc(uint32_t lo_base, uint32_t byte_off) {
+  constexpr uint32_t HI = ((1024u >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);   // SBO 1024, version 1, 128-byte swizzle
+  return ((uint64_t)HI << 32) | (lo_base + (byte_off >> 4));
+}
+__device__ __forceinline__ uint32_t wt_desc_lo(uint32_t smem_addr) {
+  return ((smem_addr >> 4) & 0x3FFFu) | (1u << 16);                            // start address, LBO 16 bytes
+}
+// byte offset of value e of an image row inside the image (atom, then position in the 128-byte row)
+__host__ __device__ constexpr uint32_t wt_elem_off(int e) { return (uint32_t)(e >> 5) * WT2_ATOM_BYTES + (uint32_t)(e & 31) * 4u; }
+
+template <int R>
+__device__ __forceinline__ void issue_chunk_mmas(int c, int rank, uint32_t bchunk, uint32_t acat, uint32_t d_tmem) {
+  constexpr uint32_t idesc = ptx::make_idesc_tf32(WT2_ROWS, WT2_COLS);
+  const uint32_t b_lo = wt_desc_lo(bchunk), a_lo = wt_desc_lo(acat);
+  const int r = R > 0 ? R : rank;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int e = 32 * c + 8 * k;                    // value index in the B row
+    if (e >= 2 * r) break;
+    const uint64_t dm = wt_desc(b_lo, (uint32_t)k * 32u);
+    if (e < r) {
+      ptx::mma_tf32_ss(d_tmem, dm, wt_desc(a_lo, wt_elem_off(e)), idesc, e != 0 ? 1u : 0u);
+      ptx::mma_tf32_ss(d_tmem, dm, wt_desc(a_lo, wt_elem_off(r + e)), idesc, 1u);
+    } else {
+      ptx::mma_tf32_ss(d_tmem, dm, wt_desc(a_lo, wt_elem_off(e - r)), idesc, 1u);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Epilogue arithmetic of an interior tile whose half rows (64 columns of one weight row) lie inside one
+// quantization group: the arithmetic of quantize_elem / ste_factor, element for element the same operations in
+// the same order as everywhere else in the library (so that every kernel takes the same rounding and gating
+// decisions, ties included), without bounds tests or group bookkeeping per element, two columns at a time on
+// the packed fp32 pipe, with the rounding done by the magic-number add (exact for the clamped range).
+// ---------------------------------------------------------------------------
+
+// Sum over j < n of (1.5 * 2^23 as bits) << (j * bits), modulo 2^32: what the magic-number bit patterns add up to
+// when n raw y words are accumulated at their bit offsets instead of the bare codes.
+__host__ __device__ constexpr uint32_t magic_bias(int n, int bits) {
+  uint32_t k = 0;
+  for (int j = 0; j < n; ++j) k += (j * bits < 32) ? ((uint32_t)0x4B400000u << (j * bits)) : 0u;
+  return k;
+}
+
+// Per-thread constants of a tile on the fast path.
+struct FastConsts {
+  float s, b, rs;        // rs = 1 / s
+  float qn, qp, gamma;
+};
+
+// One half row (64 columns) of an interior tile.  `taddr`: TMEM address of the thread's first merge column;
+// `tile_row`: the thread's row of the W0 stage (swizzled; pieces of 16 bytes).  MODE WT2_DEQUANT /
+// WT2_DEQUANT_F: W_q overwrites W0 in place, the factors go to `out1` (the tile's block of the factor array);
+// WT2_PACK (unsigned grid only): the code words go to `out1` (the tile's staging rows).
+template <int MODE, int BITS>
+__device__ __forceinline__ void wtile_half_row_fast(const FastConsts& c, uint32_t taddr, uint8_t* tile_row, int row,
+                                                    int chalf, uint8_t* out1, uint64_t* tmem_empty_bar) {
+  const float2 gamma2 = make_float2(c.gamma, c.gamma), nb2 = make_float2(-c.b, -c.b), rs2 = make_float2(c.rs, c.rs);
+  const float2 magic2 = make_float2(kRoundMagic, kRoundMagic);
+  [[maybe_unused]] const float2 nmagic2 = make_float2(-kRoundMagic, -kRoundMagic);
+  [[maybe_unused]] const float2 s2v = make_float2(c.s, c.s), b2v = make_float2(c.b, c.b);
+  [[maybe_unused]] uint32_t words[4];                                           // BITS == 4: four words = 32 codes
+  [[maybe_unused]] uint32_t h3[3] = {0u, 0u, 0u}, carry10 = 0u, carry21 = 0u;   // BITS == 3: 32 codes -> 3 words
+  uint32_t raw[2][16];
+  ptx::tmem_ld_32x16(taddr, raw[0]);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {                       // 16 columns
+    ptx::tmem_ld_wait();
+    if (q < 3) {
+      ptx::tmem_ld_32x16(taddr + (uint32_t)((q + 1) * 16), raw[(q + 1) & 1]);
+    } else {                                          // all of the thread's merge columns are in registers
+      ptx::tc_fence_before_sync();
+      ptx::mbar_arrive(tmem_empty_bar);
+    }
+    const uint32_t(&acc)[16] = raw[q & 1];
+#pragma unroll
+    for (int s2 = 0; s2 < 2; ++s2) {
+      const int pin = q * 2 + s2;                     // piece of the half row
+      const int piece = chalf * 8 + pin;              // piece of the tile row (chalf selects the 64-column box)
+      const uint32_t chunk = (uint32_t)((piece >> 3) * (WT2_STAGE_BYTES / 2) + (((piece & 7) ^ (row & 7)) << 4));
+      const uint4 wr = *reinterpret_cast<const uint4*>(tile_row + chunk);
+      const uint32_t wv[4] = {wr.x, wr.y, wr.z, wr.w};
+      [[maybe_unused]] uint32_t qo[4];
+      [[maybe_unused]] uint32_t fo[4];
+      [[maybe_unused]] uint32_t word4 = 0u;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 acc2 = make_float2(__uint_as_float(acc[s2 * 8 + 2 * e]), __uint_as_float(acc[s2 * 8 + 2 * e + 1]));
+        const float2 wc = __ffma2_rn(gamma2, acc2, make_float2(bf16_lo(wv[e]), bf16_hi(wv[e])));
+        const float2 w = __fmul2_rn(__fadd2_rn(wc, nb2), rs2);                     // (wc - b) * rs
+        const float2 wcl = make_float2(fminf(fmaxf(w.x, c.qn), c.qp), fminf(fmaxf(w.y, c.qn), c.qp));
+        const float2 y = __fadd2_rn(wcl, magic2);
+        if constexpr (MODE != WT2_PACK) {
+          const float2 code = __fadd2_rn(y, nmagic2);
+          const float2 wq = __ffma2_rn(code, s2v, b2v);
+          qo[e] = pack_bf16x2(wq.x, wq.y);
+          if constexpr (MODE == WT2_DEQUANT_F) {
+            const float2 t2 = __fadd2_rn(w, make_float2(-wcl.x, -wcl.y));          // 0 inside [Q_N, Q_P]
+            const float2 inr = __fadd2_rn(code, make_float2(-w.x, -w.y));          // w~ - w
+            const float tt[2] = {t2.x, t2.y}, ii[2] = {inr.x, inr.y};
+            float f[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const float sentinel = __uint_as_float((__float_as_uint(tt[h]) & 0x80000000u) | 0x40000000u);   // +-2
+              f[h] = (fabsf(tt[h]) > kMaskGuard) ? sentinel : ii[h];
+            }
+            const __half2 hh = __floats2half2_rn(f[0], f[1]);
+            fo[e] = *reinterpret_cast<const uint32_t*>(&hh);
+          }
+        } else {
+          const uint32_t yb[2] = {__float_as_uint(y.x), __float_as_uint(y.y)};
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            if constexpr (BITS == 4) {
+              const int j = 2 * e + h;                                           // code j of the word at bit 4 j
+              word4 = (j == 0) ? yb[h] : word4 + (yb[h] << (4 * j));
+            } else {
+              const int j = (pin & 3) * 8 + 2 * e + h;                           // code j of 32 at bit 3 j of 3 words
+              if (j < 10) h3[0] += yb[h] << (3 * j);
+              else if (j == 10) carry10 = yb[h] & 7u;
+              else if (j < 21) h3[1] += yb[h] << (3 * (j - 11) + 1);
+              else if (j == 21) carry21 = yb[h] & 7u;
+              else h3[2] += yb[h] << (3 * (j - 22) + 2);
+            }
+          }
+        }
+      }
+      if constexpr (MODE != WT2_PACK)
+        *reinterpret_cast<uint4*>(tile_row + chunk) = make_uint4(qo[0], qo[1], qo[2], qo[3]);   // in place
+      if constexpr (MODE == WT2_DEQUANT_F)
+        *reinterpret_cast<uint4*>(out1 + (piece * WT2_ROWS + row) * 16) = make_uint4(fo[0], fo[1], fo[2], fo[3]);
+      // staging row = the tile's 128 codes of this weight row; this thread writes 64 of them, 32 at a time
+      if constexpr (MODE == WT2_PACK && BITS == 4) {
+        words[pin & 3] = word4 - magic_bias(8, 4);
+        if ((pin & 3) == 3)
+          *reinterpret_cast<uint4*>(out1 + row * 64 + chalf * 32 + (pin >> 2) * 16) =
+              make_uint4(words[0], words[1], words[2], words[3]);
+      }
+      if constexpr (MODE == WT2_PACK && BITS == 3) {
+        if ((pin & 3) == 3) {
+          uint32_t* dst = reinterpret_cast<uint32_t*>(out1 + row * 48 + chalf * 24 + (pin >> 2) * 12);
+          dst[0] = (h3[0] - magic_bias(10, 3)) + (carry10 << 30);
+          dst[1] = (h3[1] - (magic_bias(10, 3) << 1)) + (carry10 >> 2) + (carry21 << 31);
+          dst[2] = (h3[2] - (magic_bias(10, 3) << 2)) + (carry21 >> 1);
+          h3[0] = h3[1] = h3[2] = 0u;
+        }
+      }
+    }
+  }
+}
+
+// The MMA issuer of the weight-tile kernel: one thread.  It shares its warp scheduler with four epilogue warps, so
+// every instruction here waits its turn: the loop is kept to the barrier polls, the MMAs with descriptors that
+// differ from precomputed ones by constants, and the tile cursor (no flag reads: a wait that gives up reports it).
+template <int R>
+__device__ __forceinline__ void wtile_mma_role(const WtileArgs& a, WtileBarriers* bars, uint32_t tmem_base,
+                                               uint32_t acat_addr, uint32_t bslot_addr) {
+  TileCursor cur(a);
+  int panel = cur.tn;
+  const int ashift = a.n_abuf - 1;                          // n_abuf is 1 or 2
+  const uint32_t a_img_bytes = (uint32_t)a.atoms * WT2_ATOM_BYTES;
+  const int atoms = R > 0 ? (2 * R + 31) / 32 : a.atoms;
+  int acc = 0; uint32_t acc_phase = 0;
+  int slot = 0; uint32_t slot_phase = 0;
+  int pseq = 0, ab = 0;
+  if (!bounded_wait(&bars->afull[0], 0u, bars)) return;
+  for (; cur.valid();) {
+    if (!bounded_wait(&bars->tmem_empty[acc], acc_phase ^ 1, bars)) return;
+    ptx::tc_fence_after_sync();
+    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * WT2_COLS);
+    const uint32_t acat_a = acat_addr + (uint32_t)ab * a_img_bytes;
+#pragma unroll
+    for (int c = 0; c < (R > 0 ? atoms : WT2_MAX_ATOMS); ++c) {
+      if (R == 0 && c >= atoms) break;
+      if (!bounded_wait(&bars->bfull[slot], slot_phase, bars)) return;
+      ptx::tc_fence_after_sync();
+      issue_chunk_mmas<R>(c, a.p.rank, bslot_addr + (uint32_t)slot * WT2_ATOM_BYTES, acat_a, d_tmem);
+      ptx::mma_commit(&bars->bempty[slot]);        // the chunk may be overwritten once these MMAs have read it
+      if (++slot == a.n_bslot) { slot = 0; slot_phase ^= 1; }
+    }
+    ptx::mma_commit(&bars->tmem_full[acc]);
+    if (++acc == WT2_ACC) { acc = 0; acc_phase ^= 1; }
+    cur.next();
+    if (cur.valid() && cur.tn != panel) {
+      // the MMAs issued so far are the last readers of this panel's A image; the next panel's is in the other
+      // buffer (or about to replace this one)
+      ptx::mma_commit(&bars->aempty[ab]);
+      panel = cur.tn;
+      ++pseq;
+      ab = pseq & ashift;
+      if (!bounded_wait(&bars->afull[ab], (uint32_t)((pseq >> ashift) & 1), bars)) return;
+    }
+  }
+}
 
 template <int MODE>
 __global__ void __launch_bounds__(WT2_THREADS, 1)
@@ -249,22 +437,32 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
   uint8_t* out_base = stage_base + (size_t)a.n_stages * WT2_STAGE_BYTES;
-  uint8_t* op_base = out_base + (size_t)a.n_out * a.out_bytes;          // operand buffer b: [acat | bcat]
-  const uint32_t op_half = (uint32_t)a.atoms * WT2_ATOM_BYTES;           // bytes of one acat or bcat
-  float* sb_base = reinterpret_cast<float*>(op_base + (size_t)a.n_opbuf * 2 * op_half);
+  uint8_t* acat_base = out_base + (size_t)a.n_out * a.out_bytes;        // A image buffer b: atoms x 16 KB
+  const uint32_t a_img_bytes = (uint32_t)a.atoms * WT2_ATOM_BYTES;
+  uint8_t* bslot_base = acat_base + (size_t)a.n_abuf * a_img_bytes;     // ring of 16 KB chunks of B images
+  float* sb_base = reinterpret_cast<float*>(bslot_base + (size_t)a.n_bslot * WT2_ATOM_BYTES);
   WtileBarriers* bars = reinterpret_cast<WtileBarriers*>(reinterpret_cast<uint8_t*>(sb_base) + wtile_sb_region_bytes(a));
   const Params& p = a.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr bool HAS_OUT1 = (MODE != WT2_DEQUANT);
+  constexpr bool HAS_OUT1 = (MODE == WT2_PACK);      // staged in shared memory: the code words of the export
 
   if (threadIdx.x == 0) {
+    const uint32_t op_arrivals = a.op_img ? 1 : 32;   // one thread announcing a bulk copy, or the warp that built the atom
     for (int i = 0; i < WT2_MAX_STAGES; ++i) {
       ptx::mbar_init(&bars->full[i], 1);
-      ptx::mbar_init(&bars->empty[i], 1);
+      // the export does not write back into the stage: the group that read it hands it back itself
+      ptx::mbar_init(&bars->empty[i], MODE == WT2_PACK ? WT2_GROUP_THREADS : 1);
       ptx::mbar_init(&bars->written[i], WT2_GROUP_THREADS);
     }
-    for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->out_empty[i], 1);
-    for (int i = 0; i < 2; ++i) ptx::mbar_init(&bars->prep_full[i], a.op_img ? 1 : WT2_GROUP_THREADS);
+    for (int i = 0; i < 3; ++i) ptx::mbar_init(&bars->out_empty[i], 1);
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&bars->afull[i], op_arrivals);
+      ptx::mbar_init(&bars->aempty[i], 1);
+    }
+    for (int i = 0; i < WT2_MAX_BSLOTS; ++i) {
+      ptx::mbar_init(&bars->bfull[i], op_arrivals);
+      ptx::mbar_init(&bars->bempty[i], 1);
+    }
     for (int i = 0; i < WT2_ACC; ++i) {
       ptx::mbar_init(&bars->tmem_full[i], 1);
       ptx::mbar_init(&bars->tmem_empty[i], WT2_GROUP_THREADS);
@@ -273,7 +471,6 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     ptx::fence_mbar_init();
     ptx::prefetch_tmap(&tmap_w0);
     ptx::prefetch_tmap(&tmap_out0);
-    if (MODE == WT2_DEQUANT_F) ptx::prefetch_tmap(&tmap_out1);
     if (a.sb_box) { ptx::prefetch_tmap(&tmap_s); ptx::prefetch_tmap(&tmap_b); }
   }
   if (warp == 1) {
@@ -312,34 +509,12 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
   } else if (warp == 1) {
     // ------------------------------ merge MMAs --------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_tf32(WT2_ROWS, WT2_COLS);
-      const int r = p.rank, ksteps = r >> 3;
-      int acc = 0; uint32_t acc_phase = 0;
-      int buf = 0; uint32_t buf_phase = 0;
-      for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next()) {
-        const uint32_t acat_a = ptx::smem_u32(op_base) + (uint32_t)buf * 2 * op_half, bcat_a = acat_a + op_half;
-        bounded_wait(&bars->prep_full[buf], buf_phase, bars);
-        bounded_wait(&bars->tmem_empty[acc], acc_phase ^ 1, bars);
-        if (bars->abort) break;
-        ptx::tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * WT2_COLS);
-        uint32_t accumulate = 0;
-        // B A = Bhi Ahi + Bhi Alo + Blo Ahi  (the tail x tail product is below fp32 resolution of the sum)
-#pragma unroll 1
-        for (int term = 0; term < 3; ++term) {
-          const int eb0 = (term == 2) ? r : 0;       // element offset into the B rows (M operand)
-          const int ea0 = (term == 1) ? r : 0;       // element offset into the A rows (N operand)
-          for (int ks = 0; ks < ksteps; ++ks) {
-            const int eb = eb0 + ks * 8, ea = ea0 + ks * 8;
-            const uint64_t dm = ptx::make_smem_desc_sw128(bcat_a + (eb >> 5) * WT2_ATOM_BYTES + (eb & 31) * 4, 16, 1024);
-            const uint64_t dn = ptx::make_smem_desc_sw128(acat_a + (ea >> 5) * WT2_ATOM_BYTES + (ea & 31) * 4, 16, 1024);
-            ptx::mma_tf32_ss(d_tmem, dm, dn, idesc, accumulate);
-            accumulate = 1;
-          }
-        }
-        ptx::mma_commit(&bars->tmem_full[acc]);
-        if (++acc == WT2_ACC) { acc = 0; acc_phase ^= 1; }
-        if (++buf == a.n_opbuf) { buf = 0; buf_phase ^= 1; }
+      switch (p.rank) {
+        case 8: wtile_mma_role<8>(a, bars, tmem_base, ptx::smem_u32(acat_base), ptx::smem_u32(bslot_base)); break;
+        case 16: wtile_mma_role<16>(a, bars, tmem_base, ptx::smem_u32(acat_base), ptx::smem_u32(bslot_base)); break;
+        case 32: wtile_mma_role<32>(a, bars, tmem_base, ptx::smem_u32(acat_base), ptx::smem_u32(bslot_base)); break;
+        case 64: wtile_mma_role<64>(a, bars, tmem_base, ptx::smem_u32(acat_base), ptx::smem_u32(bslot_base)); break;
+        default: wtile_mma_role<0>(a, bars, tmem_base, ptx::smem_u32(acat_base), ptx::smem_u32(bslot_base)); break;
       }
     }
     __syncwarp();
@@ -359,88 +534,82 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
           ptx::tma_store_2d(&tmap_out0, src, n0, m0);
           if (second_box) ptx::tma_store_2d(&tmap_out0, src + WT2_STAGE_BYTES / 2, n0 + 64, m0);
         }
-        if constexpr (MODE == WT2_DEQUANT_F) {
-          // the staging buffer is the tile's block of the factor array as it stands: one contiguous copy
-          ptx::bulk_store(a.F + ((size_t)cur.tm * a.tiles_n + cur.tn) * FACTOR_TILE_ELEMS, src1, WT2_STAGE_BYTES);
-        }
         if constexpr (MODE == WT2_PACK) ptx::tma_store_2d(&tmap_out0, src1, (n0 * p.bits) >> 5, m0);
         ptx::bulk_commit_group();
+        // hand the buffers back as soon as the copies have read them: a stage that is released a tile later is a
+        // load that starts a tile later
         ptx::bulk_wait_group_read0();
-        ptx::mbar_arrive(&bars->empty[stage]);
-        if constexpr (HAS_OUT1) {
-          ptx::mbar_arrive(&bars->out_empty[ob]);
-          if (++ob == a.n_out) ob = 0;
-        }
+        if constexpr (MODE != WT2_PACK) ptx::mbar_arrive(&bars->empty[stage]);
+        if constexpr (HAS_OUT1) ptx::mbar_arrive(&bars->out_empty[ob]);
+        if constexpr (HAS_OUT1) { if (++ob == a.n_out) ob = 0; }
         if (++stage == a.n_stages) { stage = 0; phase ^= 1; }
       }
       ptx::bulk_wait_group0();
     }
     __syncwarp();
   } else if (warp == 3) {
-    // ------------------------------ MMA operands from the ready-made images ----
-    if (lane == 0 && a.op_img) {
-      const int L = a.n_opbuf;
-      int j = 0;
-      for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next(), ++j) {
-        const int buf = j & (L - 1);
-        if (j >= L) {      // the MMAs of tile j - L, the last readers of this buffer, have completed
-          bounded_wait(&bars->tmem_full[(j - L) & 3], (uint32_t)(((j - L) >> 2) & 1), bars);
+    // ------------------------------ MMA operands ------------------------------
+    // With ready-made images one thread issues bulk copies; without, the warp builds each atom from A and B.
+    const bool img = a.op_img != nullptr;
+    if (img ? lane == 0 : true) {
+      if (img) ptx::griddep_wait();                  // k_split_operands has written the images
+      int slot = 0; uint32_t slot_phase = 0;
+      int panel = -1, pseq = -1;
+      const int ashift = a.n_abuf - 1;
+      for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next()) {
+        if (cur.tn != panel) {
+          panel = cur.tn; ++pseq;
+          const int ab = pseq & ashift, use = pseq >> ashift;     // earlier fills of this buffer
+          if (use >= 1) bounded_wait(&bars->aempty[ab], (uint32_t)((use - 1) & 1), bars);
           if (bars->abort) break;
+          uint8_t* acat = acat_base + (size_t)ab * a_img_bytes;
+          if (img) {
+            ptx::mbar_arrive_expect_tx(&bars->afull[ab], a_img_bytes);
+            ptx::bulk_load(acat, a.op_img + (size_t)cur.tn * a_img_bytes, a_img_bytes, &bars->afull[ab]);
+          } else {
+            for (int c = 0; c < a.atoms; ++c) build_atom_a(a, cur.n0(), c, acat + (size_t)c * WT2_ATOM_BYTES, lane, 32);
+            ptx::fence_proxy_async_smem();
+            ptx::mbar_arrive(&bars->afull[ab]);
+          }
         }
-        uint8_t* acat = op_base + (size_t)buf * 2 * op_half;
-        ptx::mbar_arrive_expect_tx(&bars->prep_full[buf], 2 * op_half);
-        ptx::bulk_load(acat, a.op_img + (size_t)cur.tn * op_half, op_half, &bars->prep_full[buf]);
-        ptx::bulk_load(acat + op_half, a.op_img + (size_t)(a.tiles_n + cur.tm) * op_half, op_half,
-                       &bars->prep_full[buf]);
+        for (int c = 0; c < a.atoms; ++c) {
+          bounded_wait(&bars->bempty[slot], slot_phase ^ 1, bars);
+          if (bars->abort) break;
+          uint8_t* chunk = bslot_base + (size_t)slot * WT2_ATOM_BYTES;
+          if (img) {
+            ptx::mbar_arrive_expect_tx(&bars->bfull[slot], WT2_ATOM_BYTES);
+            ptx::bulk_load(chunk, a.op_img + ((size_t)(a.tiles_n + cur.tm) * a.atoms + c) * WT2_ATOM_BYTES,
+                           WT2_ATOM_BYTES, &bars->bfull[slot]);
+          } else {
+            build_atom_b(a, cur.m0(), c, chunk, lane, 32);
+            ptx::fence_proxy_async_smem();
+            ptx::mbar_arrive(&bars->bfull[slot]);
+          }
+          if (++slot == a.n_bslot) { slot = 0; slot_phase ^= 1; }
+        }
       }
     }
     __syncwarp();
   } else if (warp >= WT2_FIRST_EPI_WARP) {
     // ------------------------------ epilogue ----------------------------------
-    // Two groups of eight warps; group grp owns the CTA's tiles i = grp, grp + 2, ... (accumulator stage i % 4,
-    // operand buffer i % 2).  A thread is one weight row (TMEM lane) and one 64-column half of its group's
-    // tile.  The groups meet only through the mbarriers.  While a group works on tile i the merge of its tile
-    // i + 2 runs into the group's other accumulator stage, and with four W0 stages two loads are in flight.
+    // Three groups of eight warps; group grp owns the CTA's tiles i = grp, grp + 3, ... (accumulator stage i % 4).
+    // A thread is one weight row (TMEM lane) and one 64-column half of its group's tile.  The groups meet only
+    // through the mbarriers: while one waits for a merge or a tile, the others keep the pipes busy.
     const int quarter = warp & 3;
     const int grp = (warp - WT2_FIRST_EPI_WARP) >> 3;
     const int chalf = ((warp - WT2_FIRST_EPI_WARP) >> 2) & 1;   // column half of the tile
     const int row = quarter * 32 + lane;
-    const int tg = chalf * WT2_ROWS + row;                       // thread index within the group
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const int r = p.rank;
-    const int L = a.n_opbuf;                                    // 1 or 2
-    const int n_items = 32 * r;                                 // (row, 4 ranks) operand items per tile
     const int sbw = 2 * a.ngt;                                  // floats per thread: s x ngt | b x ngt
     float* grp_sb = sb_base + (size_t)grp * 2 * WT2_ROWS * sbw;   // two buffers of [128 rows][s x ngt | b x ngt]
-
-    // ---- MMA operands of tile j (CTA sequence number), built by the group that owns the tile.  With two
-    //      operand buffers the buffer of tile j was last read by the MMAs of tile j - 2, the group's own
-    //      previous tile, which the caller has already seen complete; with one buffer by those of tile j - 1. ----
-    auto prep_buffer_wait = [&](int j) {
-      if (L == 1 && j >= 1) {
-        bounded_wait(&bars->tmem_full[(j - 1) & 3], (uint32_t)(((j - 1) >> 2) & 1), bars);
-        ptx::tc_fence_after_sync();
-      }
-    };
-    auto prep = [&](int j, int m0_, int n0_) {
-      if (a.op_img) return;                                     // warp 3 brings the operands in
-      prep_buffer_wait(j);
-      uint8_t* acat = op_base + (size_t)(j & (L - 1)) * 2 * op_half;
-      for (int idx = tg; idx < n_items; idx += WT2_GROUP_THREADS) {
-        OperandItem it_;
-        operand_item_load(a, m0_, n0_, idx, it_);
-        operand_item_store(a, idx, it_, acat, acat + op_half);
-      }
-      ptx::fence_proxy_async_smem();
-      ptx::mbar_arrive(&bars->prep_full[j & (L - 1)]);
-    };
+    const bool stage_sb_self = !a.fast && !a.sb_box;            // the group copies s and b itself
 
     // ---- s and b of the tile's rows for the quantization groups it intersects: the threads of column half 0
     //      (one per weight row) copy them with asynchronous 4-byte copies into the group's buffer for its next
     //      tile; the group meets at a named barrier when it starts that tile.  (Each row's values sit in a line
     //      of their own, so every copy instruction touches 32 lines: the fewer of them the better.) ----
     auto stage_sb = [&](int m0_, int n0_, int buf) {
-      if (chalf != 0 || a.sb_box) return;
+      if (chalf != 0 || !stage_sb_self) return;
       float* dst = grp_sb + ((size_t)buf * WT2_ROWS + row) * sbw;
       const int o_ = m0_ + row;
       const int gf = group_of(a, n0_);
@@ -455,18 +624,26 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
       ptx::cp_async_commit();
     };
+    // ---- fast path: s and b of this thread's half row of an interior tile, straight from global memory ----
+    auto interior = [&](int m0_, int n0_) { return a.fast && m0_ + WT2_ROWS <= p.d_out && n0_ + WT2_COLS <= p.d_in; };
+    auto fetch_sb = [&](int m0_, int n0_, float& s_out, float& b_out) {
+      if (!interior(m0_, n0_)) return;
+      const size_t idx = (size_t)(m0_ + row) * p.ngroups + group_of(a, n0_ + chalf * 64);
+      s_out = __ldg(a.s + idx); b_out = __ldg(a.b + idx);
+    };
 
     TileCursor cur(a, grp, WT2_GROUPS);
+    float s_next = 1.f, b_next = 0.f;
     if (cur.valid()) {
       stage_sb(cur.m0(), cur.n0(), 0);
-      prep(grp, cur.m0(), cur.n0());
+      fetch_sb(cur.m0(), cur.n0(), s_next, b_next);
     }
     int sb_buf = 0;
     const int qn_bits = kRoundMagicBits + (int)p.qn;
 
-    int stage = grp;                                            // W0 stage of tile i and its phase, kept without divisions
-    uint32_t phase = 0;                                         // (n_stages >= 2 = WT2_GROUPS)
     for (int i = grp; cur.valid(); cur.next(), i += WT2_GROUPS) {
+      const int stage = i % a.n_stages;                         // W0 stage of tile i and its phase
+      const uint32_t phase = (uint32_t)((i / a.n_stages) & 1);
       const int m0 = cur.m0(), n0 = cur.n0();
       const int o = m0 + row;
       const bool row_ok = o < p.d_out;
@@ -474,9 +651,15 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       const int g_first = group_of(a, n0);
       int m1 = 0, n1 = 0;
       const bool has_next = cur.peek(1, m1, n1);
+      const float s_cur = s_next, b_cur = b_next;
+      if (has_next) fetch_sb(m1, n1, s_next, b_next);           // in flight while this tile is worked on
       const float *my_s, *my_b;                                 // s and b of this row, from group sb_first on
       int sb_first;
-      if (a.sb_box) {                                           // they arrive with the W0 tile (full[stage] below)
+      if (a.fast) {                                             // general tiles of a fast launch (edges): global memory
+        my_s = a.s + (size_t)o * p.ngroups;
+        my_b = a.b + (size_t)o * p.ngroups;
+        sb_first = 0;
+      } else if (a.sb_box) {                                    // they arrive with the W0 tile (full[stage] below)
         my_s = sb_base + ((size_t)stage * 2 * WT2_ROWS + row) * a.sb_box;
         my_b = my_s + WT2_ROWS * a.sb_box;
         sb_first = g_first & ~3;
@@ -489,17 +672,38 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
       bounded_wait(&bars->tmem_full[acc], (uint32_t)((i >> 2) & 1), bars);
       ptx::tc_fence_after_sync();
-      // the merge of this tile is complete: the operands of the group's next tile can take its buffer
-      if (has_next) prep(i + WT2_GROUPS, m1, n1);
       bounded_wait(&bars->full[stage], phase, bars);
       int ob = 0;
       if constexpr (HAS_OUT1) {
-        const int uses = a.n_out == 2 ? (i >> 1) : i;           // earlier tiles that went through this buffer
-        ob = a.n_out == 2 ? (i & 1) : 0;
+        const int uses = i / a.n_out;                           // earlier tiles that went through this buffer
+        ob = i - uses * a.n_out;
         if (uses >= 1) bounded_wait(&bars->out_empty[ob], (uint32_t)((uses - 1) & 1), bars);
       }
       uint8_t* tile_rows = stage_base + (size_t)stage * WT2_STAGE_BYTES + row * 128;
-      [[maybe_unused]] uint8_t* out1 = out_base + (size_t)ob * a.out_bytes;
+      // second output: the export's staging rows in shared memory; the STE factors go straight to the tile's block
+      // of the factor array in global memory (16 bytes per thread and piece, a warp's 32 rows contiguous)
+      [[maybe_unused]] uint8_t* out1 =
+          MODE == WT2_DEQUANT_F
+              ? reinterpret_cast<uint8_t*>(a.F + ((size_t)cur.tm * a.tiles_n + cur.tn) * FACTOR_TILE_ELEMS)
+              : out_base + (size_t)ob * a.out_bytes;
+      if (interior(m0, n0)) {
+        // the thread's 64 columns lie in one quantization group
+        FastConsts fc;
+        fc.s = s_cur; fc.b = b_cur; fc.rs = 1.0f / s_cur;
+        fc.qn = p.qn; fc.qp = p.qp; fc.gamma = p.gamma;
+        const uint32_t taddr = tmem_base + lane_base + (uint32_t)(acc * WT2_COLS + chalf * 64);
+        if constexpr (MODE == WT2_PACK) {
+          if (p.bits == 4) wtile_half_row_fast<MODE, 4>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc]);
+          else wtile_half_row_fast<MODE, 3>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc]);
+          const int g = group_of(a, n0 + chalf * 64);
+          if ((n0 + chalf * 64) - g * p.group == 0) {             // first half row of its group
+            a.s16[(size_t)o * p.ngroups + g] = __float2half_rn(fc.s);
+            a.b16[(size_t)o * p.ngroups + g] = __float2half_rn(fc.b);   // Q_N = 0: b + s Q_N = b
+          }
+        } else {
+          wtile_half_row_fast<MODE, 4>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc]);
+        }
+      } else {
       float rs = 1.f, s_ = 1.f, b_ = 0.f;
       int cur_g = -1;
 #pragma unroll 1
@@ -606,12 +810,12 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
           }
         }
       }
+      }
       ptx::fence_proxy_async_smem();                   // the stores above are read by TMA
       ptx::mbar_arrive(&bars->written[stage]);
+      if constexpr (MODE == WT2_PACK) ptx::mbar_arrive(&bars->empty[stage]);   // W0 has been read
       sb_buf ^= 1;
       if (has_next) stage_sb(m1, n1, sb_buf);          // the other buffer: its readers passed this tile's barrier
-      stage += WT2_GROUPS;
-      if (stage >= a.n_stages) { stage -= a.n_stages; phase ^= 1; }
     }
   }
 
@@ -647,35 +851,52 @@ inline bool make_tmap_words(CUtensorMap* m, const void* base, uint64_t rows, uin
 
 // Shared-memory plan.  A tile being worked on holds one W0 stage and, when there is a second output, one
 // staging buffer for it: two of each keep both epilogue groups busy, further stages let the loads run ahead.
-// Candidates in order of preference (a single operand buffer makes every merge wait for the previous one).
+// The operands of the merge take one or two A-image buffers and a ring of 16 KB chunks of B images.  Of the
+// combinations that fit, the best by this order of concerns is taken: at least 3 stages; two staging buffers;
+// a ring that holds more than one tile's chunks; at least 4 stages; two A buffers; a ring of two tiles; 5 stages.
 // `sb_by_tma`: s and b may come in by TMA (the caller has checked their alignment); the shape must allow it too.
 inline bool wtile_plan(WtileArgs& a, int mode, bool sb_by_tma = true) {
   const Params& p = a.p;
   a.atoms = (2 * p.rank + 31) / 32;
   a.ngt = std::min(p.ngroups, (WT2_COLS - 1) / p.group + 2);
-  // a box starts at a group column that is a multiple of 4 (16 bytes) at or below the tile's first group, so it
-  // is up to 3 groups wider than the tile; the row pitch of s and b must be a multiple of 16 bytes
-  const int box = (a.ngt + 3 + 3) / 4 * 4;
-  a.sb_box = (sb_by_tma && p.ngroups % 4 == 0 && p.ngroups >= box && box <= 256) ? box : 0;
   a.group_shift = -1;
   for (int sh = 3; sh < 31; ++sh)
     if ((1 << sh) == p.group) a.group_shift = sh;
-  a.out_bytes = mode == WT2_DEQUANT_F ? WT2_STAGE_BYTES : mode == WT2_PACK ? WT2_ROWS * (WT2_COLS * p.bits / 8) : 0;
-  struct Cand { int opbuf, n_out, stages; };
-  static const Cand plain[] = {{2, 0, 4}, {1, 0, 4}, {2, 0, 3}, {1, 0, 3}, {2, 0, 2}, {1, 0, 2}};
-  static const Cand small_out[] = {{2, 2, 4}, {1, 2, 4}, {2, 2, 3},
-                                   {1, 2, 3}, {2, 2, 2}, {1, 2, 2}, {1, 1, 2}};
-  static const Cand big_out[] = {{2, 2, 3}, {1, 2, 3}, {2, 2, 2}, {1, 2, 2}, {2, 1, 3}, {1, 1, 3},
-                                 {2, 1, 2}, {1, 1, 2}};
-  const Cand* cands = mode == WT2_DEQUANT ? plain : mode == WT2_PACK ? small_out : big_out;
-  const int n_cands = mode == WT2_DEQUANT ? 6 : mode == WT2_PACK ? 7 : 8;
-  const int max_opbuf = p.rank <= 32 ? 2 : 1;       // rank 64: the split operands of one tile are already 128 KB
-  for (int c = 0; c < n_cands; ++c) {
-    if (cands[c].opbuf > max_opbuf) continue;
-    a.n_opbuf = cands[c].opbuf; a.n_out = cands[c].n_out; a.n_stages = cands[c].stages;
-    if (wtile_smem_bytes(a) <= 227 * 1024) return true;
-  }
-  return false;
+  // (the export's fast path builds its code words from the raw rounding results, which it does for the unsigned grid)
+  a.fast = (p.group % 64 == 0 && (mode != WT2_PACK || (p.qn == 0.f && (p.bits == 3 || p.bits == 4)))) ? 1 : 0;
+  // a box starts at a group column that is a multiple of 4 (16 bytes) at or below the tile's first group, so it
+  // is up to 3 groups wider than the tile; the row pitch of s and b must be a multiple of 16 bytes
+  const int box = (a.ngt + 3 + 3) / 4 * 4;
+  a.sb_box = (!a.fast && sb_by_tma && p.ngroups % 4 == 0 && p.ngroups >= box && box <= 256) ? box : 0;
+  a.out_bytes = mode == WT2_PACK ? WT2_ROWS * (WT2_COLS * p.bits / 8) : 0;
+  const bool has_out = mode == WT2_PACK;
+  long best = -1;
+  WtileArgs pick = a;
+  const int ring_opts[4] = {2 * a.atoms, a.atoms + 1, 3, 2};
+  for (int stages = 2; stages <= WT2_MAX_STAGES; ++stages)
+    for (int n_out = has_out ? 1 : 0; n_out <= (has_out ? WT2_GROUPS : 0); ++n_out)
+      for (int n_abuf = 1; n_abuf <= 2; ++n_abuf)
+        for (int ro = 0; ro < 4; ++ro) {
+          const int ring = ring_opts[ro];
+          if (ring < 2 || ring > WT2_MAX_BSLOTS) continue;
+          WtileArgs c = a;
+          c.n_stages = stages; c.n_out = n_out; c.n_abuf = n_abuf; c.n_bslot = ring;
+          if (wtile_smem_bytes(c) > 227 * 1024) continue;
+          long score = 0;
+          score = score * 2 + (stages >= 3);
+          score = score * 2 + (!has_out || n_out >= 2);
+          score = score * 2 + (ring > a.atoms);
+          score = score * 2 + (stages >= 4);
+          score = score * 2 + (n_abuf == 2);
+          score = score * 2 + (ring >= 2 * a.atoms);
+          score = score * 2 + (stages >= 5);
+          score = score * 2 + (!has_out || n_out >= WT2_GROUPS);
+          score = score * 16 + ring;                 // then the deeper ring
+          if (score > best) { best = score; pick = c; }
+        }
+  if (best < 0) return false;
+  a = pick;
+  return true;
 }
 
 // Whether the tensor-core weight-tile kernel covers this problem (otherwise the plain-ALU kernel runs).
@@ -688,7 +909,7 @@ inline bool wtile_tc_supported(const Params& p, int mode) {
   }
   WtileArgs a{};
   a.p = p;
-  return wtile_plan(a, mode);                       // the shared-memory plan must fit (rank 64 with the factor output does not)
+  return wtile_plan(a, mode);                       // the shared-memory plan must fit
 }
 
 // mode WT2_DEQUANT: out0 = W_q.  WT2_DEQUANT_F: out0 = W_q, out1 = STE factors.  WT2_PACK: out0 = codes.
@@ -699,8 +920,8 @@ inline size_t wtile_image_bytes(const Params& p) {
 }
 
 // `op_img` (optional, wtile_image_bytes(p) bytes of device scratch, 16-byte aligned): with it the MMA operands are
-// split once by a launch of k_split_operands and reach the tiles by bulk copies; without it the epilogue warps
-// build them tile by tile.  `zero` (optional): buffers that launch also clears; *zeroed is set when it did.
+// split once by a launch of k_split_operands and reach the tiles by bulk copies; without it one warp of every CTA
+// builds them tile by tile (slower).  `zero` (optional): buffers that launch also clears; *zeroed is set when it did.
 inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, const float* A, const float* B,
                                   const float* s, const float* b, void* out0, void* out1, __half* s16, __half* b16,
                                   cudaStream_t st, void* op_img = nullptr, const ZeroList* zero = nullptr,
@@ -726,8 +947,18 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
     if (!make_tmap_words(&t_s, s, p.d_out, p.ngroups, a.sb_box) || !make_tmap_words(&t_b, b, p.d_out, p.ngroups, a.sb_box))
       return L4Q_ERR_CUDA;
   }
-  const size_t smem = wtile_smem_bytes(a);
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
+#ifdef L4Q_EXPERIMENT
+  if (const char* e = getenv("L4Q_WT_STAGES")) a.n_stages = std::min(a.n_stages, atoi(e));
+  if (const char* e = getenv("L4Q_WT_OPS")) {     // "abuf,ring,stages"
+    int x = 0, y = 0, z = 0;
+    if (sscanf(e, "%d,%d,%d", &x, &y, &z) == 3) {
+      WtileArgs c = a; c.n_abuf = x; c.n_bslot = y; c.n_stages = z;
+      if (wtile_smem_bytes(c) <= 227 * 1024) a = c;
+    }
+  }
+#endif
+  const size_t smem = wtile_smem_bytes(a);
   if (op_img) {
     ZeroList zl{};
     if (zero) zl = *zero;
@@ -739,7 +970,17 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   auto launch = [&](auto kern) -> l4q_status {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return L4Q_ERR_CUDA;
-    kern<<<grid, WT2_THREADS, smem, st>>>(t_w0, t_o0, t_o1, t_s, t_b, a);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(WT2_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = op_img ? 1 : 0;                  // overlap with the operand split that was just launched
+    if (cudaLaunchKernelEx(&cfg, kern, t_w0, t_o0, t_o1, t_s, t_b, a) != cudaSuccess) {
+      cudaGetLastError();
+      return L4Q_ERR_CUDA;
+    }
     return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
   };
   switch (mode) {
