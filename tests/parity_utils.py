@@ -1,6 +1,6 @@
 """Comparison helpers shared by the GPU parity tests (tolerances in one place).
 
-Tolerances (stated by the task's parity bar):
+Tolerances:
   * integer codes: bit-exact, except where the fp64 grid coordinate w lies
     within 1e-6 * max(1, |w|) of a rounding boundary k + 1/2; the number of such
     mismatches must not exceed 1e-6 of all elements; any other mismatch fails;

@@ -7,20 +7,24 @@ synchronisation.  For them the library carries a fixed 32 MiB scratch array and 
 entry point that takes no workspace.  This test calls that entry point through
 the C ABI and requires its output to equal l4q_linear_fwd's (same kernels, same
 arithmetic, so the comparison is exact, well inside the 2e-2 / 1e-4 parity
-tolerances), on two calls in a row that share the array: the second call uses a
+tolerances) and to agree with the fp64 oracle within the bf16 forward tolerance,
+on two calls in a row that share the array: the second call uses a
 smaller, different layer, so anything it read from the first call's leftovers
 would show.  Collected last on purpose (file name), and self-contained so that it
 passes alone in a fresh process as well as after the other tests.
 """
 import gc
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import l4q_oracle as orc
 from paper_2402_04902_b200 import binding as l4q
 from paper_2402_04902_b200 import synth
 
 import gpu_harness as gh
+import parity_utils as pu
 
 pytestmark = pytest.mark.gpu
 
@@ -46,6 +50,30 @@ def _run_both(cfg, seed):
     return y_ws, y_static
 
 
+def _check_against_oracle(cfg, seed, y_static):
+    """The entry point's own output against the fp64 oracle (Eq. 7-10, bf16 reference mode), not only against
+    the other entry point: the same tolerance as every bf16 forward check, 2e-2.  The oracle takes its own
+    codes except where the export of the same layer holds the other neighbour of a verified in-band tie."""
+    arrays = synth.make_layer_inputs(cfg, seed=seed)
+    spec = pu.spec_of(cfg)
+    a = pu.widen(arrays)
+    d = l4q.to_device(cfg, arrays)
+    pk = l4q.alloc_pack_outputs(cfg)
+    l4q.l4q_pack_int(l4q.make_desc(cfg), d["W0"], d["A"], d["B"], d["s"], d["b"], pk["codes"], pk["s16"], pk["b16"])
+    l4q.l4q_check()
+    qn, _ = orc.grid_bounds(spec)
+    w = orc.prequant(spec, orc.merge(spec, a["W0"], a["A"], a["B"]), a["s"], a["b"])
+    got_u = orc.unpack_int(spec, pk["codes"].cpu().numpy().view(np.uint32), cfg.d_in)
+    res = pu.check_codes(got_u, spec, w)
+    assert res["out_of_band"] == 0 and res["mismatches"] <= max(1.0, res["allowed"]), res
+    codes = orc.quant_codes(spec, w)
+    tie = (got_u + qn) != codes
+    codes[tie] = (got_u + qn)[tie]
+    Y = orc.forward(spec, a["X"], a["W0"], a["A"], a["B"], a["s"], a["b"], bf16_reference=True, codes=codes)
+    err = pu.max_rel_err(y_static.double().cpu().numpy(), Y)
+    assert err <= pu.TOL_OUT["bf16"], (cfg.name, err)
+
+
 def test_static_forward_matches_workspace_forward_on_two_calls_in_a_row():
     gh.ensure_built()
     first = synth.LayerConfig("static_bf16_a", tokens=384, d_in=1024, d_out=768, rank=16, alpha=32.0, bits=4,
@@ -55,6 +83,7 @@ def test_static_forward_matches_workspace_forward_on_two_calls_in_a_row():
     for cfg, seed in ((first, 31), (second, 32)):
         y_ws, y_static = _run_both(cfg, seed)
         assert torch.equal(y_ws, y_static), cfg.name
+        _check_against_oracle(cfg, seed, y_static)
     # the fp32 validation path shares the same array
     y_ws, y_static = _run_both(synth.CONFIG1, 33)
     assert torch.equal(y_ws, y_static)
