@@ -256,6 +256,15 @@ l4q_status l4q_linear_fwd_static(const l4q_desc* desc, const void* X, const void
  * library works as before.  No counterpart in the paper.  Returns L4Q_OK if the launch succeeded. */
 l4q_status l4q_selftest_timeout(void* cuda_stream);
 
+/* Measurement helper, no counterpart in the paper: moves a dense row-major bf16 matrix `src` [rows, cols]
+ * (device pointer, 16-byte aligned, cols a multiple of 8) through shared memory in 128 x 128 tiles with the same
+ * TMA loads -- and, if `dst` (same shape, may not overlap src) is not NULL, the same TMA stores -- as the
+ * merge + fake-quantize kernel, and does nothing else.  Its device time (l4q_profile_read, L4Q_KERNEL_TILE_COPY)
+ * is the floor the memory system sets for a kernel that reads one weight (dst NULL: the export) or reads and
+ * rewrites it (the dequantize step) in one launch of that size; bench.py reports the weight-tile kernels against
+ * it.  Asynchronous on `cuda_stream`; L4Q_ERR_INVALID_ARG on a bad shape or pointer. */
+l4q_status l4q_selftest_tile_copy(const void* src, void* dst, int64_t rows, int64_t cols, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the device status word
  * (L4Q_OK, or L4Q_ERR_TIMEOUT if a kernel gave up on a bounded wait), or
  * L4Q_ERR_CUDA if the stream reported an error. */
@@ -285,7 +294,8 @@ enum {
   L4Q_KERNEL_INFER = 9,       /* Y = X W_q^T from the packed export (App. F)                */
   L4Q_KERNEL_ADAMW = 10,      /* AdamW update of one parameter tensor (App. D)              */
   L4Q_KERNEL_LORA_SIDE = 11,  /* rank-side products of the LoRA / QAT-LoRA layers (Eq. 1-2) */
-  L4Q_KERNEL_COUNT = 12
+  L4Q_KERNEL_TILE_COPY = 12,  /* l4q_selftest_tile_copy (measurement helper)                */
+  L4Q_KERNEL_COUNT = 13
 };
 l4q_status l4q_profile_enable(int enable);
 l4q_status l4q_profile_read(int kernel, uint64_t* launches, double* total_ms);

@@ -29,6 +29,7 @@ EXPORTED_SYMBOLS = (
     "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
     "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error", "l4q_linear_infer", "l4q_adamw_step",
     "l4q_lora_workspace_bytes", "l4q_lora_linear_fwd", "l4q_lora_linear_bwd", "l4q_selftest_timeout",
+    "l4q_selftest_tile_copy",
 )
 L4Q_LORA_PLAIN, L4Q_LORA_QAT = 1, 2
 LORA_KINDS = {"lora": L4Q_LORA_PLAIN, "qat_lora": L4Q_LORA_QAT}
@@ -37,7 +38,7 @@ INIT_METHODS = {"lsq+": 0, "symm": 1, "asymm": 2, "l4q": 3}
 L4Q_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 KERNEL_IDS = {"dequant": 0, "pack": 1, "gemm_fwd": 2, "gemm_dgrad": 3, "gemm_wgrad": 4, "val_gemm": 5,
-              "val_wgrad": 6, "init": 7, "error": 8, "infer": 9, "adamw": 10, "lora_side": 11}
+              "val_wgrad": 6, "init": 7, "error": 8, "infer": 9, "adamw": 10, "lora_side": 11, "tile_copy": 12}
 
 
 class L4QDesc(ctypes.Structure):
@@ -98,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.l4q_quant_error.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp]
         L.l4q_selftest_timeout.restype = ctypes.c_int
         L.l4q_selftest_timeout.argtypes = [vp]
+        L.l4q_selftest_tile_copy.restype = ctypes.c_int
+        L.l4q_selftest_tile_copy.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
         L.l4q_check.restype = ctypes.c_int
         L.l4q_check.argtypes = [vp]
         L.l4q_launch_count.restype = ctypes.c_uint64
@@ -244,6 +247,15 @@ def l4q_quant_error(desc: L4QDesc, W0, A, B, s, b, errors, stream=None) -> None:
 def l4q_selftest_timeout(stream=None) -> None:
     """Make one bounded device-side wait expire (about a millisecond); the next l4q_check raises L4Q_ERR_TIMEOUT."""
     _raise(lib().l4q_selftest_timeout(_stream(stream)), "l4q_selftest_timeout")
+
+
+def l4q_selftest_tile_copy(src, dst=None, stream=None) -> None:
+    """Move the bf16 matrix `src` through shared memory in 128 x 128 tiles by TMA (and store it to `dst` if given):
+    the memory-system floor of the weight-tile kernels on that size.  Timed by the library's per-launch events."""
+    if src.dtype != torch.bfloat16 or src.dim() != 2 or (dst is not None and (dst.dtype != src.dtype or dst.shape != src.shape)):
+        raise ValueError("src (and dst) must be 2-D bf16 CUDA tensors of the same shape")
+    _raise(lib().l4q_selftest_tile_copy(_ptr(src), _ptr(dst), src.shape[0], src.shape[1], _stream(stream)),
+           "l4q_selftest_tile_copy")
 
 
 def l4q_check(stream=None) -> None:

@@ -15,6 +15,7 @@
 #include "l4q_wtile.cuh"
 #include "l4q_infer.cuh"
 #include "l4q_variants.cuh"
+#include "l4q_tilecopy.cuh"
 
 using namespace l4q;
 
@@ -616,6 +617,14 @@ l4q_status l4q_selftest_timeout(void* cuda_stream) {
   return launch_status();
 }
 
+l4q_status l4q_selftest_tile_copy(const void* src, void* dst, int64_t rows, int64_t cols, void* cuda_stream) {
+  if (!src || rows <= 0 || cols <= 0 || rows > (1 << 30) || cols > (1 << 30) || cols % 8 != 0) return L4Q_ERR_INVALID_ARG;
+  if (!aligned16(src) || !aligned16(dst)) return L4Q_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  KernelScope ks(L4Q_KERNEL_TILE_COPY, stream);
+  return launch_tile_copy(src, dst, (int)rows, (int)cols, stream);
+}
+
 l4q_status l4q_check(void* cuda_stream) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (cudaStreamSynchronize(stream) != cudaSuccess) return L4Q_ERR_CUDA;
@@ -674,6 +683,7 @@ const char* l4q_kernel_name(int kernel) {
     case L4Q_KERNEL_INFER: return "k_infer_bf16";
     case L4Q_KERNEL_ADAMW: return "k_adamw";
     case L4Q_KERNEL_LORA_SIDE: return "k_gemm_bf16<rank side> / k_lora_cast";
+    case L4Q_KERNEL_TILE_COPY: return "k_tile_copy";
     default: return "unknown kernel";
   }
 }
