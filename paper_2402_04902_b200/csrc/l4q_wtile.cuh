@@ -19,7 +19,7 @@
 //     column-panel-major tile sequence, so the A image of its column panel stays resident (reloaded at a panel
 //     change) and only the B image of the tile's row panel streams in, 16 KB (one swizzle atom of K) at a
 //     time through a ring of chunks, each released by the MMAs that read it;
-//   * 24 epilogue warps in three groups of eight; a group owns every third tile of the CTA (accumulator stage
+//   * 16 epilogue warps in two groups of eight; a group owns every second tile of the CTA (accumulator stage
 //     tile % 4), a thread one weight row and one 64-column half of the group's tile.  It reads the
 //     merge from tensor memory with tcgen05.ld, the W0 tile from shared memory in 16-byte pieces, and does
 //     the quantizer arithmetic.  Interior tiles whose half rows lie in one quantization
@@ -27,9 +27,9 @@
 //     global memory, one pair per thread and tile, fetched a tile ahead); every other tile takes the
 //     general loop.
 //
-// Roles (896 threads): warp 0 = TMA loads (W0; s, b boxes where used), warp 1 = MMA issuer + TMEM owner,
-// warp 2 = TMA stores, warp 3 = operand loader (one thread issuing bulk copies of the ready-made images, or,
-// without images, the whole warp building the operands from A and B), warps 4..27 = epilogue (warp w: TMEM
+// Roles (672 threads): warp 0 = TMA loads (W0; s, b boxes where used), warp 1 = MMA issuer + TMEM owner,
+// warps 2 and 20 = TMA stores (one thread each, alternate tiles), warp 3 = operand loader (one thread issuing bulk copies of the ready-made images, or,
+// without images, the whole warp building the operands from A and B), warps 4..19 = epilogue (warp w: TMEM
 // lane quarter w % 4, group (w - 4) / 8, column half ((w - 4) / 4) % 2).
 // Every mbarrier wait is bounded (see bounded_wait); there is no block-level barrier after set-up.
 #pragma once
@@ -44,10 +44,13 @@ constexpr int WT2_ROWS = 128, WT2_COLS = 128;
 #ifndef WT2_NGROUPS
 #define WT2_NGROUPS 2
 #endif
-constexpr int WT2_THREADS = 128 + 256 * WT2_NGROUPS;
+constexpr int WT2_THREADS = 128 + 256 * WT2_NGROUPS + 32;   // four role warps, the epilogue groups, the second store warp
 constexpr int WT2_FIRST_EPI_WARP = 4;
+constexpr int WT2_SECOND_STORE_WARP = WT2_FIRST_EPI_WARP + 8 * WT2_NGROUPS;
+constexpr int WT2_BUILDERS = 32;                    // threads that build the merge operands where no images are given: warp 3
+                                                    // (four warps were measured too: still far slower than ready-made images)
 constexpr int WT2_EPI_THREADS = 256 * WT2_NGROUPS;
-constexpr int WT2_GROUPS = WT2_NGROUPS;                       // epilogue warp groups; each owns every third tile of the CTA
+constexpr int WT2_GROUPS = WT2_NGROUPS;                       // epilogue warp groups; group g owns tiles g, g + WT2_GROUPS, ... of the CTA
 constexpr int WT2_GROUP_THREADS = WT2_EPI_THREADS / WT2_GROUPS;
 constexpr int WT2_ACC = 4;                          // accumulator stages of 128 TMEM columns
 constexpr int WT2_STAGE_BYTES = WT2_ROWS * WT2_COLS * 2;   // one bf16 tile: two 128 x 64 swizzled boxes
@@ -58,15 +61,20 @@ constexpr int WT2_MAX_ATOMS = 4;                    // rank <= 64
 
 enum { WT2_DEQUANT = 0, WT2_DEQUANT_F = 1, WT2_PACK = 2 };
 
+// Output buffers of the caller that must start from zero (they are accumulated into with atomics later on the
+// stream): cleared by a launch that runs anyway, which saves one memset launch per buffer.
+struct ZeroList { float* ptr[4]; size_t n[4]; };
+
 struct WtileArgs {
   Params p;
   const float *A, *B, *s, *b;
   __half *s16, *b16;       // WT2_PACK
   __half* F;               // WT2_DEQUANT_F: the factor array (factor_index layout)
+  ZeroList zero;           // buffers this launch clears before anything else (all sizes 0: none)
   const uint8_t* op_img;   // optional: the split MMA operands of every panel, ready made (see k_split_operands)
   int tiles_m, tiles_n;
   int n_stages;            // W0 stages in shared memory (2..5)
-  int n_out;               // staging buffers for the code words of the export: 0 (other modes) .. 3
+  int n_out;               // staging buffers for the code words of the export: one per epilogue group (0 in other modes)
   int out_bytes;           // bytes of one such buffer
   int atoms;               // swizzle atoms per operand row: ceil(2 rank / 32)
   int ngt;                 // upper bound of the quantization groups a 128-column tile intersects
@@ -87,7 +95,7 @@ struct __align__(8) WtileBarriers {
   uint64_t full[WT2_MAX_STAGES];      // W0 tile has landed in the stage
   uint64_t empty[WT2_MAX_STAGES];     // the stage may be overwritten (its store has read it)
   uint64_t written[WT2_MAX_STAGES];   // the epilogue has written the stage's outputs
-  uint64_t out_empty[3];              // staging buffer of the code words may be overwritten
+  uint64_t out_empty[WT2_GROUPS];     // staging buffer of the code words may be overwritten
   uint64_t afull[2], aempty[2];       // A image of a column panel: complete in buffer b / no longer read by any MMA
   uint64_t bfull[WT2_MAX_BSLOTS], bempty[WT2_MAX_BSLOTS];   // one chunk of a B image, likewise
   uint64_t tmem_full[WT2_ACC], tmem_empty[WT2_ACC];
@@ -141,6 +149,21 @@ struct TileCursor {
   }
 };
 
+// The W0 stages (and, in the export, the staging buffers of the code words) are owned by the epilogue groups:
+// group g works through stages g, g + G, g + 2 G, ... of the n_stages, round after round.  Every barrier of a
+// stage then has one waiting thread per side, which sees its phases strictly in order -- a barrier that two
+// threads waited on in turn, a whole round of stages apart, could be taken for complete one phase early by the
+// parity test whenever the groups had drifted three tiles apart.
+struct StageSeq {
+  int g, n_own, slot, round;
+  __device__ StageSeq(int group, int n_stages) : g(group), slot(0), round(0) {
+    n_own = (n_stages - group + WT2_GROUPS - 1) / WT2_GROUPS;          // stages g, g + G, ... below n_stages
+  }
+  __device__ int stage() const { return g + WT2_GROUPS * slot; }
+  __device__ uint32_t parity() const { return (uint32_t)(round & 1); }
+  __device__ void advance() { if (++slot == n_own) { slot = 0; ++round; } }
+};
+
 // x = hi + lo with hi, lo representable in tf32 (low 13 mantissa bits clear): hi keeps the leading 10
 // mantissa bits of x (truncation), lo the leading bits of the exact remainder.  Plain logic ops.
 __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
@@ -154,68 +177,98 @@ __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
 // Atom c holds values 32 c .. 32 c + 31 of that concatenation (beyond 2 r: zero).  A work item is one 16-byte
 // piece (4 values) of one row: item it -> row it % 128, piece it / 128, so that a warp reads 32 consecutive
 // columns of A (coalesced) or 32 rows of B.  `dst`: the atom, in shared or global memory.
-__device__ __forceinline__ void build_atom_a(const WtileArgs& a, int n0, int c, uint8_t* dst, int tid, int nthreads) {
+// NT threads take 1024 / NT items each, in batches of up to 8 whose loads are all issued before the first is used.
+template <int NT>
+__device__ __forceinline__ void build_atom_a(const WtileArgs& a, int n0, int c, uint8_t* dst, int tid) {
   const Params& p = a.p;
-  for (int it = tid; it < 1024; it += nthreads) {
-    const int row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j, col = n0 + row;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (e0 < 2 * p.rank && col < p.d_in) {
-      const bool tail = e0 >= p.rank;
-      const int k = tail ? e0 - p.rank : e0;
-      float x[4], h[4], l[4];
+  constexpr int PER = 1024 / NT, BATCH = PER < 8 ? PER : 8;
+#pragma unroll 1
+  for (int u0 = 0; u0 < PER; u0 += BATCH) {
+    float x[BATCH][4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        x[e] = __ldg(a.A + (size_t)(k + e) * p.d_in + col);
-        split_tf32(x[e], h[e], l[e]);
-      }
-      v = tail ? make_float4(l[0], l[1], l[2], l[3]) : make_float4(h[0], h[1], h[2], h[3]);
+    for (int u = 0; u < BATCH; ++u) {
+      const int it = tid + (u0 + u) * NT, row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j, col = n0 + row;
+      const int k = e0 >= p.rank ? e0 - p.rank : e0;
+      const bool ok = e0 < 2 * p.rank && col < p.d_in;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) x[u][e] = ok ? __ldg(a.A + (size_t)(k + e) * p.d_in + col) : 0.f;
     }
-    *reinterpret_cast<float4*>(dst + row * 128 + ((j ^ (row & 7)) << 4)) = v;
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int it = tid + (u0 + u) * NT, row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j;
+      const bool tail = e0 >= p.rank;
+      float h[4], l[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) split_tf32(x[u][e], h[e], l[e]);
+      *reinterpret_cast<float4*>(dst + row * 128 + ((j ^ (row & 7)) << 4)) =
+          tail ? make_float4(l[0], l[1], l[2], l[3]) : make_float4(h[0], h[1], h[2], h[3]);
+    }
   }
 }
 
-__device__ __forceinline__ void build_atom_b(const WtileArgs& a, int m0, int c, uint8_t* dst, int tid, int nthreads) {
+template <int NT>
+__device__ __forceinline__ void build_atom_b(const WtileArgs& a, int m0, int c, uint8_t* dst, int tid) {
   const Params& p = a.p;
-  for (int it = tid; it < 1024; it += nthreads) {
-    const int row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j, o = m0 + row;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (e0 < 2 * p.rank && o < p.d_out) {
+  constexpr int PER = 1024 / NT, BATCH = PER < 8 ? PER : 8;
+#pragma unroll 1
+  for (int u0 = 0; u0 < PER; u0 += BATCH) {
+    float4 x[BATCH];
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int it = tid + (u0 + u) * NT, row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j, o = m0 + row;
+      const int k = e0 >= p.rank ? e0 - p.rank : e0;
+      x[u] = (e0 < 2 * p.rank && o < p.d_out) ? __ldg(reinterpret_cast<const float4*>(a.B + (size_t)o * p.rank + k))
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int it = tid + (u0 + u) * NT, row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j;
       const bool tail = e0 >= p.rank;
-      const int k = tail ? e0 - p.rank : e0;
-      const float4 bv = __ldg(reinterpret_cast<const float4*>(a.B + (size_t)o * p.rank + k));
-      const float x[4] = {bv.x, bv.y, bv.z, bv.w};
+      const float v[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
       float h[4], l[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) split_tf32(x[e], h[e], l[e]);
-      v = tail ? make_float4(l[0], l[1], l[2], l[3]) : make_float4(h[0], h[1], h[2], h[3]);
+      for (int e = 0; e < 4; ++e) split_tf32(v[e], h[e], l[e]);
+      *reinterpret_cast<float4*>(dst + row * 128 + ((j ^ (row & 7)) << 4)) =
+          tail ? make_float4(l[0], l[1], l[2], l[3]) : make_float4(h[0], h[1], h[2], h[3]);
     }
-    *reinterpret_cast<float4*>(dst + row * 128 + ((j ^ (row & 7)) << 4)) = v;
   }
 }
 
 // The operand images of all panels, written once per launch of the weight-tile kernel: image tn (tn < tiles_n)
 // is the A image of column panel tn, image tiles_n + tm the B image of row panel tm, each `atoms` atoms exactly
-// as they stand in shared memory, so that bulk copies bring them in.  One block per panel.
-// Output buffers of the caller that must start from zero (they are accumulated into with atomics later on the
-// stream): cleared by the same launch, which saves one memset launch per buffer.
-struct ZeroList { float* ptr[4]; size_t n[4]; };
-
-__global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8_t* __restrict__ img, const ZeroList zl) {
+// as they stand in shared memory, so that bulk copies bring them in.  One block per quarter of an atom, one
+// 16-byte piece per thread: the launch is short, and the kernel that follows waits for it.
+__global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8_t* __restrict__ img) {
   // the weight-tile kernel that follows may start now: it loads W0 tiles while the images are being written and
   // waits for this grid (griddep_wait) only before it copies the first image
   ptx::griddep_launch_dependents();
-  {
-    const size_t stride = (size_t)gridDim.x * blockDim.x;
+  const Params& p = a.p;
+  const int quarter = blockIdx.x & 3, c = (blockIdx.x >> 2) % a.atoms, panel = (blockIdx.x >> 2) / a.atoms;
+  uint8_t* dst = img + ((size_t)panel * a.atoms + c) * WT2_ATOM_BYTES;
+  const int it = quarter * 256 + threadIdx.x, row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j;
+  const bool tail = e0 >= p.rank;
+  const int k = tail ? e0 - p.rank : e0;
+  float x[4] = {0.f, 0.f, 0.f, 0.f};
+  if (e0 < 2 * p.rank) {
+    if (panel < a.tiles_n) {
+      const int col = panel * WT2_COLS + row;
+      if (col < p.d_in) {
 #pragma unroll
-    for (int b = 0; b < 4; ++b)
-      for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < zl.n[b]; e += stride) zl.ptr[b][e] = 0.f;
+        for (int e = 0; e < 4; ++e) x[e] = __ldg(a.A + (size_t)(k + e) * p.d_in + col);
+      }
+    } else {
+      const int o = (panel - a.tiles_n) * WT2_ROWS + row;
+      if (o < p.d_out) {
+        const float4 bv = __ldg(reinterpret_cast<const float4*>(a.B + (size_t)o * p.rank + k));
+        x[0] = bv.x; x[1] = bv.y; x[2] = bv.z; x[3] = bv.w;
+      }
+    }
   }
-  const int panel = blockIdx.x;
-  uint8_t* dst = img + (size_t)panel * a.atoms * WT2_ATOM_BYTES;
-  for (int c = 0; c < a.atoms; ++c) {
-    if (panel < a.tiles_n) build_atom_a(a, panel * WT2_COLS, c, dst + (size_t)c * WT2_ATOM_BYTES, threadIdx.x, blockDim.x);
-    else build_atom_b(a, (panel - a.tiles_n) * WT2_ROWS, c, dst + (size_t)c * WT2_ATOM_BYTES, threadIdx.x, blockDim.x);
-  }
+  float h[4], l[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) split_tf32(x[e], h[e], l[e]);
+  *reinterpret_cast<float4*>(dst + row * 128 + ((j ^ (row & 7)) << 4)) =
+      tail ? make_float4(l[0], l[1], l[2], l[3]) : make_float4(h[0], h[1], h[2], h[3]);
 }
 
 // Adding and subtracting 1.5 * 2^23 rounds |x| < 2^22 to the nearest integer, ties to even, exactly like
@@ -447,14 +500,14 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
   constexpr bool HAS_OUT1 = (MODE == WT2_PACK);      // staged in shared memory: the code words of the export
 
   if (threadIdx.x == 0) {
-    const uint32_t op_arrivals = a.op_img ? 1 : 32;   // one thread announcing a bulk copy, or the warp that built the atom
+    const uint32_t op_arrivals = a.op_img ? 1 : WT2_BUILDERS;   // one thread announcing a bulk copy, or the builders of the atom
     for (int i = 0; i < WT2_MAX_STAGES; ++i) {
       ptx::mbar_init(&bars->full[i], 1);
       // the export does not write back into the stage: the group that read it hands it back itself
       ptx::mbar_init(&bars->empty[i], MODE == WT2_PACK ? WT2_GROUP_THREADS : 1);
       ptx::mbar_init(&bars->written[i], WT2_GROUP_THREADS);
     }
-    for (int i = 0; i < 3; ++i) ptx::mbar_init(&bars->out_empty[i], 1);
+    for (int i = 0; i < WT2_GROUPS; ++i) ptx::mbar_init(&bars->out_empty[i], 1);
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&bars->afull[i], op_arrivals);
       ptx::mbar_init(&bars->aempty[i], 1);
@@ -482,14 +535,26 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = bars->tmem_base;
 
+  if (warp >= WT2_FIRST_EPI_WARP && warp < WT2_SECOND_STORE_WARP) {
+    // the epilogue warps have nothing to do until the first merge is complete: they clear the caller's buffers
+    const size_t stride = (size_t)gridDim.x * WT2_EPI_THREADS;
+    const size_t first = (size_t)blockIdx.x * WT2_EPI_THREADS + (threadIdx.x - WT2_FIRST_EPI_WARP * 32);
+#pragma unroll
+    for (int z = 0; z < 4; ++z)
+      for (size_t e = first; e < a.zero.n[z]; e += stride) a.zero.ptr[z][e] = 0.f;
+  }
+
   if (warp == 0) {
     // ------------------------------ TMA loads of W0 ---------------------------
     if (lane == 0) {
-      int stage = 0; uint32_t phase = 0;
+      StageSeq seq0(0, a.n_stages), seq1(1, a.n_stages);
+      static_assert(WT2_GROUPS == 2, "one stage sequence per epilogue group");
+      int grp = 0;                                   // tile i belongs to group i % WT2_GROUPS
       for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next()) {
         const int m0 = cur.m0(), n0 = cur.n0();
-        bounded_wait(&bars->empty[stage], phase ^ 1, bars);
-        if (bars->abort) break;
+        StageSeq& sq = grp ? seq1 : seq0;
+        const int stage = sq.stage();
+        if (!bounded_wait(&bars->empty[stage], sq.parity() ^ 1, bars)) break;
         uint8_t* dst = stage_base + (size_t)stage * WT2_STAGE_BYTES;
         const uint32_t sb_box_bytes = (uint32_t)(WT2_ROWS * a.sb_box * sizeof(float));
         ptx::mbar_arrive_expect_tx(&bars->full[stage], WT2_STAGE_BYTES + 2 * sb_box_bytes);
@@ -502,7 +567,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
           ptx::tma_load_2d(sdst, &tmap_s, &bars->full[stage], x0, m0);
           ptx::tma_load_2d(sdst + sb_box_bytes, &tmap_b, &bars->full[stage], x0, m0);
         }
-        if (++stage == a.n_stages) { stage = 0; phase ^= 1; }
+        sq.advance();
+        grp ^= 1;
       }
     }
     __syncwarp();
@@ -518,15 +584,19 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
     }
     __syncwarp();
-  } else if (warp == 2) {
+  } else if (warp == 2 || warp == WT2_SECOND_STORE_WARP) {
     // ------------------------------ TMA stores --------------------------------
+    // Two issuing threads, one per epilogue group (tiles sid, sid + 2, ...): a thread hands a stage back only
+    // after its copy has read it, which takes the TMA unit a thousand cycles or more behind the loads queued
+    // before it, and one thread doing that for every tile in turn was the slowest role of the kernel.
     if (lane == 0) {
-      int stage = 0; uint32_t phase = 0;
-      int ob = 0;
-      for (TileCursor cur(a); !bars->abort && cur.valid(); cur.next()) {
+      const int sid = warp == 2 ? 0 : 1;
+      StageSeq sq(sid, a.n_stages);
+      const int ob = sid;                            // the group's own staging buffer of code words
+      for (TileCursor cur(a, sid, WT2_GROUPS); !bars->abort && cur.valid(); cur.next()) {
         const int m0 = cur.m0(), n0 = cur.n0();
-        bounded_wait(&bars->written[stage], phase, bars);
-        if (bars->abort) break;
+        const int stage = sq.stage();
+        if (!bounded_wait(&bars->written[stage], sq.parity(), bars)) break;
         const uint8_t* src = stage_base + (size_t)stage * WT2_STAGE_BYTES;
         const uint8_t* src1 = out_base + (size_t)ob * a.out_bytes;
         const bool second_box = n0 + 64 < p.d_in;
@@ -541,8 +611,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
         ptx::bulk_wait_group_read0();
         if constexpr (MODE != WT2_PACK) ptx::mbar_arrive(&bars->empty[stage]);
         if constexpr (HAS_OUT1) ptx::mbar_arrive(&bars->out_empty[ob]);
-        if constexpr (HAS_OUT1) { if (++ob == a.n_out) ob = 0; }
-        if (++stage == a.n_stages) { stage = 0; phase ^= 1; }
+        sq.advance();
       }
       ptx::bulk_wait_group0();
     }
@@ -551,7 +620,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     // ------------------------------ MMA operands ------------------------------
     // With ready-made images one thread issues bulk copies; without, the warp builds each atom from A and B.
     const bool img = a.op_img != nullptr;
-    if (img ? lane == 0 : true) {
+    const int btid = lane;                           // builder thread index
+    if (img ? btid == 0 : true) {
       if (img) ptx::griddep_wait();                  // k_split_operands has written the images
       int slot = 0; uint32_t slot_phase = 0;
       int panel = -1, pseq = -1;
@@ -567,7 +637,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
             ptx::mbar_arrive_expect_tx(&bars->afull[ab], a_img_bytes);
             ptx::bulk_load(acat, a.op_img + (size_t)cur.tn * a_img_bytes, a_img_bytes, &bars->afull[ab]);
           } else {
-            for (int c = 0; c < a.atoms; ++c) build_atom_a(a, cur.n0(), c, acat + (size_t)c * WT2_ATOM_BYTES, lane, 32);
+            for (int c = 0; c < a.atoms; ++c) build_atom_a<WT2_BUILDERS>(a, cur.n0(), c, acat + (size_t)c * WT2_ATOM_BYTES, btid);
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(&bars->afull[ab]);
           }
@@ -581,7 +651,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
             ptx::bulk_load(chunk, a.op_img + ((size_t)(a.tiles_n + cur.tm) * a.atoms + c) * WT2_ATOM_BYTES,
                            WT2_ATOM_BYTES, &bars->bfull[slot]);
           } else {
-            build_atom_b(a, cur.m0(), c, chunk, lane, 32);
+            build_atom_b<WT2_BUILDERS>(a, cur.m0(), c, chunk, btid);
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(&bars->bfull[slot]);
           }
@@ -590,11 +660,12 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
     }
     __syncwarp();
-  } else if (warp >= WT2_FIRST_EPI_WARP) {
+  } else if (warp >= WT2_FIRST_EPI_WARP && warp < WT2_SECOND_STORE_WARP) {
     // ------------------------------ epilogue ----------------------------------
-    // Three groups of eight warps; group grp owns the CTA's tiles i = grp, grp + 3, ... (accumulator stage i % 4).
+    // Two groups of eight warps; group grp owns the CTA's tiles i = grp, grp + 2, ... (accumulator stage i % 4).
     // A thread is one weight row (TMEM lane) and one 64-column half of its group's tile.  The groups meet only
-    // through the mbarriers: while one waits for a merge or a tile, the others keep the pipes busy.
+    // through the mbarriers: while one waits for a merge or a tile, the other keeps the pipes busy.  (Three groups
+    // were measured: each tile then takes longer, the stages are held longer, and nothing is gained.)
     const int quarter = warp & 3;
     const int grp = (warp - WT2_FIRST_EPI_WARP) >> 3;
     const int chalf = ((warp - WT2_FIRST_EPI_WARP) >> 2) & 1;   // column half of the tile
@@ -641,9 +712,14 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     int sb_buf = 0;
     const int qn_bits = kRoundMagicBits + (int)p.qn;
 
+    // the group's own W0 stages and staging buffer of code words (no division per tile: that is dozens of
+    // instructions, on warps whose issue slots are the scarce thing here)
+    StageSeq sq(grp, a.n_stages);
+    const int ob = grp;
+    [[maybe_unused]] int ob_uses = 0;
     for (int i = grp; cur.valid(); cur.next(), i += WT2_GROUPS) {
-      const int stage = i % a.n_stages;                         // W0 stage of tile i and its phase
-      const uint32_t phase = (uint32_t)((i / a.n_stages) & 1);
+      const int stage = sq.stage();
+      const uint32_t phase = sq.parity();
       const int m0 = cur.m0(), n0 = cur.n0();
       const int o = m0 + row;
       const bool row_ok = o < p.d_out;
@@ -673,11 +749,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       bounded_wait(&bars->tmem_full[acc], (uint32_t)((i >> 2) & 1), bars);
       ptx::tc_fence_after_sync();
       bounded_wait(&bars->full[stage], phase, bars);
-      int ob = 0;
       if constexpr (HAS_OUT1) {
-        const int uses = i / a.n_out;                           // earlier tiles that went through this buffer
-        ob = i - uses * a.n_out;
-        if (uses >= 1) bounded_wait(&bars->out_empty[ob], (uint32_t)((uses - 1) & 1), bars);
+        if (ob_uses >= 1) bounded_wait(&bars->out_empty[ob], (uint32_t)((ob_uses - 1) & 1), bars);
       }
       uint8_t* tile_rows = stage_base + (size_t)stage * WT2_STAGE_BYTES + row * 128;
       // second output: the export's staging rows in shared memory; the STE factors go straight to the tile's block
@@ -816,6 +889,8 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       if constexpr (MODE == WT2_PACK) ptx::mbar_arrive(&bars->empty[stage]);   // W0 has been read
       sb_buf ^= 1;
       if (has_next) stage_sb(m1, n1, sb_buf);          // the other buffer: its readers passed this tile's barrier
+      sq.advance();
+      ++ob_uses;
     }
   }
 
@@ -874,7 +949,7 @@ inline bool wtile_plan(WtileArgs& a, int mode, bool sb_by_tma = true) {
   WtileArgs pick = a;
   const int ring_opts[4] = {2 * a.atoms, a.atoms + 1, 3, 2};
   for (int stages = 2; stages <= WT2_MAX_STAGES; ++stages)
-    for (int n_out = has_out ? 1 : 0; n_out <= (has_out ? WT2_GROUPS : 0); ++n_out)
+    for (int n_out = has_out ? WT2_GROUPS : 0; n_out <= (has_out ? WT2_GROUPS : 0); ++n_out)   // one per group
       for (int n_abuf = 1; n_abuf <= 2; ++n_abuf)
         for (int ro = 0; ro < 4; ++ro) {
           const int ring = ring_opts[ro];
@@ -959,13 +1034,17 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   }
 #endif
   const size_t smem = wtile_smem_bytes(a);
+#ifdef L4Q_EXPERIMENT
+  if (const char* e = getenv("L4Q_WT_IMG")) { if (!atoi(e)) op_img = nullptr; }
+#endif
   if (op_img) {
-    ZeroList zl{};
-    if (zero) zl = *zero;
-    k_split_operands<<<a.tiles_n + a.tiles_m, 256, 0, st>>>(a, static_cast<uint8_t*>(op_img), zl);
+    k_split_operands<<<(a.tiles_n + a.tiles_m) * a.atoms * 4, 256, 0, st>>>(a, static_cast<uint8_t*>(op_img));
     if (cudaGetLastError() != cudaSuccess) return L4Q_ERR_CUDA;
-    if (zero && zeroed) *zeroed = true;
     a.op_img = static_cast<const uint8_t*>(op_img);
+  }
+  if (zero) {                                       // the kernel's epilogue warps clear these before their first tile
+    a.zero = *zero;
+    if (zeroed) *zeroed = true;
   }
   auto launch = [&](auto kern) -> l4q_status {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
