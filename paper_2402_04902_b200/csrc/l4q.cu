@@ -107,24 +107,53 @@ size_t operand_image_bytes(const l4q_desc* d, const Params& p) {
   return d->io_dtype == L4Q_BF16 && wtile_tc_supported(p, WT2_DEQUANT) ? align_up(wtile_image_bytes(p), 256) : 0;
 }
 
+// bf16 copies of A and B^T for the weight-gradient kernel (rows up to the MMA's N, see Bf16Copies)
+size_t wgrad_copy_bytes(const l4q_desc* d, const Params& p) {
+  if (d->io_dtype != L4Q_BF16 || !wgrad_rank_supported(p.rank)) return 0;
+  const size_t rn = (size_t)wgrad_rn(p.rank);
+  return align_up(rn * p.d_in * 2, 256) + align_up(rn * p.d_out * 2, 256);
+}
+
 size_t factor_scratch_bytes(const l4q_desc* d) {
   return align_up(factor_elems((int)d->d_out, (int)d->d_in) * sizeof(__half), 256);
 }
 
 inline l4q_status launch_status() { return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA; }
 
+// The bf16 copies of A and B^T inside a scratch region of wgrad_copy_bytes().
+Bf16Copies carve_copies(const Params& p, void* base) {
+  Bf16Copies cp{};
+  cp.rn = wgrad_rn(p.rank);
+  cp.A16 = reinterpret_cast<__nv_bfloat16*>(base);
+  cp.Bt16 = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(base) + align_up((size_t)cp.rn * p.d_in * 2, 256));
+  return cp;
+}
+
+// The copies by a launch of their own (where no operand-split launch made them).
+l4q_status launch_copies(const Params& p, const float* A, const float* B, const Bf16Copies& cp, cudaStream_t st) {
+  WtileArgs a{};
+  a.p = p; a.A = A; a.B = B;
+  const int blocks = (int)(((long long)cp.rn * (p.d_in + p.d_out) / 8 + 255) / 256);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  k_split_operands<<<blocks, 256, 0, st>>>(a, nullptr, 0, cp);
+  return launch_status();
+}
+
 // Merge + fake-quantize the whole weight into `wq` (io dtype) -- the recompute step of fwd and bwd.
 // `fac` (optional, bf16 mode only) also receives the fp16 STE factors the weight-gradient kernel reads.
 template <bool IO_BF16>
 l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const float* B, const float* s,
                           const float* b, void* wq, __half* fac, cudaStream_t st, void* op_img = nullptr,
-                          const ZeroList* zero = nullptr, bool* zeroed = nullptr) {
+                          const ZeroList* zero = nullptr, bool* zeroed = nullptr, const Bf16Copies* copies = nullptr,
+                          bool* copied = nullptr) {
   if constexpr (IO_BF16) {
     const int mode = fac ? WT2_DEQUANT_F : WT2_DEQUANT;
     if (wtile_tc_supported(p, mode)) {               // tensor-core merge, TMA in and out
       KernelScope ks(L4Q_KERNEL_DEQUANT, st);   // covers the operand split too, which is one more launch
       if (op_img) g_launches.fetch_add(1, std::memory_order_relaxed);
-      return launch_wtile_tc(mode, p, W0, A, B, s, b, wq, fac, nullptr, nullptr, st, op_img, zero, zeroed);
+      if (op_img && copies && copied) *copied = true;
+      return launch_wtile_tc(mode, p, W0, A, B, s, b, wq, fac, nullptr, nullptr, st, op_img, zero, zeroed,
+                             op_img ? copies : nullptr);
     }
   }
   const size_t smem = weight_tile_smem_bytes(p.rank);
@@ -169,6 +198,7 @@ struct LoraWorkspace {
   float* zero_B = nullptr;       // QAT-LoRA: a zero LoRA factor, so that the weight-tile kernel quantizes W0 alone
   void* op_img = nullptr;        // QAT-LoRA: the split operands of that kernel's merge (operand_image_bytes)
   float *dA_unused = nullptr, *dB_unused = nullptr;   // QAT-LoRA backward: the merged-layer LoRA gradients, not wanted
+  void* copies = nullptr;        // QAT-LoRA backward: bf16 copies of A and the zero factor for the weight-gradient kernel
   size_t bytes = 0;
 };
 
@@ -189,6 +219,7 @@ LoraWorkspace lora_workspace(const l4q_desc* d, const Params& p, int kind, int o
     if (op == L4Q_OP_BWD) {
       w.dA_unused = reinterpret_cast<float*>(take((size_t)p.rank * p.d_in * sizeof(float)));
       w.dB_unused = reinterpret_cast<float*>(take((size_t)p.d_out * p.rank * sizeof(float)));
+      if (wgrad_copy_bytes(d, p)) w.copies = take(wgrad_copy_bytes(d, p));
     }
   }
   w.bytes = off + 256;
@@ -215,7 +246,7 @@ size_t l4q_workspace_bytes(const l4q_desc* desc, int op) {
       return wq_scratch_bytes(desc) + operand_image_bytes(desc, p) + 256;
     case L4Q_OP_BWD:   // W_q for the input gradient, and in bf16 mode the fp16 STE factors for the weight gradient
       return wq_scratch_bytes(desc) + (desc->io_dtype == L4Q_BF16 ? factor_scratch_bytes(desc) : 0) +
-             operand_image_bytes(desc, p) + 256;
+             operand_image_bytes(desc, p) + wgrad_copy_bytes(desc, p) + 256;
     case L4Q_OP_PACK:   // optional (see l4q_pack_int)
       return operand_image_bytes(desc, p);
     default:
@@ -284,14 +315,15 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
   __half* fac = (!f32 && n_param_out == 4)
                     ? reinterpret_cast<__half*>(static_cast<unsigned char*>(workspace) + wq_scratch_bytes(desc))
                     : nullptr;
+  unsigned char* ws_tail = static_cast<unsigned char*>(workspace) + wq_scratch_bytes(desc) +
+                           (f32 ? 0 : factor_scratch_bytes(desc));
+  Bf16Copies copies{};
+  bool copied = false;
+  if (!f32 && n_param_out == 4) copies = carve_copies(p, ws_tail + operand_image_bytes(desc, p));
   if (dX || fac) {
     st = f32 ? launch_dequant<false>(p, W0, A, B, s, b, wq, nullptr, stream)
-             : launch_dequant<true>(p, W0, A, B, s, b, wq, fac, stream,
-                                    operand_image_bytes(desc, p)
-                                        ? static_cast<unsigned char*>(workspace) + wq_scratch_bytes(desc) +
-                                              factor_scratch_bytes(desc)
-                                        : nullptr,
-                                    n_param_out == 4 ? &grads : nullptr, &zeroed);
+             : launch_dequant<true>(p, W0, A, B, s, b, wq, fac, stream, operand_image_bytes(desc, p) ? ws_tail : nullptr,
+                                    n_param_out == 4 ? &grads : nullptr, &zeroed, fac ? &copies : nullptr, &copied);
     if (st != L4Q_OK) return st;
   }
   if (n_param_out == 4 && !zeroed) {
@@ -328,8 +360,9 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
     if (st != L4Q_OK) return st;
   }
   if (n_param_out == 4) {
+    if (!copied && (st = launch_copies(p, A, B, copies, stream)) != L4Q_OK) return st;
     KernelScope ks(L4Q_KERNEL_GEMM_WGRAD, stream);
-    st = gemm_wgrad_bf16(p, X, dY, fac, A, B, dA, dB, ds, db, stream);
+    st = gemm_wgrad_bf16(p, X, dY, fac, copies.A16, copies.Bt16, dA, dB, ds, db, stream);
     if (st != L4Q_OK) return st;
   }
   return L4Q_OK;
@@ -432,8 +465,10 @@ l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, co
     const size_t gsz = (size_t)p.d_out * p.ngroups * sizeof(float);
     if (cudaMemsetAsync(ds, 0, gsz, stream) != cudaSuccess || cudaMemsetAsync(db, 0, gsz, stream) != cudaSuccess)
       return L4Q_ERR_CUDA;
+    const Bf16Copies cp = carve_copies(p, w.copies);
+    if ((st = launch_copies(p, A, w.zero_B, cp, stream)) != L4Q_OK) return st;
     KernelScope ks(L4Q_KERNEL_GEMM_WGRAD, stream);
-    if ((st = gemm_wgrad_bf16(p, X, dY, w.fac, A, w.zero_B, w.dA_unused, w.dB_unused, ds, db, stream)) != L4Q_OK)
+    if ((st = gemm_wgrad_bf16(p, X, dY, w.fac, cp.A16, cp.Bt16, w.dA_unused, w.dB_unused, ds, db, stream)) != L4Q_OK)
       return st;
   }
   return L4Q_OK;

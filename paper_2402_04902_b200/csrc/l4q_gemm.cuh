@@ -67,7 +67,6 @@ struct GemmArgs {
   Params p;
   const __half* F;             // STE factors of the weights (ste_factor), in the factor_index layout
   int f_tiles_n;               // column tiles of that layout
-  const float *A, *B;
   float *dA, *dB, *ds, *db;
 };
 
@@ -75,6 +74,7 @@ struct __align__(8) GemmBarriers {
   uint64_t full[8], empty[8];
   uint64_t tmem_full[ACC_STAGES], tmem_empty[ACC_STAGES];
   uint64_t epi_mma;            // wgrad: the epilogue's own MMAs have completed
+  uint64_t epi_ops;            // wgrad: the tile's bf16 slices of A and B^T have landed
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
@@ -218,7 +218,9 @@ template <int RANK>
 __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, int n0, uint32_t tmem_acc, int quarter,
                                                     int lane, int eg, uint8_t* epi_smem, GemmBarriers* bars,
                                                     uint64_t* tmem_full_bar, uint32_t full_parity,
-                                                    uint64_t* tmem_empty_bar, uint32_t& epi_phase) {
+                                                    uint64_t* tmem_empty_bar, uint32_t& epi_phase,
+                                                    const CUtensorMap* tmap_a16, const CUtensorMap* tmap_bt16,
+                                                    uint32_t& ops_phase) {
   constexpr int RN = wgrad_rn(RANK);
   const Params& p = g.p;
   uint8_t* gm = epi_smem;
@@ -231,37 +233,16 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
   constexpr uint32_t DB_COL = 0, DA_COL0 = RN, DA_COL1 = 128;   // result columns inside the drained accumulator
 
-  // ---- bf16 copies of the tile's slices of A and B (nothing here depends on the accumulator) ----
-  // The MMAs of the previous tile that read these buffers have completed: every thread waited for them.
+  // ---- the tile's slices of A and B^T, ready-made bf16 (the operand-split launch of the same backward call wrote
+  //      them), by TMA into the swizzled K-major layout the MMAs read.  The MMAs of the previous tile that read
+  //      these buffers have completed: every thread waited for them. ----
+  if (t256 == 0) {
+    ptx::mbar_arrive_expect_tx(&bars->epi_ops, 6 * RN * 128);
 #pragma unroll
-  for (int u = 0; u < (RN * 32) / EPI_THREADS; ++u) {
-    const int q = t256 + u * EPI_THREADS;              // 16-byte chunk: rank k, columns n0 + 8 jc .. + 7
-    const int k = q >> 5, jc = q & 31;
-    const int col = n0 + jc * 8;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (k < RANK && col < p.d_in) {
-      const float4* src = reinterpret_cast<const float4*>(g.A + (size_t)k * p.d_in + col);
-      const float4 a0 = __ldg(src), a1 = __ldg(src + 1);
-      v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w);
-      v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
-    }
-    *reinterpret_cast<uint4*>(abf + (jc >> 3) * (RN * 128) + k * 128 + (((jc & 7) ^ (k & 7)) << 4)) = v;
+    for (int blk = 0; blk < 4; ++blk) ptx::tma_load_2d(abf + blk * (RN * 128), tmap_a16, &bars->epi_ops, n0 + blk * 64, 0);
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) ptx::tma_load_2d(btbf + blk * (RN * 128), tmap_bt16, &bars->epi_ops, m0 + blk * 64, 0);
   }
-#pragma unroll
-  for (int u = 0; u < RN / 2; u += 4) {                // thread = (weight row t, half eg of the ranks)
-    const int n = eg * (RN / 2) + u;
-    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (row_ok && n < RANK) bv = __ldg(reinterpret_cast<const float4*>(g.B + (size_t)o * RANK + n));
-    const float be[4] = {bv.x, bv.y, bv.z, bv.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int nn = n + e;
-      uint8_t* dst = btbf + (t >> 6) * (RN * 128) + nn * 128 + ((((t & 63) >> 3) ^ (nn & 7)) << 4) + (t & 7) * 2;
-      *reinterpret_cast<__nv_bfloat16*>(dst) = __float2bfloat16_rn(be[e]);
-    }
-  }
-  ptx::fence_proxy_async_smem();
-  ptx::named_bar_sync(3, EPI_THREADS);
 
   bounded_wait(tmem_full_bar, full_parity, bars);
   ptx::tc_fence_after_sync();
@@ -335,6 +316,7 @@ __device__ __forceinline__ void wgrad_epilogue_tile(const GemmArgs& g, int m0, i
     ptx::tc_fence_before_sync();                       // the TMEM reads above come before the MMAs below
     ptx::named_bar_sync(3, EPI_THREADS);
     if (t256 == 0 && !bars->abort) {
+      if (h == 0) { bounded_wait(&bars->epi_ops, ops_phase, bars); ops_phase ^= 1; }   // the slices of A and B^T
       ptx::tc_fence_after_sync();
       constexpr uint32_t idesc_db = ptx::make_idesc_bf16(128, RN, false, false);
       constexpr uint32_t idesc_da = ptx::make_idesc_bf16(128, RN, true, false);
@@ -406,7 +388,9 @@ template <int RANK>
 __device__ __forceinline__ void wgrad_epilogue_tile_q(const GemmArgs& g, int m0, int n0, uint32_t tmem_acc, int quarter,
                                                       int lane, int eg, uint8_t* epi_smem, GemmBarriers* bars,
                                                       uint64_t* tmem_full_bar, uint32_t full_parity,
-                                                      uint64_t* tmem_empty_bar, uint32_t& epi_phase) {
+                                                      uint64_t* tmem_empty_bar, uint32_t& epi_phase,
+                                                      const CUtensorMap* tmap_a16, const CUtensorMap* tmap_bt16,
+                                                      uint32_t& ops_phase) {
   constexpr int RN = wgrad_rn(RANK);
   static_assert(RN == 16, "quarter path");
   constexpr int GMQ = GM_BYTES / 2;
@@ -420,36 +404,14 @@ __device__ __forceinline__ void wgrad_epilogue_tile_q(const GemmArgs& g, int m0,
   const bool row_ok = o < p.d_out;
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
 
-  // ---- bf16 copies of the tile's slices of A and B (as in wgrad_epilogue_tile) ----
+  // ---- the tile's bf16 slices of A and B^T by TMA (as in wgrad_epilogue_tile) ----
+  if (t256 == 0) {
+    ptx::mbar_arrive_expect_tx(&bars->epi_ops, 6 * RN * 128);
 #pragma unroll
-  for (int u = 0; u < (RN * 32) / EPI_THREADS; ++u) {
-    const int q = t256 + u * EPI_THREADS;
-    const int k = q >> 5, jc = q & 31;
-    const int col = n0 + jc * 8;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (k < RANK && col < p.d_in) {
-      const float4* src = reinterpret_cast<const float4*>(g.A + (size_t)k * p.d_in + col);
-      const float4 a0 = __ldg(src), a1 = __ldg(src + 1);
-      v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w);
-      v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
-    }
-    *reinterpret_cast<uint4*>(abf + (jc >> 3) * (RN * 128) + k * 128 + (((jc & 7) ^ (k & 7)) << 4)) = v;
+    for (int blk = 0; blk < 4; ++blk) ptx::tma_load_2d(abf + blk * (RN * 128), tmap_a16, &bars->epi_ops, n0 + blk * 64, 0);
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) ptx::tma_load_2d(btbf + blk * (RN * 128), tmap_bt16, &bars->epi_ops, m0 + blk * 64, 0);
   }
-#pragma unroll
-  for (int u = 0; u < RN / 2; u += 4) {
-    const int n = eg * (RN / 2) + u;
-    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (row_ok && n < RANK) bv = __ldg(reinterpret_cast<const float4*>(g.B + (size_t)o * RANK + n));
-    const float be[4] = {bv.x, bv.y, bv.z, bv.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int nn = n + e;
-      uint8_t* dst = btbf + (t >> 6) * (RN * 128) + nn * 128 + ((((t & 63) >> 3) ^ (nn & 7)) << 4) + (t & 7) * 2;
-      *reinterpret_cast<__nv_bfloat16*>(dst) = __float2bfloat16_rn(be[e]);
-    }
-  }
-  ptx::fence_proxy_async_smem();
-  ptx::named_bar_sync(3, EPI_THREADS);
 
   bounded_wait(tmem_full_bar, full_parity, bars);
   ptx::tc_fence_after_sync();
@@ -519,6 +481,7 @@ __device__ __forceinline__ void wgrad_epilogue_tile_q(const GemmArgs& g, int m0,
     ptx::tc_fence_before_sync();
     ptx::named_bar_sync(3, EPI_THREADS);
     if (t256 == 0 && !bars->abort) {
+      if (q == 0) { bounded_wait(&bars->epi_ops, ops_phase, bars); ops_phase ^= 1; }   // the slices of A and B^T
       ptx::tc_fence_after_sync();
       constexpr uint32_t idesc_db = ptx::make_idesc_bf16(128, RN, false, false);
       constexpr uint32_t idesc_da = ptx::make_idesc_bf16(64, RN, true, false);
@@ -606,11 +569,12 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::mbar_init(&bars->tmem_empty[i], EPI_THREADS);
     }
     ptx::mbar_init(&bars->epi_mma, 1);
+    ptx::mbar_init(&bars->epi_ops, 1);
     bars->abort = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tmap(&tmap_a);
     ptx::prefetch_tmap(&tmap_b);
-    if constexpr (EXT) { ptx::prefetch_tmap(&tmap_a2); ptx::prefetch_tmap(&tmap_b2); }
+    if constexpr (EXT || EPI == EPI_WGRAD) { ptx::prefetch_tmap(&tmap_a2); ptx::prefetch_tmap(&tmap_b2); }
     if constexpr (TMA_STORE) ptx::prefetch_tmap(&tmap_c);
   }
   if (warp == 1) {
@@ -738,7 +702,7 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int quarter = warp & 3;
     const int eg = (warp - EPI_FIRST_WARP) >> 2;
     int acc = 0; uint32_t acc_phase = 0;
-    [[maybe_unused]] uint32_t epi_phase = 0;
+    [[maybe_unused]] uint32_t epi_phase = 0, ops_phase = 0;
     WorkIter<TAIL_SPLIT> work(num_tiles, total_kb);
     WorkUnit u;
     while (work.next(u)) {
@@ -836,10 +800,10 @@ k_gemm_bf16(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       } else {
         if constexpr (wgrad_quarters(RANK))
           wgrad_epilogue_tile_q<RANK>(g, m0, n0, tmem_acc, quarter, lane, eg, epi_smem, bars, &bars->tmem_full[acc],
-                                      acc_phase, &bars->tmem_empty[acc], epi_phase);
+                                      acc_phase, &bars->tmem_empty[acc], epi_phase, &tmap_a2, &tmap_b2, ops_phase);
         else
           wgrad_epilogue_tile<RANK>(g, m0, n0, tmem_acc, quarter, lane, eg, epi_smem, bars, &bars->tmem_full[acc],
-                                    acc_phase, &bars->tmem_empty[acc], epi_phase);
+                                    acc_phase, &bars->tmem_empty[acc], epi_phase, &tmap_a2, &tmap_b2, ops_phase);
       }
       if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1; }
     }
@@ -922,7 +886,8 @@ inline int sm_count() {
   return n;
 }
 
-// `ta2`, `tb2`: second operand pair of an EXT launch (g.num_kb2 K blocks); ignored otherwise.
+// `ta2`, `tb2`: second operand pair of an EXT launch (g.num_kb2 K blocks), or, for the weight-gradient epilogue, the
+// maps of the bf16 copies of A [rn, d_in] and B^T [rn, d_out] (boxes of 64 columns x rn rows); ignored otherwise.
 template <bool A_MN, bool B_MN, int EPI, int RANK, int STAGES, int TN = BN, bool EXT = false>
 l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g, cudaStream_t st,
                        const CUtensorMap* ta2 = nullptr, const CUtensorMap* tb2 = nullptr) {
@@ -936,7 +901,8 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
   // wave is cut along K, is better off with 16 rows
   g.band = EPI == EPI_STORE ? tile_band_rows(g.tiles_m, (size_t)BM * g.K * 2) : std::min(16, g.tiles_m);
   if (!EXT) g.num_kb2 = 0;
-  if (EXT && (!ta2 || !tb2)) return L4Q_ERR_INVALID_ARG;
+  constexpr bool SECOND_MAPS = EXT || EPI == EPI_WGRAD;   // EXT: a second operand pair; WGRAD: the bf16 copies of A and B^T
+  if (SECOND_MAPS && (!ta2 || !tb2)) return L4Q_ERR_INVALID_ARG;
   auto kern = k_gemm_bf16<A_MN, B_MN, EPI, RANK, STAGES, TN, EXT>;
   const size_t smem = gemm_smem_bytes(STAGES, EPI == EPI_WGRAD ? wgrad_epi_smem_bytes(RANK)
                                               : TMA_STORE ? store_epi_smem_bytes() : 0, stage_bytes_for(TN));
@@ -945,7 +911,7 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
   const int tiles = g.tiles_m * g.tiles_n, sms = sm_count();
   int grid = std::min(tiles, sms);
   if (EPI != EPI_STORE && tiles < sms) grid = tiles * std::min(sms / tiles, g.num_kb);   // K slices for the idle SMs
-  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, EXT ? *ta2 : ta, EXT ? *tb2 : tb, tc, g);
+  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, SECOND_MAPS ? *ta2 : ta, SECOND_MAPS ? *tb2 : tb, tc, g);
   return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
 }
 
@@ -972,23 +938,25 @@ inline l4q_status gemm_dgrad_bf16(const Params& p, const void* dY, const void* W
 }
 
 // G[d_out, d_in] = dY^T X reduced on chip into dA, dB, ds, db (which must be zero on entry).
-inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY, const void* F, const float* A,
-                                  const float* B, float* dA, float* dB, float* ds, float* db, cudaStream_t st) {
-  CUtensorMap ta, tb;
-  if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BK) || !make_tmap_bf16(&tb, X, p.tokens, p.d_in, BK))
+// A16 [rn, d_in], Bt16 [rn, d_out]: bf16 copies of A and B^T with rn = wgrad_rn(rank) rows, rows beyond the rank zero.
+inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY, const void* F, const void* A16,
+                                  const void* Bt16, float* dA, float* dB, float* ds, float* db, cudaStream_t st) {
+  CUtensorMap ta, tb, ta16, tbt16;
+  const int rn = wgrad_rn(p.rank);
+  if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BK) || !make_tmap_bf16(&tb, X, p.tokens, p.d_in, BK) ||
+      !make_tmap_bf16(&ta16, A16, rn, p.d_in, rn) || !make_tmap_bf16(&tbt16, Bt16, rn, p.d_out, rn))
     return L4Q_ERR_CUDA;
   GemmArgs g{};
   g.M = p.d_out; g.N = p.d_in; g.K = p.tokens;
   g.p = p;
   g.F = reinterpret_cast<const __half*>(F);
   g.f_tiles_n = factor_tiles_n(p.d_in);
-  g.A = A; g.B = B;
   g.dA = dA; g.dB = dB; g.ds = ds; g.db = db;
   switch (p.rank) {
-    case 8: return launch_gemm<true, true, EPI_WGRAD, 8, wgrad_stages(8)>(ta, tb, g, st);
-    case 16: return launch_gemm<true, true, EPI_WGRAD, 16, wgrad_stages(16)>(ta, tb, g, st);
-    case 32: return launch_gemm<true, true, EPI_WGRAD, 32, 3>(ta, tb, g, st);
-    case 64: return launch_gemm<true, true, EPI_WGRAD, 64, 3>(ta, tb, g, st);
+    case 8: return launch_gemm<true, true, EPI_WGRAD, 8, wgrad_stages(8)>(ta, tb, g, st, &ta16, &tbt16);
+    case 16: return launch_gemm<true, true, EPI_WGRAD, 16, wgrad_stages(16)>(ta, tb, g, st, &ta16, &tbt16);
+    case 32: return launch_gemm<true, true, EPI_WGRAD, 32, 3>(ta, tb, g, st, &ta16, &tbt16);
+    case 64: return launch_gemm<true, true, EPI_WGRAD, 64, 3>(ta, tb, g, st, &ta16, &tbt16);
     default: return L4Q_ERR_UNSUPPORTED;
   }
 }

@@ -65,6 +65,14 @@ enum { WT2_DEQUANT = 0, WT2_DEQUANT_F = 1, WT2_PACK = 2 };
 // stream): cleared by a launch that runs anyway, which saves one memset launch per buffer.
 struct ZeroList { float* ptr[4]; size_t n[4]; };
 
+// bf16 copies of the LoRA factors for the weight-gradient kernel of the same backward call, which contracts its
+// G * m tiles with them on the tensor cores (Eq. 13-14): A16 [rn, d_in] and Bt16 = B^T [rn, d_out], row-major,
+// rows beyond the rank zero (rn = the MMA's N, a multiple of 16).  Written by the operand-split launch.
+struct Bf16Copies {
+  __nv_bfloat16 *A16, *Bt16;
+  int rn;
+};
+
 struct WtileArgs {
   Params p;
   const float *A, *B, *s, *b;
@@ -238,11 +246,43 @@ __device__ __forceinline__ void build_atom_b(const WtileArgs& a, int m0, int c, 
 // is the A image of column panel tn, image tiles_n + tm the B image of row panel tm, each `atoms` atoms exactly
 // as they stand in shared memory, so that bulk copies bring them in.  One block per quarter of an atom, one
 // 16-byte piece per thread: the launch is short, and the kernel that follows waits for it.
-__global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8_t* __restrict__ img) {
+__global__ void __launch_bounds__(256) k_split_operands(const WtileArgs a, uint8_t* __restrict__ img, int image_blocks,
+                                                        const Bf16Copies cp) {
   // the weight-tile kernel that follows may start now: it loads W0 tiles while the images are being written and
   // waits for this grid (griddep_wait) only before it copies the first image
   ptx::griddep_launch_dependents();
   const Params& p = a.p;
+  if ((int)blockIdx.x >= image_blocks) {
+    // the blocks after the images: bf16 copies of A and of B^T, 8 values per thread
+    const long long e = ((long long)(blockIdx.x - image_blocks) * 256 + threadIdx.x) * 8;
+    const long long na = (long long)cp.rn * p.d_in, nb = (long long)cp.rn * p.d_out;
+    float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    __nv_bfloat16* dst = nullptr;
+    if (e < na) {                                    // A16[k, col .. col + 7]   (d_in is a multiple of 8)
+      const int k = (int)(e / p.d_in), col = (int)(e - (long long)k * p.d_in);
+      if (k < p.rank) {
+        const float4 x0 = __ldg(reinterpret_cast<const float4*>(a.A + (size_t)k * p.d_in + col));
+        const float4 x1 = __ldg(reinterpret_cast<const float4*>(a.A + (size_t)k * p.d_in + col + 4));
+        v[0] = x0.x; v[1] = x0.y; v[2] = x0.z; v[3] = x0.w; v[4] = x1.x; v[5] = x1.y; v[6] = x1.z; v[7] = x1.w;
+      }
+      dst = cp.A16 + e;
+    } else if (e - na < nb) {                        // Bt16[k, o .. o + 7]      (d_out is a multiple of 8)
+      const long long f = e - na;
+      const int k = (int)(f / p.d_out), o = (int)(f - (long long)k * p.d_out);
+      if (k < p.rank) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = __ldg(a.B + (size_t)(o + j) * p.rank + k);
+      }
+      dst = cp.Bt16 + f;
+    }
+    if (dst) {
+      uint4 o4;
+      o4.x = pack_bf16x2(v[0], v[1]); o4.y = pack_bf16x2(v[2], v[3]);
+      o4.z = pack_bf16x2(v[4], v[5]); o4.w = pack_bf16x2(v[6], v[7]);
+      *reinterpret_cast<uint4*>(dst) = o4;
+    }
+    return;
+  }
   const int quarter = blockIdx.x & 3, c = (blockIdx.x >> 2) % a.atoms, panel = (blockIdx.x >> 2) / a.atoms;
   uint8_t* dst = img + ((size_t)panel * a.atoms + c) * WT2_ATOM_BYTES;
   const int it = quarter * 256 + threadIdx.x, row = it & 127, j = it >> 7, e0 = 32 * c + 4 * j;
@@ -994,13 +1034,14 @@ inline size_t wtile_image_bytes(const Params& p) {
   return ((size_t)ceil_div(p.d_out, WT2_ROWS) + (size_t)ceil_div(p.d_in, WT2_COLS)) * atoms * WT2_ATOM_BYTES;
 }
 
+// `copies` (optional, needs `op_img`): the operand-split launch also writes these bf16 copies of A and B^T.
 // `op_img` (optional, wtile_image_bytes(p) bytes of device scratch, 16-byte aligned): with it the MMA operands are
 // split once by a launch of k_split_operands and reach the tiles by bulk copies; without it one warp of every CTA
 // builds them tile by tile (slower).  `zero` (optional): buffers that launch also clears; *zeroed is set when it did.
 inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, const float* A, const float* B,
                                   const float* s, const float* b, void* out0, void* out1, __half* s16, __half* b16,
                                   cudaStream_t st, void* op_img = nullptr, const ZeroList* zero = nullptr,
-                                  bool* zeroed = nullptr) {
+                                  bool* zeroed = nullptr, const Bf16Copies* copies = nullptr) {
   WtileArgs a{};
   a.p = p; a.A = A; a.B = B; a.s = s; a.b = b; a.s16 = s16; a.b16 = b16;
   a.tiles_m = ceil_div(p.d_out, WT2_ROWS);
@@ -1038,7 +1079,14 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   if (const char* e = getenv("L4Q_WT_IMG")) { if (!atoi(e)) op_img = nullptr; }
 #endif
   if (op_img) {
-    k_split_operands<<<(a.tiles_n + a.tiles_m) * a.atoms * 4, 256, 0, st>>>(a, static_cast<uint8_t*>(op_img));
+    const int image_blocks = (a.tiles_n + a.tiles_m) * a.atoms * 4;
+    Bf16Copies cp{};
+    int copy_blocks = 0;
+    if (copies) {
+      cp = *copies;
+      copy_blocks = (int)(((long long)cp.rn * (p.d_in + p.d_out) / 8 + 255) / 256);
+    }
+    k_split_operands<<<image_blocks + copy_blocks, 256, 0, st>>>(a, static_cast<uint8_t*>(op_img), image_blocks, cp);
     if (cudaGetLastError() != cudaSuccess) return L4Q_ERR_CUDA;
     a.op_img = static_cast<const uint8_t*>(op_img);
   }
