@@ -592,6 +592,18 @@ def run_extras(args):
     n2 = cfg.rank * (cfg.d_in + cfg.d_out) + 2 * cfg.d_out * G
     us = timed("adamw", lambda k: l4q.l4q_adamw_step(p_[:n2], g_[:n2], m_[:n2], v_[:n2], k + 1, 1e-4), reps * 8)
     out["adamw_layer_params"] = {"us": us, "elements": n2, "bytes": 28 * n2}
+    # the same parameters as the four tensors they are (A, B, s, b), one launch each against one launch for all
+    sizes = [cfg.rank * cfg.d_in, cfg.d_out * cfg.rank, cfg.d_out * G, cfg.d_out * G]
+    offs = np.cumsum([0] + sizes)
+    views = [(p_[a:b], g_[a:b], m_[a:b], v_[a:b]) for a, b in zip(offs[:-1], offs[1:])]
+
+    def four_launches(k):
+        for t in views:
+            l4q.l4q_adamw_step(*t, k + 1, 1e-4)
+
+    us4 = timed("adamw", four_launches, reps * 8) * 4            # per-launch average x 4 launches
+    us1 = timed("adamw", lambda k: l4q.l4q_adamw_step_multi(views, k + 1, 1e-4), reps * 8)
+    out["adamw_layer_A_B_s_b"] = {"us_four_launches": us4, "us_one_launch": us1, "elements": int(offs[-1])}
 
     print(json.dumps({"op": "extras", "unit": "us per launch (CUDA events around each launch)", "hbm_peak_gbs": pk_["hbm_gbs"],
                       "peak_source": pk_["source"], "l2": "weights rotated over copies totalling 1.5x L2",

@@ -104,6 +104,11 @@ l4q_status l4q_linear_fwd(const l4q_desc* desc, const void* X, const void* W0,
  *   dB = gamma * (G*m) A^T                        (Eq. 14, App. A.2)
  * Any of dX, dA, dB, ds, db may be NULL to skip it (dA, dB, ds, db are produced
  * together: pass all four or none).  Outputs are overwritten.
+ * dA, dB, ds, db are sums over tiles of G that the bf16 path accumulates with fp32 atomic adds: their last bits
+ * depend on the order in which the tiles finish and differ from run to run (relative differences of ~1e-6, far
+ * inside the 3e-2 comparison tolerance).  There is no deterministic mode: it would need the per-tile partial sums
+ * in the workspace (d_out/128 copies of dA, d_in/256 copies of dB) and a second reduction pass over them, which is
+ * more memory traffic than the reduction itself.  dX and Y do not depend on any order.
  */
 l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, const void* W0,
                           const float* A, const float* B, const float* s, const float* b,
@@ -215,6 +220,23 @@ l4q_status l4q_quant_error(const l4q_desc* desc, const void* W0, const float* A,
  */
 l4q_status l4q_adamw_step(float* param, const float* grad, float* m, float* v, size_t n, int64_t step, float lr,
                           float beta1, float beta2, float eps, float weight_decay, void* cuda_stream);
+
+/*
+ * The same AdamW step (App. D) for up to 8 tensors in ONE launch: the trainable tensors of a layer (A, B, s, b)
+ * are small, and a launch per tensor is bound by the launch.  `tensors`: HOST array of `count` entries, each with
+ * DEVICE pointers to param, grad, m, v (fp32, n elements, n > 0); the entries are read during the call and need
+ * not outlive it.  All tensors take the same hyper-parameters and step.  Tensors must not overlap.
+ * L4Q_ERR_INVALID_ARG on count outside 1..8, a null pointer, n = 0, step < 1 or betas outside [0, 1).
+ */
+typedef struct {
+  float* param;
+  const float* grad;
+  float* m;
+  float* v;
+  size_t n;
+} l4q_adamw_tensor;
+l4q_status l4q_adamw_step_multi(const l4q_adamw_tensor* tensors, int count, int64_t step, float lr, float beta1,
+                                float beta2, float eps, float weight_decay, void* cuda_stream);
 
 /*
  * Forward pass for callers that cannot hand the library any scratch memory.

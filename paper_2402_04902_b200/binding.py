@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = (
     "l4q_profile_enable", "l4q_profile_read", "l4q_kernel_name",
     "l4q_linear_fwd_static", "l4q_init_params", "l4q_quant_error", "l4q_linear_infer", "l4q_adamw_step",
     "l4q_lora_workspace_bytes", "l4q_lora_linear_fwd", "l4q_lora_linear_bwd", "l4q_selftest_timeout",
-    "l4q_selftest_tile_copy",
+    "l4q_selftest_tile_copy", "l4q_adamw_step_multi",
 )
 L4Q_LORA_PLAIN, L4Q_LORA_QAT = 1, 2
 LORA_KINDS = {"lora": L4Q_LORA_PLAIN, "qat_lora": L4Q_LORA_QAT}
@@ -50,6 +50,13 @@ class L4QDesc(ctypes.Structure):
         ("bits", ctypes.c_int32), ("group_size", ctypes.c_int32),
         ("io_dtype", ctypes.c_int32), ("flags", ctypes.c_uint32), ("grad_scale", ctypes.c_float),
     ]
+
+
+class L4QAdamwTensor(ctypes.Structure):
+    """Mirror of ``l4q_adamw_tensor``."""
+
+    _fields_ = [("param", ctypes.c_void_p), ("grad", ctypes.c_void_p), ("m", ctypes.c_void_p), ("v", ctypes.c_void_p),
+                ("n", ctypes.c_size_t)]
 
 
 class L4QError(RuntimeError):
@@ -97,6 +104,9 @@ def lib() -> ctypes.CDLL:
         L.l4q_init_params.argtypes = [dp, vp, ctypes.c_int, fp, fp, vp]
         L.l4q_quant_error.restype = ctypes.c_int
         L.l4q_quant_error.argtypes = [dp, vp, fp, fp, fp, fp, vp, vp]
+        L.l4q_adamw_step_multi.restype = ctypes.c_int
+        L.l4q_adamw_step_multi.argtypes = [ctypes.POINTER(L4QAdamwTensor), ctypes.c_int, ctypes.c_int64, ctypes.c_float,
+                                           ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_float, vp]
         L.l4q_selftest_timeout.restype = ctypes.c_int
         L.l4q_selftest_timeout.argtypes = [vp]
         L.l4q_selftest_tile_copy.restype = ctypes.c_int
@@ -227,6 +237,20 @@ def l4q_adamw_step(param, grad, m, v, step: int, lr: float, beta1: float = 0.9, 
     st = lib().l4q_adamw_step(_ptr(param), _ptr(grad), _ptr(m), _ptr(v), param.numel(), int(step), float(lr),
                               float(beta1), float(beta2), float(eps), float(weight_decay), _stream(stream))
     _raise(st, "l4q_adamw_step")
+
+
+def l4q_adamw_step_multi(tensors, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                         weight_decay: float = 0.01, stream=None) -> None:
+    """In-place AdamW update (App. D) of up to 8 fp32 tensors in one launch; `tensors`: (param, grad, m, v) tuples."""
+    table = (L4QAdamwTensor * len(tensors))()
+    for k, (param, grad, m, v) in enumerate(tensors):
+        for t in (param, grad, m, v):
+            if t.dtype != torch.float32 or t.numel() != param.numel():
+                raise ValueError("AdamW tensors must be float32 and of one size per entry")
+        table[k] = L4QAdamwTensor(_ptr(param), _ptr(grad), _ptr(m), _ptr(v), param.numel())
+    st = lib().l4q_adamw_step_multi(table, len(tensors), int(step), float(lr), float(beta1), float(beta2), float(eps),
+                                    float(weight_decay), _stream(stream))
+    _raise(st, "l4q_adamw_step_multi")
 
 
 def l4q_init_params(desc: L4QDesc, W, method: str, s, b, stream=None) -> None:

@@ -147,7 +147,7 @@ l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const
                           const ZeroList* zero = nullptr, bool* zeroed = nullptr, const Bf16Copies* copies = nullptr,
                           bool* copied = nullptr) {
   if constexpr (IO_BF16) {
-    const int mode = fac ? WT2_DEQUANT_F : WT2_DEQUANT;
+    const int mode = fac ? (wq ? WT2_DEQUANT_F : WT2_FACTORS) : WT2_DEQUANT;
     if (wtile_tc_supported(p, mode)) {               // tensor-core merge, TMA in and out
       KernelScope ks(L4Q_KERNEL_DEQUANT, st);   // covers the operand split too, which is one more launch
       if (op_img) g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -322,7 +322,10 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
   if (!f32 && n_param_out == 4) copies = carve_copies(p, ws_tail + operand_image_bytes(desc, p));
   if (dX || fac) {
     st = f32 ? launch_dequant<false>(p, W0, A, B, s, b, wq, nullptr, stream)
-             : launch_dequant<true>(p, W0, A, B, s, b, wq, fac, stream, operand_image_bytes(desc, p) ? ws_tail : nullptr,
+             : launch_dequant<true>(p, W0, A, B, s, b,
+                                    // W_q is only needed for the input gradient (the plain-ALU kernel always writes it)
+                                    (dX || !wtile_tc_supported(p, WT2_FACTORS)) ? wq : nullptr, fac, stream,
+                                    operand_image_bytes(desc, p) ? ws_tail : nullptr,
                                     n_param_out == 4 ? &grads : nullptr, &zeroed, fac ? &copies : nullptr, &copied);
     if (st != L4Q_OK) return st;
   }
@@ -529,6 +532,29 @@ l4q_status l4q_adamw_step(float* param, const float* grad, float* m, float* v, s
   return launch_status();
 }
 
+l4q_status l4q_adamw_step_multi(const l4q_adamw_tensor* tensors, int count, int64_t step, float lr, float beta1,
+                                float beta2, float eps, float weight_decay, void* cuda_stream) {
+  if (!tensors || count < 1 || count > ADAMW_MAX_TENSORS || step < 1) return L4Q_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f) || !(lr == lr))
+    return L4Q_ERR_INVALID_ARG;
+  AdamwTable t{};
+  unsigned long long total = 0;
+  for (int k = 0; k < count; ++k) {
+    const l4q_adamw_tensor& x = tensors[k];
+    if (!x.param || !x.grad || !x.m || !x.v || x.n == 0) return L4Q_ERR_INVALID_ARG;
+    t.param[k] = x.param; t.grad[k] = x.grad; t.m[k] = x.m; t.v[k] = x.v;
+    total += x.n;
+    t.end[k] = total;
+  }
+  t.count = count;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const double c1 = 1.0 - std::pow((double)beta1, (double)step), c2 = 1.0 - std::pow((double)beta2, (double)step);
+  const int blocks = (int)std::min<unsigned long long>((total + 255) / 256, (unsigned long long)sm_count() * 8);
+  KernelScope ks(L4Q_KERNEL_ADAMW, stream);
+  k_adamw_multi<<<blocks, 256, 0, stream>>>(t, lr, beta1, beta2, eps, weight_decay, (float)(1.0 / c1), (float)(1.0 / c2));
+  return launch_status();
+}
+
 l4q_status l4q_init_params(const l4q_desc* desc, const void* W, int method, float* s, float* b, void* cuda_stream) {
   l4q_desc d2;
   if (!desc) return L4Q_ERR_INVALID_ARG;
@@ -570,6 +596,11 @@ l4q_status l4q_quant_error(const l4q_desc* desc, const void* W0, const float* A,
   if (!aligned16(W0) || !aligned16(A) || (reinterpret_cast<uintptr_t>(errors) & 7u)) return L4Q_ERR_INVALID_ARG;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(errors, 0, 2 * sizeof(double), stream) != cudaSuccess) return L4Q_ERR_CUDA;
+  if (desc->io_dtype == L4Q_BF16 && wtile_tc_supported(p, WT2_ERROR)) {   // tensor-core merge, W0 by TMA; no scratch:
+    KernelScope ks(L4Q_KERNEL_ERROR, stream);                              // one warp builds the merge operands
+    return launch_wtile_tc(WT2_ERROR, p, W0, A, B, s, b, nullptr, nullptr, nullptr, nullptr, stream, nullptr, nullptr,
+                           nullptr, nullptr, errors);
+  }
   const size_t smem = weight_tile_smem_bytes(p.rank);
   dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
   auto launch = [&](auto kern) -> l4q_status {

@@ -316,4 +316,38 @@ k_adamw(float* __restrict__ param, const float* __restrict__ grad, float* __rest
   }
 }
 
+// The same update for several tensors in one launch (the four trainable tensors of a layer -- A, B, s, b -- are
+// small: one launch each is bound by the launch, not by memory).  Element e of the concatenation of the tensors
+// belongs to the tensor whose [begin, end) holds it; a thread finds it by scanning the (at most 8) ends.
+constexpr int ADAMW_MAX_TENSORS = 8;
+struct AdamwTable {
+  float* param[ADAMW_MAX_TENSORS];
+  const float* grad[ADAMW_MAX_TENSORS];
+  float* m[ADAMW_MAX_TENSORS];
+  float* v[ADAMW_MAX_TENSORS];
+  unsigned long long end[ADAMW_MAX_TENSORS];   // running totals of the element counts
+  int count;
+};
+
+__global__ void __launch_bounds__(256)
+k_adamw_multi(const AdamwTable t, float lr, float beta1, float beta2, float eps, float weight_decay, float inv_c1,
+              float inv_c2) {
+  const unsigned long long total = t.end[t.count - 1];
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  for (unsigned long long e = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+    int k = 0;
+#pragma unroll
+    for (int j = 0; j < ADAMW_MAX_TENSORS - 1; ++j) k += (j < t.count - 1 && e >= t.end[j]) ? 1 : 0;
+    const size_t i = (size_t)(e - (k ? t.end[k - 1] : 0ull));
+    const float g = t.grad[k][i];
+    float p = t.param[k][i];
+    p = fmaf(-lr * weight_decay, p, p);
+    const float mi = fmaf(beta1, t.m[k][i], (1.f - beta1) * g);
+    const float vi = fmaf(beta2, t.v[k][i], (1.f - beta2) * g * g);
+    t.m[k][i] = mi;
+    t.v[k][i] = vi;
+    t.param[k][i] = p - lr * (mi * inv_c1) / (sqrtf(vi * inv_c2) + eps);
+  }
+}
+
 }  // namespace l4q

@@ -4,6 +4,8 @@
 //   WT2_DEQUANT_F  W_q (bf16) + STE factors (fp16) -- backward: input gradient + weight-gradient reduction
 //                  (the factors leave from registers, 16 bytes per thread and 8-column piece, coalesced)
 //   WT2_PACK       bit-packed codes + fp16 s, b    -- export (Sec. 3.2)
+//   WT2_FACTORS    STE factors alone               -- backward without the input gradient: W_q is not needed
+//   WT2_ERROR      E_quant, E_clip (two sums)      -- the quantization-error metric of Table 4; nothing else is written
 //
 // HBM-bound by design (2 bytes in, 0.4-4 bytes out per weight), so everything else is arranged to stay out
 // of the way of the copies:
@@ -59,7 +61,9 @@ constexpr int WT2_MAX_STAGES = 6;
 constexpr int WT2_MAX_BSLOTS = 8;
 constexpr int WT2_MAX_ATOMS = 4;                    // rank <= 64
 
-enum { WT2_DEQUANT = 0, WT2_DEQUANT_F = 1, WT2_PACK = 2 };
+enum { WT2_DEQUANT = 0, WT2_DEQUANT_F = 1, WT2_PACK = 2, WT2_ERROR = 3, WT2_FACTORS = 4 };
+__host__ __device__ constexpr bool wt2_has_factors(int mode) { return mode == WT2_DEQUANT_F || mode == WT2_FACTORS; }
+__host__ __device__ constexpr bool wt2_has_wq(int mode) { return mode == WT2_DEQUANT || mode == WT2_DEQUANT_F; }
 
 // Output buffers of the caller that must start from zero (they are accumulated into with atomics later on the
 // stream): cleared by a launch that runs anyway, which saves one memset launch per buffer.
@@ -78,6 +82,7 @@ struct WtileArgs {
   const float *A, *B, *s, *b;
   __half *s16, *b16;       // WT2_PACK
   __half* F;               // WT2_DEQUANT_F: the factor array (factor_index layout)
+  double* errors;          // WT2_ERROR: E_quant, E_clip (accumulated with fp64 atomics; zero on entry)
   ZeroList zero;           // buffers this launch clears before anything else (all sizes 0: none)
   const uint8_t* op_img;   // optional: the split MMA operands of every panel, ready made (see k_split_operands)
   int tiles_m, tiles_n;
@@ -379,7 +384,8 @@ struct FastConsts {
 // WT2_PACK (unsigned grid only): the code words go to `out1` (the tile's staging rows).
 template <int MODE, int BITS>
 __device__ __forceinline__ void wtile_half_row_fast(const FastConsts& c, uint32_t taddr, uint8_t* tile_row, int row,
-                                                    int chalf, uint8_t* out1, uint64_t* tmem_empty_bar) {
+                                                    int chalf, uint8_t* out1, uint64_t* tmem_empty_bar,
+                                                    float& e_quant, float& e_clip) {
   const float2 gamma2 = make_float2(c.gamma, c.gamma), nb2 = make_float2(-c.b, -c.b), rs2 = make_float2(c.rs, c.rs);
   const float2 magic2 = make_float2(kRoundMagic, kRoundMagic);
   [[maybe_unused]] const float2 nmagic2 = make_float2(-kRoundMagic, -kRoundMagic);
@@ -419,7 +425,13 @@ __device__ __forceinline__ void wtile_half_row_fast(const FastConsts& c, uint32_
           const float2 code = __fadd2_rn(y, nmagic2);
           const float2 wq = __ffma2_rn(code, s2v, b2v);
           qo[e] = pack_bf16x2(wq.x, wq.y);
-          if constexpr (MODE == WT2_DEQUANT_F) {
+          if constexpr (MODE == WT2_ERROR) {                                       // |W_comb - W_q|, and its part outside the range
+            const float2 t2 = __fadd2_rn(w, make_float2(-wcl.x, -wcl.y));
+            const float ex = fabsf(wc.x - wq.x), ey = fabsf(wc.y - wq.y);
+            e_quant += ex + ey;
+            e_clip += (fabsf(t2.x) > kMaskGuard ? ex : 0.f) + (fabsf(t2.y) > kMaskGuard ? ey : 0.f);
+          }
+          if constexpr (wt2_has_factors(MODE)) {
             const float2 t2 = __fadd2_rn(w, make_float2(-wcl.x, -wcl.y));          // 0 inside [Q_N, Q_P]
             const float2 inr = __fadd2_rn(code, make_float2(-w.x, -w.y));          // w~ - w
             const float tt[2] = {t2.x, t2.y}, ii[2] = {inr.x, inr.y};
@@ -450,9 +462,9 @@ __device__ __forceinline__ void wtile_half_row_fast(const FastConsts& c, uint32_
           }
         }
       }
-      if constexpr (MODE != WT2_PACK)
+      if constexpr (wt2_has_wq(MODE))
         *reinterpret_cast<uint4*>(tile_row + chunk) = make_uint4(qo[0], qo[1], qo[2], qo[3]);   // in place
-      if constexpr (MODE == WT2_DEQUANT_F)
+      if constexpr (wt2_has_factors(MODE))
         *reinterpret_cast<uint4*>(out1 + (piece * WT2_ROWS + row) * 16) = make_uint4(fo[0], fo[1], fo[2], fo[3]);
       // staging row = the tile's 128 codes of this weight row; this thread writes 64 of them, 32 at a time
       if constexpr (MODE == WT2_PACK && BITS == 4) {
@@ -538,13 +550,14 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
   const Params& p = a.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr bool HAS_OUT1 = (MODE == WT2_PACK);      // staged in shared memory: the code words of the export
+  constexpr bool READ_ONLY = !wt2_has_wq(MODE);      // W0 stages are read, never written back
 
   if (threadIdx.x == 0) {
     const uint32_t op_arrivals = a.op_img ? 1 : WT2_BUILDERS;   // one thread announcing a bulk copy, or the builders of the atom
     for (int i = 0; i < WT2_MAX_STAGES; ++i) {
       ptx::mbar_init(&bars->full[i], 1);
       // the export does not write back into the stage: the group that read it hands it back itself
-      ptx::mbar_init(&bars->empty[i], MODE == WT2_PACK ? WT2_GROUP_THREADS : 1);
+      ptx::mbar_init(&bars->empty[i], READ_ONLY ? WT2_GROUP_THREADS : 1);
       ptx::mbar_init(&bars->written[i], WT2_GROUP_THREADS);
     }
     for (int i = 0; i < WT2_GROUPS; ++i) ptx::mbar_init(&bars->out_empty[i], 1);
@@ -629,7 +642,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     // Two issuing threads, one per epilogue group (tiles sid, sid + 2, ...): a thread hands a stage back only
     // after its copy has read it, which takes the TMA unit a thousand cycles or more behind the loads queued
     // before it, and one thread doing that for every tile in turn was the slowest role of the kernel.
-    if (lane == 0) {
+    if (lane == 0 && (wt2_has_wq(MODE) || MODE == WT2_PACK)) {
       const int sid = warp == 2 ? 0 : 1;
       StageSeq sq(sid, a.n_stages);
       const int ob = sid;                            // the group's own staging buffer of code words
@@ -640,7 +653,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
         const uint8_t* src = stage_base + (size_t)stage * WT2_STAGE_BYTES;
         const uint8_t* src1 = out_base + (size_t)ob * a.out_bytes;
         const bool second_box = n0 + 64 < p.d_in;
-        if constexpr (MODE != WT2_PACK) {
+        if constexpr (!READ_ONLY) {
           ptx::tma_store_2d(&tmap_out0, src, n0, m0);
           if (second_box) ptx::tma_store_2d(&tmap_out0, src + WT2_STAGE_BYTES / 2, n0 + 64, m0);
         }
@@ -649,7 +662,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
         // hand the buffers back as soon as the copies have read them: a stage that is released a tile later is a
         // load that starts a tile later
         ptx::bulk_wait_group_read0();
-        if constexpr (MODE != WT2_PACK) ptx::mbar_arrive(&bars->empty[stage]);
+        if constexpr (!READ_ONLY) ptx::mbar_arrive(&bars->empty[stage]);
         if constexpr (HAS_OUT1) ptx::mbar_arrive(&bars->out_empty[ob]);
         sq.advance();
       }
@@ -751,6 +764,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
     }
     int sb_buf = 0;
     const int qn_bits = kRoundMagicBits + (int)p.qn;
+    [[maybe_unused]] float e_quant = 0.f, e_clip = 0.f;         // WT2_ERROR: this thread's partial sums
 
     // the group's own W0 stages and staging buffer of code words (no division per tile: that is dozens of
     // instructions, on warps whose issue slots are the scarce thing here)
@@ -796,7 +810,7 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       // second output: the export's staging rows in shared memory; the STE factors go straight to the tile's block
       // of the factor array in global memory (16 bytes per thread and piece, a warp's 32 rows contiguous)
       [[maybe_unused]] uint8_t* out1 =
-          MODE == WT2_DEQUANT_F
+          wt2_has_factors(MODE)
               ? reinterpret_cast<uint8_t*>(a.F + ((size_t)cur.tm * a.tiles_n + cur.tn) * FACTOR_TILE_ELEMS)
               : out_base + (size_t)ob * a.out_bytes;
       if (interior(m0, n0)) {
@@ -806,15 +820,15 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
         fc.qn = p.qn; fc.qp = p.qp; fc.gamma = p.gamma;
         const uint32_t taddr = tmem_base + lane_base + (uint32_t)(acc * WT2_COLS + chalf * 64);
         if constexpr (MODE == WT2_PACK) {
-          if (p.bits == 4) wtile_half_row_fast<MODE, 4>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc]);
-          else wtile_half_row_fast<MODE, 3>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc]);
+          if (p.bits == 4) wtile_half_row_fast<MODE, 4>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc], e_quant, e_clip);
+          else wtile_half_row_fast<MODE, 3>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc], e_quant, e_clip);
           const int g = group_of(a, n0 + chalf * 64);
           if ((n0 + chalf * 64) - g * p.group == 0) {             // first half row of its group
             a.s16[(size_t)o * p.ngroups + g] = __float2half_rn(fc.s);
             a.b16[(size_t)o * p.ngroups + g] = __float2half_rn(fc.b);   // Q_N = 0: b + s Q_N = b
           }
         } else {
-          wtile_half_row_fast<MODE, 4>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc]);
+          wtile_half_row_fast<MODE, 4>(fc, taddr, tile_rows, row, chalf, out1, &bars->tmem_empty[acc], e_quant, e_clip);
         }
       } else {
       float rs = 1.f, s_ = 1.f, b_ = 0.f;
@@ -867,7 +881,15 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
               const float2 code = __fadd2_rn(y, nmagic2);
               const float2 q = __ffma2_rn(code, s2v, b2v);
               wq[e] = q.x; wq[e + 1] = q.y;
-              if constexpr (MODE == WT2_DEQUANT_F) {
+              if constexpr (MODE == WT2_ERROR) {
+                if (ok) {                                                           // |W_comb - W_q|, and its part outside the range
+                  const float2 t2 = __fadd2_rn(w, make_float2(-wcl.x, -wcl.y));
+                  const float ex = fabsf(wc.x - q.x), ey = fabsf(wc.y - q.y);
+                  e_quant += ex + ey;
+                  e_clip += (fabsf(t2.x) > kMaskGuard ? ex : 0.f) + (fabsf(t2.y) > kMaskGuard ? ey : 0.f);
+                }
+              }
+              if constexpr (wt2_has_factors(MODE)) {
                 const float2 t2 = __fadd2_rn(w, make_float2(-wcl.x, -wcl.y));                 // 0 inside [Q_N, Q_P]
                 const float2 inr = __fadd2_rn(code, make_float2(-w.x, -w.y));                 // code - w
                 const float tt[2] = {t2.x, t2.y}, ii[2] = {inr.x, inr.y};
@@ -893,13 +915,13 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
                 }
               }
             }
-            if constexpr (MODE != WT2_PACK) {
+            if constexpr (wt2_has_wq(MODE)) {
               uint4 o4;
               o4.x = pack_bf16x2(wq[0], wq[1]); o4.y = pack_bf16x2(wq[2], wq[3]);
               o4.z = pack_bf16x2(wq[4], wq[5]); o4.w = pack_bf16x2(wq[6], wq[7]);
               *reinterpret_cast<uint4*>(tile_rows + chunk) = o4;                    // in place, same swizzled position
             }
-            if constexpr (MODE == WT2_DEQUANT_F) {
+            if constexpr (wt2_has_factors(MODE)) {
               __half2 h[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) h[e] = __floats2half2_rn(fac[2 * e], fac[2 * e + 1]);
@@ -926,11 +948,22 @@ k_wtile_tc(const __grid_constant__ CUtensorMap tmap_w0,     // load:  W0 [d_out,
       }
       ptx::fence_proxy_async_smem();                   // the stores above are read by TMA
       ptx::mbar_arrive(&bars->written[stage]);
-      if constexpr (MODE == WT2_PACK) ptx::mbar_arrive(&bars->empty[stage]);   // W0 has been read
+      if constexpr (READ_ONLY) ptx::mbar_arrive(&bars->empty[stage]);   // W0 has been read
       sb_buf ^= 1;
       if (has_next) stage_sb(m1, n1, sb_buf);          // the other buffer: its readers passed this tile's barrier
       sq.advance();
       ++ob_uses;
+    }
+    if constexpr (MODE == WT2_ERROR) {                 // the warp's partial sums, then one fp64 atomic per warp and sum
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        e_quant += __shfl_xor_sync(0xffffffffu, e_quant, off);
+        e_clip += __shfl_xor_sync(0xffffffffu, e_clip, off);
+      }
+      if (lane == 0) {
+        atomicAdd(a.errors, (double)e_quant);
+        atomicAdd(a.errors + 1, (double)e_clip);
+      }
     }
   }
 
@@ -978,7 +1011,7 @@ inline bool wtile_plan(WtileArgs& a, int mode, bool sb_by_tma = true) {
   for (int sh = 3; sh < 31; ++sh)
     if ((1 << sh) == p.group) a.group_shift = sh;
   // (the export's fast path builds its code words from the raw rounding results, which it does for the unsigned grid)
-  a.fast = (p.group % 64 == 0 && (mode != WT2_PACK || (p.qn == 0.f && (p.bits == 3 || p.bits == 4)))) ? 1 : 0;
+  a.fast = (p.group % 64 == 0 && (mode != WT2_PACK || (p.qn == 0.f && (p.bits == 3 || p.bits == 4)))) ? 1 : 0;   // (WT2_ERROR: as the dequantize modes)
   // a box starts at a group column that is a multiple of 4 (16 bytes) at or below the tile's first group, so it
   // is up to 3 groups wider than the tile; the row pitch of s and b must be a multiple of 16 bytes
   const int box = (a.ngt + 3 + 3) / 4 * 4;
@@ -1028,6 +1061,7 @@ inline bool wtile_tc_supported(const Params& p, int mode) {
 }
 
 // mode WT2_DEQUANT: out0 = W_q.  WT2_DEQUANT_F: out0 = W_q, out1 = STE factors.  WT2_PACK: out0 = codes.
+// WT2_ERROR: no outputs but `errors` (two doubles, zero on entry).
 // Bytes of the operand images of a problem (see k_split_operands).
 inline size_t wtile_image_bytes(const Params& p) {
   const size_t atoms = (2 * (size_t)p.rank + 31) / 32;
@@ -1041,9 +1075,9 @@ inline size_t wtile_image_bytes(const Params& p) {
 inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, const float* A, const float* B,
                                   const float* s, const float* b, void* out0, void* out1, __half* s16, __half* b16,
                                   cudaStream_t st, void* op_img = nullptr, const ZeroList* zero = nullptr,
-                                  bool* zeroed = nullptr, const Bf16Copies* copies = nullptr) {
+                                  bool* zeroed = nullptr, const Bf16Copies* copies = nullptr, double* errors = nullptr) {
   WtileArgs a{};
-  a.p = p; a.A = A; a.B = B; a.s = s; a.b = b; a.s16 = s16; a.b16 = b16;
+  a.p = p; a.A = A; a.B = B; a.s = s; a.b = b; a.s16 = s16; a.b16 = b16; a.errors = errors;
   a.tiles_m = ceil_div(p.d_out, WT2_ROWS);
   a.tiles_n = ceil_div(p.d_in, WT2_COLS);
   const bool sb_aligned = ((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(b)) & 15u) == 0;
@@ -1054,6 +1088,9 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   if (mode == WT2_PACK) {
     if (!make_tmap_words(&t_o0, out0, p.d_out, ((uint64_t)p.d_in * p.bits) >> 5, WT2_COLS * p.bits / 32))
       return L4Q_ERR_CUDA;
+  } else if (mode == WT2_ERROR || mode == WT2_FACTORS) {
+    t_o0 = t_w0;                                    // nothing is stored by TMA
+    a.F = reinterpret_cast<__half*>(out1);
   } else {
     if (!make_tmap_bf16(&t_o0, out0, p.d_out, p.d_in, WT2_ROWS)) return L4Q_ERR_CUDA;
     a.F = reinterpret_cast<__half*>(out1);
@@ -1113,6 +1150,8 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   switch (mode) {
     case WT2_DEQUANT: return launch(k_wtile_tc<WT2_DEQUANT>);
     case WT2_DEQUANT_F: return launch(k_wtile_tc<WT2_DEQUANT_F>);
+    case WT2_ERROR: return launch(k_wtile_tc<WT2_ERROR>);
+    case WT2_FACTORS: return launch(k_wtile_tc<WT2_FACTORS>);
     default: return launch(k_wtile_tc<WT2_PACK>);
   }
 }
