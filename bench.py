@@ -361,7 +361,7 @@ def run_ours(args, layers, wl_name):
     value = world * flops_step_rank / (ms_step * 1e-3) / 1e12
 
     # ---- the same step for at least 1.5 s: the GPU reaches its power cap and settles at its sustained clock ----
-    n_sus = max(args.steps, int(1500.0 / ms_step) + 1)
+    n_sus = max(args.steps, int(args.sustained_seconds * 1e3 / ms_step) + 1)
     with ClockSampler(local_rank) as clk_sus:
         ms_sus = timed(False, n_sus, 0) / n_sus
     sus_value = world * flops_step_rank / (ms_sus * 1e-3) / 1e12
@@ -619,6 +619,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layer", default="l4q", choices=["l4q", "lora", "qat_lora"],
                     help="l4q = the benchmark; lora / qat_lora = the comparison layers (ours arm only)")
+    ap.add_argument("--sustained-seconds", type=float, default=1.5,
+                    help="length of the second, sustained timed region (0: as many steps as --steps; for profiler captures)")
     ap.add_argument("--op", default="train", choices=["train", "extras"],
                     help="train = the benchmark; extras = inference / initialisation / error sums / AdamW kernels")
     args = ap.parse_args()

@@ -392,21 +392,27 @@ __device__ __forceinline__ void wtile_half_row_fast(const FastConsts& c, uint32_
   [[maybe_unused]] const float2 s2v = make_float2(c.s, c.s), b2v = make_float2(c.b, c.b);
   [[maybe_unused]] uint32_t words[4];                                           // BITS == 4: four words = 32 codes
   [[maybe_unused]] uint32_t h3[3] = {0u, 0u, 0u}, carry10 = 0u, carry21 = 0u;   // BITS == 3: 32 codes -> 3 words
+  // The 64 columns in two rounds of 32 (a loop, not unrolled: the straight-line code of all 64 is several times
+  // the instruction cache of a scheduler, and two groups run it at different places), each round two TMEM loads
+  // of 16 columns, the second in flight while the first is worked on.
+#pragma unroll 1
+  for (int hq = 0; hq < 2; ++hq) {
   uint32_t raw[2][16];
-  ptx::tmem_ld_32x16(taddr, raw[0]);
+  ptx::tmem_ld_32x16(taddr + (uint32_t)(hq * 32), raw[0]);
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {                       // 16 columns
+  for (int ql = 0; ql < 2; ++ql) {                    // 16 columns
     ptx::tmem_ld_wait();
-    if (q < 3) {
-      ptx::tmem_ld_32x16(taddr + (uint32_t)((q + 1) * 16), raw[(q + 1) & 1]);
-    } else {                                          // all of the thread's merge columns are in registers
+    if (ql == 0) {
+      ptx::tmem_ld_32x16(taddr + (uint32_t)(hq * 32 + 16), raw[1]);
+    } else if (hq == 1) {                             // all of the thread's merge columns are in registers
       ptx::tc_fence_before_sync();
       ptx::mbar_arrive(tmem_empty_bar);
     }
-    const uint32_t(&acc)[16] = raw[q & 1];
+    const uint32_t(&acc)[16] = raw[ql];
 #pragma unroll
     for (int s2 = 0; s2 < 2; ++s2) {
-      const int pin = q * 2 + s2;                     // piece of the half row
+      const int pl = ql * 2 + s2;                     // piece of the round (static), of the half row:
+      const int pin = hq * 4 + pl;
       const int piece = chalf * 8 + pin;              // piece of the tile row (chalf selects the 64-column box)
       const uint32_t chunk = (uint32_t)((piece >> 3) * (WT2_STAGE_BYTES / 2) + (((piece & 7) ^ (row & 7)) << 4));
       const uint4 wr = *reinterpret_cast<const uint4*>(tile_row + chunk);
@@ -452,7 +458,7 @@ __device__ __forceinline__ void wtile_half_row_fast(const FastConsts& c, uint32_
               const int j = 2 * e + h;                                           // code j of the word at bit 4 j
               word4 = (j == 0) ? yb[h] : word4 + (yb[h] << (4 * j));
             } else {
-              const int j = (pin & 3) * 8 + 2 * e + h;                           // code j of 32 at bit 3 j of 3 words
+              const int j = pl * 8 + 2 * e + h;                                  // code j of 32 at bit 3 j of 3 words
               if (j < 10) h3[0] += yb[h] << (3 * j);
               else if (j == 10) carry10 = yb[h] & 7u;
               else if (j < 21) h3[1] += yb[h] << (3 * (j - 11) + 1);
@@ -468,14 +474,14 @@ __device__ __forceinline__ void wtile_half_row_fast(const FastConsts& c, uint32_
         *reinterpret_cast<uint4*>(out1 + (piece * WT2_ROWS + row) * 16) = make_uint4(fo[0], fo[1], fo[2], fo[3]);
       // staging row = the tile's 128 codes of this weight row; this thread writes 64 of them, 32 at a time
       if constexpr (MODE == WT2_PACK && BITS == 4) {
-        words[pin & 3] = word4 - magic_bias(8, 4);
-        if ((pin & 3) == 3)
-          *reinterpret_cast<uint4*>(out1 + row * 64 + chalf * 32 + (pin >> 2) * 16) =
+        words[pl] = word4 - magic_bias(8, 4);
+        if (pl == 3)
+          *reinterpret_cast<uint4*>(out1 + row * 64 + chalf * 32 + hq * 16) =
               make_uint4(words[0], words[1], words[2], words[3]);
       }
       if constexpr (MODE == WT2_PACK && BITS == 3) {
-        if ((pin & 3) == 3) {
-          uint32_t* dst = reinterpret_cast<uint32_t*>(out1 + row * 48 + chalf * 24 + (pin >> 2) * 12);
+        if (pl == 3) {
+          uint32_t* dst = reinterpret_cast<uint32_t*>(out1 + row * 48 + chalf * 24 + hq * 12);
           dst[0] = (h3[0] - magic_bias(10, 3)) + (carry10 << 30);
           dst[1] = (h3[1] - (magic_bias(10, 3) << 1)) + (carry10 >> 2) + (carry21 << 31);
           dst[2] = (h3[2] - (magic_bias(10, 3) << 2)) + (carry21 >> 1);
@@ -483,6 +489,7 @@ __device__ __forceinline__ void wtile_half_row_fast(const FastConsts& c, uint32_
         }
       }
     }
+  }
   }
 }
 
