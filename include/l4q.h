@@ -59,6 +59,7 @@ typedef enum {
 
 enum { L4Q_BF16 = 0, L4Q_F32 = 1 };                 /* io_dtype */
 enum { L4Q_OP_FWD = 0, L4Q_OP_BWD = 1, L4Q_OP_PACK = 2 };
+#define L4Q_MAX_RANK 128   /* largest LoRA rank any entry point takes (else L4Q_ERR_UNSUPPORTED) */
 enum {
   L4Q_FLAG_SIGNED_GRID = 1u   /* codes in [-2^(bits-1), 2^(bits-1)-1] as in Eq. 3 */
 };
@@ -68,7 +69,7 @@ typedef struct l4q_desc {
   int64_t  tokens;      /* rows of X / Y                                                   */
   int64_t  d_in;        /* i: columns of W0; multiple of group_size                        */
   int64_t  d_out;       /* o: rows of W0                                                   */
-  int32_t  rank;        /* r of the LoRA factors                                           */
+  int32_t  rank;        /* r of the LoRA factors, 1..L4Q_MAX_RANK                          */
   float    alpha;       /* LoRA constant; the merge uses gamma = alpha / rank              */
   int32_t  bits;        /* n: 2..8 for fwd/bwd, 3 or 4 for l4q_pack_int                    */
   int32_t  group_size;  /* g: quantization group along d_in; multiple of 8                 */

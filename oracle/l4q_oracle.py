@@ -16,8 +16,7 @@ Layout (row-major, tokens flattened; the paper writes column vectors,
     s, b [o, i/g]  scale / offset of each group of g consecutive elements
                    of a weight row (groups run along d_in)
 
-Readings taken where the paper is silent (each is also listed in the design
-notes of the repository):
+Readings taken where the paper is silent or needs a finite-precision rule:
   * the paper's constant "alpha" in Eq. 7 is ``gamma = alpha / rank`` here;
   * round() is round-half-to-even;
   * the integer grid is [Q_N, Q_P] = [-2^(n-1), 2^(n-1)-1] as in Eq. 3 when
@@ -36,7 +35,8 @@ Pinned by tests/test_oracle_pins.py and tests/test_oracle_init_pins.py
 against: B = 0 => merge == W0; grid membership; zero clipping under the
 Asymm / L4Q_init initialisations (Table 4, "Initial" E_clip = 0.0); the LoRA
 limits of Eq. 1-2; finite differences of the STE surrogate; a hand-worked
-example; scalar brute force on tiny layers; pack/unpack round trips.
+example; scalar brute force on tiny layers; pack/unpack round trips; the
+printed gate of App. A.1 (guard band 0) away from the bounds.
 """
 from __future__ import annotations
 

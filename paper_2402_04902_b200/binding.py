@@ -22,6 +22,7 @@ L4Q_OK = 0
 L4Q_BF16, L4Q_F32 = 0, 1
 L4Q_OP_FWD, L4Q_OP_BWD, L4Q_OP_PACK = 0, 1, 2
 L4Q_FLAG_SIGNED_GRID = 1
+L4Q_MAX_RANK = 128
 
 EXPORTED_SYMBOLS = (
     "l4q_workspace_bytes", "l4q_linear_fwd", "l4q_linear_bwd", "l4q_pack_int",

@@ -79,7 +79,7 @@ l4q_status make_params(const l4q_desc* d, Params* p) {
   if (d->bits < 2 || d->bits > 8) return L4Q_ERR_UNSUPPORTED;
   if (d->d_in % d->group_size != 0) return L4Q_ERR_UNSUPPORTED;
   if (d->group_size % 8 != 0 || d->d_in % 8 != 0) return L4Q_ERR_UNSUPPORTED;
-  if (d->rank > 256) return L4Q_ERR_UNSUPPORTED;
+  if (d->rank > L4Q_MAX_RANK) return L4Q_ERR_UNSUPPORTED;   // the plain-ALU weight-tile kernel keeps rank x 320 floats in shared memory
   if (d->io_dtype == L4Q_BF16 && d->d_out % 8 != 0) return L4Q_ERR_UNSUPPORTED;
   p->tokens = (int)d->tokens; p->d_in = (int)d->d_in; p->d_out = (int)d->d_out;
   p->rank = d->rank; p->bits = d->bits; p->group = d->group_size;
@@ -160,7 +160,7 @@ l4q_status launch_dequant(const Params& p, const void* W0, const float* A, const
   auto kern = k_weight_tile<IO_BF16, WT_MODE_DEQUANT>;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
   KernelScope ks(L4Q_KERNEL_DEQUANT, st);
   kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, wq, fac, nullptr, nullptr, nullptr, nullptr);
@@ -182,7 +182,7 @@ l4q_status launch_pack(const Params& p, const void* W0, const float* A, const fl
   auto kern = k_weight_tile<IO_BF16, WT_MODE_PACK>;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   dim3 grid(ceil_div(p.d_in, WT_COLS), ceil_div(p.d_out, WT_ROWS));
   KernelScope ks(L4Q_KERNEL_PACK, st);
   kern<<<grid, WT_THREADS, smem, st>>>(p, W0, A, B, s, b, nullptr, nullptr, codes, s16, b16, nullptr);
@@ -334,7 +334,7 @@ l4q_status l4q_linear_bwd(const l4q_desc* desc, const void* X, const void* dY, c
         cudaMemsetAsync(dB, 0, grads.n[1] * sizeof(float), stream) != cudaSuccess ||
         cudaMemsetAsync(ds, 0, grads.n[2] * sizeof(float), stream) != cudaSuccess ||
         cudaMemsetAsync(db, 0, grads.n[3] * sizeof(float), stream) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
   }
   if (f32) {
     if (dX) {
@@ -394,7 +394,7 @@ l4q_status l4q_lora_linear_fwd(const l4q_desc* desc, int kind, const void* X, co
   const void* W = W0;
   if (qat) {
     if (cudaMemsetAsync(w.zero_B, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     if ((st = launch_dequant<true>(p, W0, A, w.zero_B, s, b, w.wq, nullptr, stream, w.op_img)) != L4Q_OK) return st;
     W = w.wq;
   }
@@ -432,7 +432,7 @@ l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, co
   const void* W = W0;
   if (qat && (dX || ds)) {
     if (cudaMemsetAsync(w.zero_B, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     if ((st = launch_dequant<true>(p, W0, A, w.zero_B, s, b, w.wq, ds ? w.fac : nullptr, stream, w.op_img)) != L4Q_OK)
       return st;
     W = w.wq;
@@ -452,7 +452,7 @@ l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, co
   if (dA) {
     if (cudaMemsetAsync(dA, 0, (size_t)p.rank * p.d_in * sizeof(float), stream) != cudaSuccess ||
         cudaMemsetAsync(dB, 0, (size_t)p.d_out * p.rank * sizeof(float), stream) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     {
       KernelScope ks(L4Q_KERNEL_LORA_SIDE, stream);                                  // Xt = X A^T, recomputed
       if ((st = gemm_lora_down_bf16(p, X, w.v, stream)) != L4Q_OK) return st;
@@ -467,7 +467,7 @@ l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, co
   if (qat && ds) {
     const size_t gsz = (size_t)p.d_out * p.ngroups * sizeof(float);
     if (cudaMemsetAsync(ds, 0, gsz, stream) != cudaSuccess || cudaMemsetAsync(db, 0, gsz, stream) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     const Bf16Copies cp = carve_copies(p, w.copies);
     if ((st = launch_copies(p, A, w.zero_B, cp, stream)) != L4Q_OK) return st;
     KernelScope ks(L4Q_KERNEL_GEMM_WGRAD, stream);
@@ -595,7 +595,7 @@ l4q_status l4q_quant_error(const l4q_desc* desc, const void* W0, const float* A,
   if (!W0 || !A || !B || !s || !b || !errors) return L4Q_ERR_INVALID_ARG;
   if (!aligned16(W0) || !aligned16(A) || (reinterpret_cast<uintptr_t>(errors) & 7u)) return L4Q_ERR_INVALID_ARG;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (cudaMemsetAsync(errors, 0, 2 * sizeof(double), stream) != cudaSuccess) return L4Q_ERR_CUDA;
+  if (cudaMemsetAsync(errors, 0, 2 * sizeof(double), stream) != cudaSuccess) return cuda_fail();
   if (desc->io_dtype == L4Q_BF16 && wtile_tc_supported(p, WT2_ERROR)) {   // tensor-core merge, W0 by TMA; no scratch:
     KernelScope ks(L4Q_KERNEL_ERROR, stream);                              // one warp builds the merge operands
     return launch_wtile_tc(WT2_ERROR, p, W0, A, B, s, b, nullptr, nullptr, nullptr, nullptr, stream, nullptr, nullptr,
@@ -606,7 +606,7 @@ l4q_status l4q_quant_error(const l4q_desc* desc, const void* W0, const float* A,
   auto launch = [&](auto kern) -> l4q_status {
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     KernelScope ks(L4Q_KERNEL_ERROR, stream);
     kern<<<grid, WT_THREADS, smem, stream>>>(p, W0, A, B, s, b, nullptr, nullptr, nullptr, nullptr, nullptr, errors);
     return launch_status();
@@ -634,11 +634,11 @@ void* g_static_ptr[kMaxDevices];   // device address of g_fwd_static_scratch, pe
 // use.  The device address is looked up once per device, with that device current.
 l4q_status static_scratch_for_current_device(void** out) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return L4Q_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cuda_fail();
   std::lock_guard<std::mutex> lk(g_static_mu);
   if (!g_static_ptr[dev]) {
     void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_fwd_static_scratch) != cudaSuccess || !ptr) return L4Q_ERR_CUDA;
+    if (cudaGetSymbolAddress(&ptr, g_fwd_static_scratch) != cudaSuccess || !ptr) return cuda_fail();
     g_static_ptr[dev] = ptr;
   }
   *out = g_static_ptr[dev];
@@ -693,12 +693,12 @@ l4q_status l4q_selftest_tile_copy(const void* src, void* dst, int64_t rows, int6
 
 l4q_status l4q_check(void* cuda_stream) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (cudaStreamSynchronize(stream) != cudaSuccess) return L4Q_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return cuda_fail();
   unsigned int word = 0;
-  if (cudaMemcpyFromSymbol(&word, g_l4q_status, sizeof(word)) != cudaSuccess) return L4Q_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(&word, g_l4q_status, sizeof(word)) != cudaSuccess) return cuda_fail();
   if (word != 0) {
     const unsigned int zero = 0;
-    if (cudaMemcpyToSymbol(g_l4q_status, &zero, sizeof(zero)) != cudaSuccess) return L4Q_ERR_CUDA;
+    if (cudaMemcpyToSymbol(g_l4q_status, &zero, sizeof(zero)) != cudaSuccess) return cuda_fail();
     return (l4q_status)word;
   }
   return L4Q_OK;
@@ -713,7 +713,7 @@ l4q_status l4q_profile_enable(int enable) {
     for (auto& sl : g_prof_pool) {
       if (cudaEventCreate(&sl.begin) != cudaSuccess || cudaEventCreate(&sl.end) != cudaSuccess) {
         g_prof_pool.clear();
-        return L4Q_ERR_CUDA;
+        return cuda_fail();
       }
     }
   }

@@ -74,6 +74,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Status of a failed runtime call.  Reads the runtime's last-error word so that the failure does not surface a
+// second time, as the result of an unrelated later call of the same thread.
+inline l4q_status cuda_fail() {
+  (void)cudaGetLastError();
+  return L4Q_ERR_CUDA;
+}
+
 // Layout of the STE factor array that the weight-tile kernel hands to the weight-gradient kernel (internal, in the
 // workspace): tiles of 128 rows x 128 columns, each one contiguous block of 32 KB ordered [piece of 8 columns]
 // [row][8 values], tiles row-major over (row tile, column tile).  A thread that owns a weight row reads 16 bytes

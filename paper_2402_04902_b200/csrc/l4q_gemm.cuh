@@ -30,6 +30,8 @@
 // its tensor memory before returning.
 #pragma once
 
+#include <atomic>
+
 #include <algorithm>
 
 #include "l4q_common.cuh"
@@ -833,17 +835,45 @@ typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// The driver's tensor-map encoder: one entry point for the whole process, looked up once (the initialisation of a
+// function-local static is thread-safe).
 inline PFN_encodeTiled get_encode_fn() {
-  static PFN_encodeTiled fn = nullptr;
-  if (!fn) {
+  static const PFN_encodeTiled fn = [] {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
         qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<PFN_encodeTiled>(p);
-  }
+      p = nullptr;
+    return reinterpret_cast<PFN_encodeTiled>(p);
+  }();
   return fn;
+}
+
+// SM count and L2 size of the CURRENT device, cached per device ordinal.  Concurrent first calls may both query
+// the runtime; they store the same values, and every slot is an atomic, so no caller reads a torn or foreign entry.
+struct DeviceFacts {
+  int sms;
+  size_t l2;
+};
+inline DeviceFacts device_facts() {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> sms[kMaxDevices];        // zero-initialised: 0 = not queried yet
+  static std::atomic<size_t> l2[kMaxDevices];
+  int dev = 0;
+  cudaGetDevice(&dev);
+  const bool cached = dev >= 0 && dev < kMaxDevices;
+  DeviceFacts f{cached ? sms[dev].load(std::memory_order_acquire) : 0, cached ? l2[dev].load(std::memory_order_acquire) : 0};
+  if (f.sms > 0 && f.l2 > 0) return f;
+  int n = 0, bytes = 0;
+  cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  cudaDeviceGetAttribute(&bytes, cudaDevAttrL2CacheSize, dev);
+  f.sms = n > 0 ? n : 148;
+  f.l2 = bytes > 0 ? (size_t)bytes : (size_t)96 << 20;
+  if (cached) {
+    l2[dev].store(f.l2, std::memory_order_release);
+    sms[dev].store(f.sms, std::memory_order_release);
+  }
+  return f;
 }
 
 // bf16 row-major matrix [rows, cols]; box = [box_rows, 64 columns (128 bytes)], 128-byte swizzle, zero fill.
@@ -862,29 +892,14 @@ inline bool make_tmap_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint
 // Tile rows per band: as many A panels (128 rows x K, bf16) as fit in half of L2, the rest being left to the
 // streamed operand and the output; at least 8, and split evenly so that the last band is not a sliver.
 inline int tile_band_rows(int tiles_m, size_t a_panel_bytes) {
-  static size_t l2 = 0;
-  if (!l2) {
-    int dev = 0, bytes = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&bytes, cudaDevAttrL2CacheSize, dev);
-    l2 = bytes > 0 ? (size_t)bytes : (size_t)96 << 20;
-  }
+  const size_t l2 = device_facts().l2;
   int rows = (int)std::max<size_t>(8, (l2 / 2) / std::max<size_t>(a_panel_bytes, 1));
   rows = std::min(rows, tiles_m);
   const int bands = ceil_div(tiles_m, rows);
   return ceil_div(tiles_m, bands);
 }
 
-inline int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
-}
+inline int sm_count() { return device_facts().sms; }
 
 // `ta2`, `tb2`: second operand pair of an EXT launch (g.num_kb2 K blocks), or, for the weight-gradient epilogue, the
 // maps of the bf16 copies of A [rn, d_in] and B^T [rn, d_out] (boxes of 64 columns x rn rows); ignored otherwise.
@@ -893,7 +908,7 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
                        const CUtensorMap* ta2 = nullptr, const CUtensorMap* tb2 = nullptr) {
   constexpr bool TMA_STORE = (EPI == EPI_STORE && TN == BN);
   CUtensorMap tc = ta;                                  // placeholder where the epilogue does not store by TMA
-  if (TMA_STORE && !make_tmap_bf16(&tc, g.C, (uint64_t)g.M, (uint64_t)g.N, 128)) return L4Q_ERR_CUDA;
+  if (TMA_STORE && !make_tmap_bf16(&tc, g.C, (uint64_t)g.M, (uint64_t)g.N, 128)) return cuda_fail();
   g.tiles_m = ceil_div(g.M, BM);
   g.tiles_n = ceil_div(g.N, TN);
   g.num_kb = ceil_div(g.K, BK);
@@ -907,7 +922,7 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
   const size_t smem = gemm_smem_bytes(STAGES, EPI == EPI_WGRAD ? wgrad_epi_smem_bytes(RANK)
                                               : TMA_STORE ? store_epi_smem_bytes() : 0, stage_bytes_for(TN));
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   const int tiles = g.tiles_m * g.tiles_n, sms = sm_count();
   int grid = std::min(tiles, sms);
   if (EPI != EPI_STORE && tiles < sms) grid = tiles * std::min(sms / tiles, g.num_kb);   // K slices for the idle SMs
@@ -919,7 +934,7 @@ l4q_status launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, GemmArgs& g
 inline l4q_status gemm_forward_bf16(const Params& p, const void* X, const void* Wq, void* Y, cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, X, p.tokens, p.d_in, BM) || !make_tmap_bf16(&tb, Wq, p.d_out, p.d_in, BN))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.tokens; g.N = p.d_out; g.K = p.d_in;
   g.C = reinterpret_cast<__nv_bfloat16*>(Y);
@@ -930,7 +945,7 @@ inline l4q_status gemm_forward_bf16(const Params& p, const void* X, const void* 
 inline l4q_status gemm_dgrad_bf16(const Params& p, const void* dY, const void* Wq, void* dX, cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BM) || !make_tmap_bf16(&tb, Wq, p.d_out, p.d_in, BK))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.tokens; g.N = p.d_in; g.K = p.d_out;
   g.C = reinterpret_cast<__nv_bfloat16*>(dX);
@@ -945,7 +960,7 @@ inline l4q_status gemm_wgrad_bf16(const Params& p, const void* X, const void* dY
   const int rn = wgrad_rn(p.rank);
   if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BK) || !make_tmap_bf16(&tb, X, p.tokens, p.d_in, BK) ||
       !make_tmap_bf16(&ta16, A16, rn, p.d_in, rn) || !make_tmap_bf16(&tbt16, Bt16, rn, p.d_out, rn))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.d_out; g.N = p.d_in; g.K = p.tokens;
   g.p = p;

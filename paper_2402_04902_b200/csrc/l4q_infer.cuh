@@ -436,7 +436,7 @@ inline l4q_status launch_infer_gemv(const Params& p, const void* X, const uint32
   const int grid = std::min(ceil_div(quads, GEMV_THREADS / 32), sm_count() * per_sm);
   auto launch = [&](auto kern) -> l4q_status {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     kern<<<grid, GEMV_THREADS, smem, st>>>(reinterpret_cast<const __nv_bfloat16*>(X), codes, s16, b16,
                                            reinterpret_cast<__nv_bfloat16*>(Y), p.d_in, p.d_out, shift, p.group, p.ngroups);
     return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
@@ -489,13 +489,13 @@ inline l4q_status launch_infer_bf16(const Params& p, const void* X, const uint32
   a.Y = reinterpret_cast<__nv_bfloat16*>(Y);
   CUtensorMap tx, tc;
   a.x_rows = std::min(INF_M, (p.tokens + 7) / 8 * 8);
-  if (!make_tmap_bf16(&tx, X, p.tokens, p.d_in, a.x_rows)) return L4Q_ERR_CUDA;
-  if (!make_tmap_words(&tc, codes, p.d_out, ((uint64_t)p.d_in * p.bits) >> 5, 4 * p.bits, a.tile_n)) return L4Q_ERR_CUDA;
+  if (!make_tmap_bf16(&tx, X, p.tokens, p.d_in, a.x_rows)) return cuda_fail();
+  if (!make_tmap_words(&tc, codes, p.d_out, ((uint64_t)p.d_in * p.bits) >> 5, 4 * p.bits, a.tile_n)) return cuda_fail();
   const size_t smem = infer_smem_bytes();
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
   auto launch = [&](auto kern) -> l4q_status {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     kern<<<grid, INF_THREADS, smem, st>>>(tx, tc, a);
     return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
   };

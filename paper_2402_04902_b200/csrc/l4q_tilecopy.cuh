@@ -69,14 +69,14 @@ k_tile_copy(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__
 // src, dst: bf16 [rows, cols] row-major (cols a multiple of 8, pointers 16-byte aligned); dst null = read only.
 inline l4q_status launch_tile_copy(const void* src, void* dst, int rows, int cols, cudaStream_t st) {
   CUtensorMap t_in, t_out;
-  if (!make_tmap_bf16(&t_in, src, rows, cols, TC_ROWS)) return L4Q_ERR_CUDA;
+  if (!make_tmap_bf16(&t_in, src, rows, cols, TC_ROWS)) return cuda_fail();
   t_out = t_in;
-  if (dst && !make_tmap_bf16(&t_out, dst, rows, cols, TC_ROWS)) return L4Q_ERR_CUDA;
+  if (dst && !make_tmap_bf16(&t_out, dst, rows, cols, TC_ROWS)) return cuda_fail();
   const int tiles_m = ceil_div(rows, TC_ROWS), tiles_n = ceil_div(cols, TC_COLS);
   const size_t smem = 1024 + (size_t)TC_STAGES * TC_STAGE_BYTES + sizeof(TileCopyBarriers);
   if (cudaFuncSetAttribute(k_tile_copy, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     cudaGetLastError();
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   }
   k_tile_copy<<<std::min(tiles_m * tiles_n, sm_count()), 64, smem, st>>>(t_in, t_out, tiles_m, tiles_n, cols, dst != nullptr);
   return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;

@@ -80,7 +80,7 @@ inline l4q_status launch_lora_cast(const Params& p, const float* A, const float*
 inline l4q_status gemm_lora_down_bf16(const Params& p, const void* X, const VariantScratch& v, cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, X, p.tokens, p.d_in, BM) || !make_tmap_bf16(&tb, v.Ab, LORA_PAD, p.d_in, LORA_PAD))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.tokens; g.N = LORA_PAD; g.K = p.d_in;
   g.C = v.Xt;
@@ -91,7 +91,7 @@ inline l4q_status gemm_lora_down_bf16(const Params& p, const void* X, const Vari
 inline l4q_status gemm_lora_up_t_bf16(const Params& p, const void* dY, const VariantScratch& v, cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BM) || !make_tmap_bf16(&tb, v.Bb, p.d_out, LORA_PAD, BK))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.tokens; g.N = LORA_PAD; g.K = p.d_out;
   g.C = v.dYt;
@@ -104,7 +104,7 @@ inline l4q_status gemm_forward_lora_bf16(const Params& p, const void* X, const v
   CUtensorMap ta, tb, ta2, tb2;
   if (!make_tmap_bf16(&ta, X, p.tokens, p.d_in, BM) || !make_tmap_bf16(&tb, W, p.d_out, p.d_in, BN) ||
       !make_tmap_bf16(&ta2, v.Xt, p.tokens, LORA_PAD, BM) || !make_tmap_bf16(&tb2, v.gBb, p.d_out, LORA_PAD, BN))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.tokens; g.N = p.d_out; g.K = p.d_in;
   g.num_kb2 = 1;
@@ -118,7 +118,7 @@ inline l4q_status gemm_dgrad_lora_bf16(const Params& p, const void* dY, const vo
   CUtensorMap ta, tb, ta2, tb2;
   if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BM) || !make_tmap_bf16(&tb, W, p.d_out, p.d_in, BK) ||
       !make_tmap_bf16(&ta2, v.dYt, p.tokens, LORA_PAD, BM) || !make_tmap_bf16(&tb2, v.gAb, LORA_PAD, p.d_in, BK))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.tokens; g.N = p.d_in; g.K = p.d_out;
   g.num_kb2 = 1;
@@ -131,7 +131,7 @@ inline l4q_status gemm_lora_da_bf16(const Params& p, const void* X, const Varian
                                     cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, v.dYt, p.tokens, LORA_PAD, BK) || !make_tmap_bf16(&tb, X, p.tokens, p.d_in, BK))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.rank; g.N = p.d_in; g.K = p.tokens;
   g.C32 = dA; g.ldc = p.d_in; g.scale = p.gamma;
@@ -143,7 +143,7 @@ inline l4q_status gemm_lora_db_bf16(const Params& p, const void* dY, const Varia
                                     cudaStream_t st) {
   CUtensorMap ta, tb;
   if (!make_tmap_bf16(&ta, dY, p.tokens, p.d_out, BK) || !make_tmap_bf16(&tb, v.Xt, p.tokens, LORA_PAD, BK))
-    return L4Q_ERR_CUDA;
+    return cuda_fail();
   GemmArgs g{};
   g.M = p.d_out; g.N = p.rank; g.K = p.tokens;
   g.C32 = dB; g.ldc = p.rank; g.scale = p.gamma;

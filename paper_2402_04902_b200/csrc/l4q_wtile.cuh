@@ -1090,22 +1090,22 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   const bool sb_aligned = ((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(b)) & 15u) == 0;
   if (!wtile_plan(a, mode, sb_aligned)) return L4Q_ERR_UNSUPPORTED;
   CUtensorMap t_w0, t_o0, t_o1, t_s, t_b;
-  if (!make_tmap_bf16(&t_w0, W0, p.d_out, p.d_in, WT2_ROWS)) return L4Q_ERR_CUDA;
+  if (!make_tmap_bf16(&t_w0, W0, p.d_out, p.d_in, WT2_ROWS)) return cuda_fail();
   t_o1 = t_w0;
   if (mode == WT2_PACK) {
     if (!make_tmap_words(&t_o0, out0, p.d_out, ((uint64_t)p.d_in * p.bits) >> 5, WT2_COLS * p.bits / 32))
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
   } else if (mode == WT2_ERROR || mode == WT2_FACTORS) {
     t_o0 = t_w0;                                    // nothing is stored by TMA
     a.F = reinterpret_cast<__half*>(out1);
   } else {
-    if (!make_tmap_bf16(&t_o0, out0, p.d_out, p.d_in, WT2_ROWS)) return L4Q_ERR_CUDA;
+    if (!make_tmap_bf16(&t_o0, out0, p.d_out, p.d_in, WT2_ROWS)) return cuda_fail();
     a.F = reinterpret_cast<__half*>(out1);
   }
   t_s = t_w0; t_b = t_w0;                          // placeholders when unused
   if (a.sb_box) {                                   // fp32 moved as 32-bit words
     if (!make_tmap_words(&t_s, s, p.d_out, p.ngroups, a.sb_box) || !make_tmap_words(&t_b, b, p.d_out, p.ngroups, a.sb_box))
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
   }
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
 #ifdef L4Q_EXPERIMENT
@@ -1131,7 +1131,7 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
       copy_blocks = (int)(((long long)cp.rn * (p.d_in + p.d_out) / 8 + 255) / 256);
     }
     k_split_operands<<<image_blocks + copy_blocks, 256, 0, st>>>(a, static_cast<uint8_t*>(op_img), image_blocks, cp);
-    if (cudaGetLastError() != cudaSuccess) return L4Q_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     a.op_img = static_cast<const uint8_t*>(op_img);
   }
   if (zero) {                                       // the kernel's epilogue warps clear these before their first tile
@@ -1140,7 +1140,7 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
   }
   auto launch = [&](auto kern) -> l4q_status {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(WT2_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -1150,7 +1150,7 @@ inline l4q_status launch_wtile_tc(int mode, const Params& p, const void* W0, con
     cfg.numAttrs = op_img ? 1 : 0;                  // overlap with the operand split that was just launched
     if (cudaLaunchKernelEx(&cfg, kern, t_w0, t_o0, t_o1, t_s, t_b, a) != cudaSuccess) {
       cudaGetLastError();
-      return L4Q_ERR_CUDA;
+      return cuda_fail();
     }
     return cudaGetLastError() == cudaSuccess ? L4Q_OK : L4Q_ERR_CUDA;
   };

@@ -55,11 +55,25 @@ def test_workspace_query_and_rejections(lib):
 @pytest.mark.parametrize("mutation,expected", [
     (dict(tokens=0), 1), (dict(rank=0), 1), (dict(group_size=96), 2), (dict(bits=9), 2), (dict(bits=1), 2),
     (dict(group_size=4, d_in=256), 2),
+    (dict(rank=129), 2), (dict(rank=256), 2),       # above L4Q_MAX_RANK
 ])
 def test_bad_desc_is_an_error_code_not_a_crash(lib, mutation, expected):
     d = l4q.make_desc(CONFIG1.with_(**mutation))
     st = lib.l4q_linear_fwd(ctypes.byref(d), None, None, None, None, None, None, None, None, 0, None)
     assert st == expected
+
+
+@pytest.mark.parametrize("rank", [64, 128])
+def test_ranks_up_to_the_limit_get_a_workspace_size(lib, rank):
+    """Ranks the header admits pass the descriptor check in both modes (the plain-ALU weight-tile kernel serves ranks
+    above 64; its shared-memory need of rank x 320 floats fits at the limit), and the first rank above it does not."""
+    for dt in ("bf16", "f32"):
+        d = l4q.make_desc(CONFIG1.with_(rank=rank, io_dtype=dt))
+        assert l4q.l4q_workspace_bytes(d, l4q.L4Q_OP_FWD) > 0
+        assert l4q.l4q_workspace_bytes(d, l4q.L4Q_OP_BWD) >= l4q.l4q_workspace_bytes(d, l4q.L4Q_OP_FWD)
+    assert l4q.L4Q_MAX_RANK == 128 and l4q.L4Q_MAX_RANK * 320 * 4 <= 227 * 1024
+    d = l4q.make_desc(CONFIG1.with_(rank=l4q.L4Q_MAX_RANK + 1))
+    assert l4q.l4q_workspace_bytes(d, l4q.L4Q_OP_FWD) == 0
 
 
 def test_null_pointers_rejected_before_any_launch(lib):

@@ -430,3 +430,49 @@ def test_mask_guard_band_and_fp32_minmax_init_never_clips():
     assert (w > 15).any()                                             # rounding of s does push some maxima past Q_P
     g = orc.backward(spec, rng.normal(size=(4, i)), rng.normal(size=(4, o)), W0, A, B, s32, b32)
     assert np.all(g["db"] == 0.0)
+
+
+def test_guard_band_zero_is_the_printed_gate_and_changes_nothing_away_from_the_bounds():
+    """App. A.1 prints the plain test Q_N <= w <= Q_P.  With mask_guard = 0 the oracle is that test: an element
+    2^-12 of a step outside a bound is gated out.  And on a layer none of whose w lies within 2^-10 of a bound, the
+    default band gives bit for bit the gradients of a scalar loop that applies the printed test element by element
+    (Eq. 5-6 for ds, db; Eq. 13-14 for dA, dB), so the band only ever decides elements on a bound."""
+    from dataclasses import replace
+    spec0 = L4QSpec(rank=1, alpha=1.0, bits=2, group_size=4, mask_guard=0.0)
+    s = np.array([[1.0]]); b = np.array([[0.0]])
+    W0 = np.array([[-2.0 ** -12, 3.0 + 2.0 ** -12, 0.0, 3.0]])
+    A = np.array([[1.0, 1.0, 1.0, 1.0]]); B = np.array([[0.0]])
+    X = np.eye(4); dY = np.array([[1.0], [10.0], [100.0], [1000.0]])
+    g = orc.backward(spec0, X, dY, W0, A, B, s, b)
+    assert g["dB"][0, 0] == 100.0 + 1000.0                            # on the bounds: inside (inclusive)
+    assert g["db"][0, 0] == 1.0 + 10.0                                # a hair outside: clipped
+
+    rng = np.random.default_rng(33)
+    spec, X, dY, W0, A, B, s, b = _layer(rng, o=5, i=24, r=3, M=7, g=8, bits=3, bscale=0.2, spread=0.8)
+    qn, qp = orc.grid_bounds(spec)
+    w = orc.prequant(spec, orc.merge(spec, W0, A, B), s, b)
+    assert np.all(np.minimum(np.abs(w - qn), np.abs(w - qp)) > 2.0 ** -9)        # nobody near a bound ...
+    assert (w < qn).any() and (w > qp).any() and ((w > qn) & (w < qp)).any()      # ... and all three branches occur
+    got = orc.backward(spec, X, dY, W0, A, B, s, b)
+    got0 = orc.backward(replace(spec, mask_guard=0.0), X, dY, W0, A, B, s, b)
+    o, i = W0.shape
+    gsz = spec.group_size
+    G = dY.T @ X
+    ds = np.zeros_like(s); db = np.zeros_like(b); Gm = np.zeros_like(G)
+    for r_ in range(o):
+        for c in range(i):
+            k = c // gsz
+            wv = w[r_, c]
+            if wv < qn:
+                ds[r_, k] += G[r_, c] * qn; db[r_, k] += G[r_, c]
+            elif wv > qp:
+                ds[r_, k] += G[r_, c] * qp; db[r_, k] += G[r_, c]
+            else:
+                ds[r_, k] += G[r_, c] * (np.rint(wv) - wv); Gm[r_, c] = G[r_, c]
+    for res in (got, got0):
+        np.testing.assert_allclose(res["ds"], ds, rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(res["db"], db, rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(res["dA"], spec.gamma * B.T @ Gm, rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(res["dB"], spec.gamma * Gm @ A.T, rtol=1e-12, atol=1e-12)
+    for k_ in ("dX", "dA", "dB", "ds", "db"):
+        np.testing.assert_array_equal(got[k_], got0[k_])
