@@ -106,6 +106,49 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Bar
   return true;
 }
 
+// The same wait for a role that runs ahead of its ring and has time to spare (a TMA producer waiting for a free
+// slot, an epilogue warp waiting for a whole tile): between polls the thread sleeps, so that its polling does
+// not take issue slots from the warps that share its scheduler.
+template <class Barriers>
+__device__ __forceinline__ bool bounded_wait_relaxed(uint64_t* bar, uint32_t parity, Barriers* bars, unsigned sleep_ns = 256,
+                                                     long long limit_cycles = WAIT_LIMIT_CYCLES) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!ptx::mbar_try_wait(bar, parity)) {
+    __nanosleep(sleep_ns);
+    if ((++spins & 0x3Fu) == 0) {
+      if (bars->abort) return false;
+      if (clock64() - t0 > limit_cycles) {
+        bars->abort = 1;
+        atomicExch(&g_l4q_status, (unsigned int)L4Q_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+// The same wait on a shared-window address (no generic-to-shared conversion per call).
+template <class Barriers>
+__device__ __forceinline__ bool bounded_wait_a(uint32_t bar_a, uint32_t parity, Barriers* bars,
+                                               long long limit_cycles = WAIT_LIMIT_CYCLES) {
+  if (ptx::mbar_try_wait_a(bar_a, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!ptx::mbar_try_wait_a(bar_a, parity)) {
+    if ((++spins & 0xFFu) == 0) {
+      if (bars->abort) return false;
+      if (clock64() - t0 > limit_cycles) {
+        bars->abort = 1;
+        atomicExch(&g_l4q_status, (unsigned int)L4Q_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
 // Self-test of the error path of bounded_wait: one block waits on a barrier that nothing ever arrives on, with
 // a limit of about a millisecond.  The wait gives up, records L4Q_ERR_TIMEOUT and the kernel returns normally.
 struct SelftestBarriers { uint64_t never; volatile uint32_t abort; };

@@ -2,19 +2,21 @@
 // kept -- bit-packed unsigned codes u and one fp16 scale / offset per group, W_q = u * s16 + b16.
 //
 // The regime of the paper's deployment measurements is a handful of tokens per step (batch 1..64), so the
-// kernel is bound by reading the packed weight once (bits/8 bytes per weight) and is built around that:
-//   * tokens are the MMA's M (one 128-row tile, zero-filled beyond the batch), output features its N, in
-//     tiles of 64 rows of W so that even a 4096-row layer gives every SM work;
+// kernel is bound by reading the packed weight once (bits/8 bytes per weight) and by turning it into bf16,
+// and is built around that:
+//   * tokens are the MMA's M (one 128-row tile; only the rows that hold tokens are loaded), output features
+//     its N, in tiles of 16..128 rows of W chosen so that the tiles fill the SMs evenly;
 //   * the packed code words of a tile (N rows x 64 or 48 bytes per 128-deep k-step) arrive by TMA through a
 //     deep ring (8 steps in flight: they are the only HBM traffic), the X tile (128-byte-swizzled, from L2)
-//     and the dequantized operand through a shallow one (3 steps);
-//   * up to 384 dequantizer threads (one per weight row and 32 codes) turn the words into bf16 W_q = u * s + b
-//     (fp32 arithmetic) and write the MMA's B operand in the swizzled K-major layout; one thread issues
-//     tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory);
-//   * 4 epilogue warps drain the 128 x N accumulator of the previous tile meanwhile;
-//   * N (16..96 weight rows per tile) is chosen per layer so that the tiles fill whole waves of SMs.
-// Roles (640 threads): warp 0 = TMA of X, warp 2 = TMA of the code words, warp 1 = MMA issuer + TMEM owner,
-// warps 4..7 = epilogue, warps 8..19 = dequantizers.  Every mbarrier wait is bounded (bounded_wait).
+//     and the dequantized operand through a ring of as many steps as shared memory holds (up to 6);
+//   * 16 dequantizer warps: a warp takes one block of 16 weight rows x 128 k at a time (thread = one row and
+//     two runs of 32 codes), the blocks of consecutive k-steps going round the warps, so that all of them stay
+//     busy whatever N is and several k-steps are being dequantized at once.  Codes become bf16
+//     W_q = u * s + b with fp32 arithmetic and are written as the MMA's B operand in
+//     the swizzled K-major layout; one thread issues tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory);
+//   * warps 4..7 drain the 128 x N accumulator when a tile's k loop is done.
+// Roles (640 threads): warp 0 = TMA of X, warp 2 = TMA of the code words, warps 1 and 3 = MMA issuers (1 owns TMEM),
+// warps 4..19 = dequantizers.  Every mbarrier wait is bounded (bounded_wait).
 #pragma once
 
 #include "l4q_common.cuh"
@@ -25,33 +27,33 @@
 namespace l4q {
 
 constexpr int INF_M = 128;                 // tokens per tile (MMA M)
-constexpr int INF_NMAX = 96;               // most weight rows per tile (MMA N, a multiple of 16 chosen per problem)
+constexpr int INF_NMAX = 128;              // most weight rows per tile (MMA N, a multiple of 16 chosen per problem)
 constexpr int INF_BK = 128;                // k per pipeline step
-constexpr int INF_OP_STAGES = 3;           // X tile + dequantized W tile
+constexpr int INF_MAX_OP_STAGES = 6;       // X tile + dequantized W tile
 constexpr int INF_C_STAGES = 8;            // packed code words, loaded far ahead: they are what comes from HBM
 constexpr int INF_THREADS = 640;
-constexpr int INF_DEQ_THREADS = 384;       // warps 8..19: one thread per (weight row, 32 codes) unit, 4 * INF_NMAX
-constexpr int INF_X_BYTES = INF_M * INF_BK * 2;         // 32 KB: two 128 x 64 swizzled boxes
-constexpr int INF_W_BYTES = INF_NMAX * INF_BK * 2;      // 24 KB reserved: two (N x 64) swizzled tiles, 12 KB apart
-constexpr int INF_OP_BYTES = INF_X_BYTES + INF_W_BYTES;
-constexpr int INF_C_BYTES = INF_NMAX * 16 * 4;          // 6 KB reserved: N rows x (16 | 12) words
+constexpr int INF_WORKERS = 16;            // dequantizer warps (4..19)
 constexpr int INF_ACC = 2;
-constexpr int INF_ACC_COLS = 128;          // TMEM columns per accumulator stage
+constexpr int INF_HALF_COLS = 128;         // TMEM columns of one issuer's half of an accumulator stage
+constexpr int INF_ACC_COLS = 2 * INF_HALF_COLS;
 
 struct InferArgs {
   int tokens, d_in, d_out, bits, group, ngroups;
   int tile_n;                              // weight rows per tile
+  int nb;                                  // tile_n / 16: blocks of 16 rows per k-step
   int group_shift;                         // log2(group size) if it is a power of two, else -1
   int x_rows;                              // token rows a TMA box of X brings in (8 .. 128)
   int tiles_m, tiles_n, num_kb;
+  int op_stages;                           // depth of the operand ring
+  int workers;                             // dequantizer warps at work: min(INF_WORKERS, nb * op_stages)
+  uint32_t x_bytes, w_bytes, c_bytes;      // per stage: X tile (two boxes of x_rows x 64), W tile (two of N x 64), codes
   const __half *s16, *b16;
   __nv_bfloat16* Y;
 };
 
 struct __align__(8) InferBarriers {
-  uint64_t full_x[INF_OP_STAGES];          // X tile has landed
-  uint64_t full_w[INF_OP_STAGES];          // the dequantized B operand of the stage is complete
-  uint64_t empty_op[INF_OP_STAGES];        // the MMAs reading the operand stage have completed
+  uint64_t full_op[INF_MAX_OP_STAGES];     // the X tile has landed and the dequantized B operand of the stage is complete
+  uint64_t empty_op[INF_MAX_OP_STAGES];    // the MMAs reading the operand stage have completed
   uint64_t full_c[INF_C_STAGES];           // code words have landed
   uint64_t empty_c[INF_C_STAGES];          // the dequantizers have read the code words
   uint64_t tmem_full[INF_ACC], tmem_empty[INF_ACC];
@@ -59,9 +61,7 @@ struct __align__(8) InferBarriers {
   volatile uint32_t abort;
 };
 
-inline size_t infer_smem_bytes() {
-  return 1024 + (size_t)INF_OP_STAGES * INF_OP_BYTES + (size_t)INF_C_STAGES * INF_C_BYTES + sizeof(InferBarriers);
-}
+constexpr size_t INF_SMEM_LIMIT = 227 * 1024;
 
 // 32 unsigned codes of one weight row (starting at a multiple of 32 codes of the LSB-first bitstream), each
 // returned as the float m = 1 + u / 2^BITS: the code is moved into the top mantissa bits under the exponent
@@ -84,35 +84,86 @@ __device__ __forceinline__ void unpack_codes32(const uint32_t (&w)[BITS], float 
   for (int j = 0; j < 32; ++j) m[j] = unpack_code<BITS>(w, j);
 }
 
+// (a & b) | c in one logic instruction, all three operands in registers.
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
+// 32 codes of one weight row -> 16 words of bf16 pairs W_q = u * s + b (Eq. 9 on the unsigned code), formed in
+// fp32 and rounded once.  The bitstream is cut into windows of 12 bits (3 or 4 codes); one funnel shift puts a
+// window at mantissa bits 11..22, so that a code at bit position p reads, with the exponent of 1.0 or-ed in, as
+// m = 1 + u 2^(p-23), and u s + b = m S_p + (b - S_p) with S_p = s 2^(23-p): one logic op and one fma
+// per code, with three or four (S_p, b - S_p) pairs per thread.  S_p <= 2^12 s, so b - S_p is exact to
+// 2^-12 of a quantization step.
+template <int BITS>
+__device__ __forceinline__ void dequant_codes32(const uint32_t (&w)[BITS], float s, float b, uint32_t (&out)[16]) {
+  constexpr int CPW = 12 / BITS;                               // codes per window
+  constexpr uint32_t MASK = (1u << BITS) - 1u;
+  float S[CPW], C[CPW];
+  uint32_t mask[CPW];
+  // the masks and the exponent of 1.0 are kept in registers (opaque to the compiler), so that a code costs one
+  // three-input logic instruction; written as immediates they cost two
+  uint32_t one = 0x3F800000u;
+  asm volatile("" : "+r"(one));
+#pragma unroll
+  for (int i = 0; i < CPW; ++i) {
+    S[i] = s * (float)(1 << (12 - BITS * i));                  // 2^(23 - p), p = 11 + BITS i
+    C[i] = b - S[i];
+    mask[i] = MASK << (11 + BITS * i);
+    asm volatile("" : "+r"(mask[i]));
+  }
+  constexpr int NWIN = (32 + CPW - 1) / CPW;
+  uint32_t win[NWIN];
+#pragma unroll
+  for (int v = 0; v < NWIN; ++v) {
+    if (v == 0) {
+      win[v] = w[0] << 11;
+    } else {
+      const int sh = 12 * v - 11, wd = sh >> 5, off = sh & 31;
+      win[v] = __funnelshift_r(w[wd], wd + 1 < BITS ? w[wd + 1] : 0u, off);
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < 32; c += 2) {
+    const int v0 = c / CPW, i0 = c % CPW, v1 = (c + 1) / CPW, i1 = (c + 1) % CPW;
+    const float m0 = __uint_as_float(and_or(win[v0], mask[i0], one));
+    const float m1 = __uint_as_float(and_or(win[v1], mask[i1], one));
+    out[c >> 1] = pack_bf16x2(fmaf(m0, S[i0], C[i0]), fmaf(m1, S[i1], C[i1]));
+  }
+}
+
 template <int BITS>
 __global__ void __launch_bounds__(INF_THREADS, 1)
-k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in] bf16, box 64 x 128, swizzled
+k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in] bf16, box 64 x x_rows, swizzled
              const __grid_constant__ CUtensorMap tmap_c,      // codes [d_out, words] uint32, box (4 BITS) x tile_n
              const InferArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* c_base = smem + (size_t)INF_OP_STAGES * INF_OP_BYTES;
-  InferBarriers* bars = reinterpret_cast<InferBarriers*>(c_base + (size_t)INF_C_STAGES * INF_C_BYTES);
+  const uint32_t op_bytes = a.x_bytes + a.w_bytes;
+  const int S = a.op_stages;
+  uint8_t* c_base = smem + (size_t)S * op_bytes;
+  InferBarriers* bars = reinterpret_cast<InferBarriers*>(c_base + (size_t)INF_C_STAGES * a.c_bytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = a.tiles_m * a.tiles_n;
-  const int N = a.tile_n;
+  const int N = a.tile_n, NB = a.nb;
   constexpr int CW = 4 * BITS;                                 // code words per row and k-step (128 codes)
-  auto x_tile = [&](int st) { return smem + (size_t)st * INF_OP_BYTES; };
-  auto w_tile = [&](int st) { return smem + (size_t)st * INF_OP_BYTES + INF_X_BYTES; };
-  auto c_tile = [&](int st) { return c_base + (size_t)st * INF_C_BYTES; };
+  auto x_tile = [&](int st) { return smem + (size_t)st * op_bytes; };
+  auto w_tile = [&](int st) { return smem + (size_t)st * op_bytes + a.x_bytes; };
+  auto c_tile = [&](int st) { return c_base + (size_t)st * a.c_bytes; };
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < INF_OP_STAGES; ++i) {
-      ptx::mbar_init(&bars->full_x[i], 1);
-      ptx::mbar_init(&bars->full_w[i], INF_DEQ_THREADS);
+    for (int i = 0; i < S; ++i) {
+      ptx::mbar_init(&bars->full_op[i], (uint32_t)(NB * 32 + 1));
       ptx::mbar_init(&bars->empty_op[i], 1);
     }
     for (int i = 0; i < INF_C_STAGES; ++i) {
       ptx::mbar_init(&bars->full_c[i], 1);
-      ptx::mbar_init(&bars->empty_c[i], INF_DEQ_THREADS);
+      ptx::mbar_init(&bars->empty_c[i], (uint32_t)(NB * 32));
     }
     for (int i = 0; i < INF_ACC; ++i) {
-      ptx::mbar_init(&bars->tmem_full[i], 1);
+      ptx::mbar_init(&bars->tmem_full[i], 2);
       ptx::mbar_init(&bars->tmem_empty[i], 128);
     }
     bars->abort = 0;
@@ -130,19 +181,19 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
   const uint32_t tmem_base = bars->tmem_base;
 
   if (warp == 0) {
-    // ------------------------------ TMA: X tiles (shallow ring) ------------------------------
+    // ------------------------------ TMA: X tiles ------------------------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       for (int t = blockIdx.x; t < num_tiles && !bars->abort; t += gridDim.x) {
         const int m0 = (t / a.tiles_n) * INF_M;
         for (int kb = 0; kb < a.num_kb; ++kb) {      // no flag loads here: see the GEMM producers
-          bounded_wait(&bars->empty_op[stage], phase ^ 1, bars);
-          // only the rows that hold tokens are copied; the other rows of the operand are never stored
-          // from (an MMA output row depends on its own input row only)
-          ptx::mbar_arrive_expect_tx(&bars->full_x[stage], (uint32_t)(2 * a.x_rows * 128));
-          ptx::tma_load_2d(x_tile(stage), &tmap_x, &bars->full_x[stage], kb * INF_BK, m0);
-          ptx::tma_load_2d(x_tile(stage) + INF_X_BYTES / 2, &tmap_x, &bars->full_x[stage], kb * INF_BK + 64, m0);
-          if (++stage == INF_OP_STAGES) { stage = 0; phase ^= 1; }
+          bounded_wait_relaxed(&bars->empty_op[stage], phase ^ 1, bars);
+          // only the rows that hold tokens are copied; the other rows of the operand hold whatever the ring
+          // held before (an MMA output row depends on its own input row only, and they are never stored)
+          ptx::mbar_arrive_expect_tx(&bars->full_op[stage], a.x_bytes);
+          ptx::tma_load_2d(x_tile(stage), &tmap_x, &bars->full_op[stage], kb * INF_BK, m0);
+          ptx::tma_load_2d(x_tile(stage) + a.x_bytes / 2, &tmap_x, &bars->full_op[stage], kb * INF_BK + 64, m0);
+          if (++stage == S) { stage = 0; phase ^= 1; }
         }
       }
     }
@@ -154,7 +205,7 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
       for (int t = blockIdx.x; t < num_tiles && !bars->abort; t += gridDim.x) {
         const int n0 = (t % a.tiles_n) * N;
         for (int kb = 0; kb < a.num_kb; ++kb) {      // no flag loads here: see the GEMM producers
-          bounded_wait(&bars->empty_c[cs], cphase ^ 1, bars);
+          bounded_wait_relaxed(&bars->empty_c[cs], cphase ^ 1, bars);
           ptx::mbar_arrive_expect_tx(&bars->full_c[cs], (uint32_t)(N * CW * 4));
           ptx::tma_load_2d(c_tile(cs), &tmap_c, &bars->full_c[cs], kb * CW, n0);
           if (++cs == INF_C_STAGES) { cs = 0; cphase ^= 1; }
@@ -162,132 +213,187 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
+  } else if (warp == 1 || warp == 3) {
+    // ------------------------------ MMA issuers ------------------------------
+    // Two threads on two warp schedulers: issuer i takes the k-steps whose running number (over all tiles of the
+    // CTA) is i modulo 2 and accumulates them into its own half of the accumulator stage; the epilogue adds the
+    // halves.  One thread alone, sharing its scheduler with four busy dequantizer warps, needed 650..900 cycles
+    // to issue the eight MMAs of a k-step that execute in about 420.
     if (lane == 0) {
+      const int me = warp >> 1;                                // 0 or 1
       const uint32_t idesc = ptx::make_idesc_bf16(INF_M, N, false, false);
-      int stage = 0; uint32_t phase = 0;
+      // Descriptors differ in the start-address field only (16-byte units in the low word; shared memory is
+      // < 256 KB, so sums never leave the field): the eight offsets of a k-step are kept in registers.
+      const uint64_t dx0 = ptx::make_smem_desc_sw128(ptx::smem_u32(smem), 16, 1024);
+      const uint64_t dw0 = ptx::make_smem_desc_sw128(ptx::smem_u32(smem) + a.x_bytes, 16, 1024);
+      const uint32_t d_hi = (uint32_t)(dx0 >> 32);             // same for both operands
+      uint32_t ox[INF_BK / UMMA_K], ow[INF_BK / UMMA_K];
+#pragma unroll
+      for (int ks = 0; ks < INF_BK / UMMA_K; ++ks) {           // steps 4..7 are the second 64-wide tile
+        ox[ks] = (uint32_t)dx0 + (uint32_t)((ks >> 2) * (a.x_bytes >> 5) + (ks & 3) * 2);
+        ow[ks] = (uint32_t)dw0 + (uint32_t)((ks >> 2) * (a.w_bytes >> 5) + (ks & 3) * 2);
+      }
+      const uint32_t step = op_bytes >> 4;
+      const uint32_t full_op_a = ptx::smem_u32(&bars->full_op[0]);
+      // this issuer's next k-step: number within the tile, ring stage and phase (S >= 2)
+      int kb = me, stage = me; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       for (int t = blockIdx.x; t < num_tiles && !bars->abort; t += gridDim.x) {
         bounded_wait(&bars->tmem_empty[acc], acc_phase ^ 1, bars);
         if (bars->abort) break;
         ptx::tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * INF_ACC_COLS);
-        for (int kb = 0; kb < a.num_kb; ++kb) {
-          bounded_wait(&bars->full_x[stage], phase, bars);
-          bounded_wait(&bars->full_w[stage], phase, bars);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * INF_ACC_COLS + me * INF_HALF_COLS);
+        uint32_t accumulate = 0;
+        for (; kb < a.num_kb; kb += 2) {
+          bounded_wait_a(full_op_a + (uint32_t)stage * 8u, phase, bars);
           ptx::tc_fence_after_sync();
-          const uint32_t xa = ptx::smem_u32(x_tile(stage)), wa = ptx::smem_u32(w_tile(stage));
+          const uint32_t so = (uint32_t)stage * step;
 #pragma unroll
-          for (int ks = 0; ks < INF_BK / UMMA_K; ++ks) {     // 8 steps of 16; steps 4..7 are the second 64-wide tile
-            const uint64_t da = ptx::make_smem_desc_sw128(xa + (ks >> 2) * (INF_X_BYTES / 2) + (ks & 3) * 32, 16, 1024);
-            const uint64_t db = ptx::make_smem_desc_sw128(wa + (ks >> 2) * (INF_W_BYTES / 2) + (ks & 3) * 32, 16, 1024);
-            ptx::mma_bf16_ss(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+          for (int ks = 0; ks < INF_BK / UMMA_K; ++ks) {
+            const uint64_t da = ((uint64_t)d_hi << 32) | (uint64_t)(ox[ks] + so);
+            const uint64_t db = ((uint64_t)d_hi << 32) | (uint64_t)(ow[ks] + so);
+            ptx::mma_bf16_ss(d_tmem, da, db, idesc, ks != 0 ? 1u : accumulate);
           }
+          accumulate = 1;
           ptx::mma_commit(&bars->empty_op[stage]);
-          if (++stage == INF_OP_STAGES) { stage = 0; phase ^= 1; }
+          stage += 2;
+          if (stage >= S) { stage -= S; phase ^= 1; }
         }
-        ptx::mma_commit(&bars->tmem_full[acc]);
+        kb -= a.num_kb;                                        // the same k-step, counted within the next tile
+        if (accumulate) ptx::mma_commit(&bars->tmem_full[acc]);
+        else ptx::mbar_arrive(&bars->tmem_full[acc]);          // (a one-step tile: nothing from this issuer)
         if (++acc == INF_ACC) { acc = 0; acc_phase ^= 1; }
       }
     }
     __syncwarp();
-  } else if (warp >= 4 && warp < 8) {
-    // ------------------------------ epilogue: lane = token ------------------------------
-    const int quarter = warp & 3;
+  } else if (warp >= 4) {
+    // ------------------------------ dequantizers: warp = block of 16 rows x 128 k, thread = (row, 2 x 32 codes) ----
+    const int worker = warp - 4;                               // 0 .. 15
+    // Row of the block and the two 32-code quarters of the k-step a thread takes.  The eight lanes that one
+    // shared-memory wavefront serves hold eight different rows, each with quarter (row / 2 + j) % 4: their 16-byte
+    // loads of the code words fall into eight different bank groups, and so do their stores into the swizzled
+    // operand (chunk ((q & 1) * 4 + c) ^ (row % 8)).  The second quarter is two further on.
+    const int r16 = (lane >> 4) * 8 + (lane & 7);
+    const int q0 = (((lane & 7) >> 1) + ((lane >> 3) & 1)) & 3;
+    const int quarter = warp & 3;                              // epilogue (warps 4..7): TMEM lane quarter
+    const uint32_t smem_a = ptx::smem_u32(smem);
+    const uint32_t c_base_a = smem_a + (uint32_t)S * op_bytes;
+    const uint32_t full_c_a = ptx::smem_u32(&bars->full_c[0]), empty_c_a = ptx::smem_u32(&bars->empty_c[0]);
+    const uint32_t full_op_a = ptx::smem_u32(&bars->full_op[0]), empty_op_a = ptx::smem_u32(&bars->empty_op[0]);
+    int stage = 0; uint32_t phase = 0;                         // operand ring, at k-step `ks` of the current tile
+    int cs = 0; uint32_t cphase = 0;                           // code ring
+    auto advance = [&](int d) {
+      stage += d; while (stage >= S) { stage -= S; phase ^= 1; }
+      cs += d; while (cs >= INF_C_STAGES) { cs -= INF_C_STAGES; cphase ^= 1; }
+    };
     int acc = 0; uint32_t acc_phase = 0;
+    uint32_t tiles_done = 0;                                   // tiles of this CTA so far (epilogue warps)
+    // The warps at work together span ceil(workers / NB) k-steps.  A wait on a ring barrier tells phases apart by
+    // parity only, so a warp must never be two laps of a ring ahead of it: the span may not exceed the depth of
+    // either ring, which is what limits the number of warps at work when N is small (the others only idle).
+    const bool works = worker < a.workers;
+    // from one block to the warp's next: a.workers blocks further on
+    const int step_ks = a.workers / NB, step_blk = a.workers - step_ks * NB;
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
       const int m0 = (t / a.tiles_n) * INF_M, n0 = (t % a.tiles_n) * N;
-      bounded_wait(&bars->tmem_full[acc], acc_phase, bars);
-      ptx::tc_fence_after_sync();
-      const int tok = m0 + quarter * 32 + lane;
-      const int nchunks = N >> 4;                              // 16 columns at a time
-      for (int c = 0; c < nchunks; ++c) {
-        uint32_t raw[16];
-        ptx::tmem_ld_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * INF_ACC_COLS + c * 16), raw);
-        ptx::tmem_ld_wait();
-        if (c == nchunks - 1) {
-          ptx::tc_fence_before_sync();
-          ptx::mbar_arrive(&bars->tmem_empty[acc]);
-        }
-        if (tok < a.tokens) {
-          __nv_bfloat16* dst = a.Y + (size_t)tok * a.d_out + n0 + c * 16;
+      int ks = works ? 0 : a.num_kb, blk = worker;
+      while (works && blk >= NB) { blk -= NB; ++ks; }
+      advance(min(ks, a.num_kb));                            // (a warp without a block in this tile just moves on)
+      // s, b (fp16 bit patterns) of the groups of this thread's codes (group size is a multiple of 32), for quarter
+      // q0 and for quarter q0 ^ 2, fetched one block ahead and left untouched in registers until they are used
+      auto load_sb = [&](int ks_, int blk_, unsigned short (&sv)[2], unsigned short (&bv)[2]) {
+        const int o = n0 + blk_ * 16 + r16;
+        sv[0] = sv[1] = bv[0] = bv[1] = 0;                     // rows / columns beyond the weight contribute nothing
+        if (ks_ < a.num_kb && o < a.d_out) {
+          const unsigned short* s_row = reinterpret_cast<const unsigned short*>(a.s16) + (size_t)o * a.ngroups;
+          const unsigned short* b_row = reinterpret_cast<const unsigned short*>(a.b16) + (size_t)o * a.ngroups;
 #pragma unroll
-          for (int v = 0; v < 2; ++v) {
-            if (n0 + c * 16 + v * 8 < a.d_out) {
-              uint4 o4;
-              o4.x = pack_bf16x2(__uint_as_float(raw[v * 8 + 0]), __uint_as_float(raw[v * 8 + 1]));
-              o4.y = pack_bf16x2(__uint_as_float(raw[v * 8 + 2]), __uint_as_float(raw[v * 8 + 3]));
-              o4.z = pack_bf16x2(__uint_as_float(raw[v * 8 + 4]), __uint_as_float(raw[v * 8 + 5]));
-              o4.w = pack_bf16x2(__uint_as_float(raw[v * 8 + 6]), __uint_as_float(raw[v * 8 + 7]));
-              *reinterpret_cast<uint4*>(dst + v * 8) = o4;
+          for (int h = 0; h < 2; ++h) {
+            const int k = ks_ * INF_BK + (q0 ^ (h * 2)) * 32;
+            if (k < a.d_in) {
+              const int g = a.group_shift >= 0 ? (k >> a.group_shift) : (k / a.group);
+              sv[h] = __ldg(s_row + g);
+              bv[h] = __ldg(b_row + g);
             }
           }
         }
-      }
-      if (++acc == INF_ACC) { acc = 0; acc_phase ^= 1; }
-    }
-  } else if (warp >= 8) {
-    // ------------------------------ dequantizers: thread = (weight row, 32 codes) ------------------------------
-    const int pt = threadIdx.x - 256;                          // 0 .. 383
-    const int row = pt >> 2, q = pt & 3;                       // row of the tile, 32-code quarter of the k-step
-    const bool active = row < N;
-    constexpr float kScale = (float)(1 << BITS);
-    int stage = 0; uint32_t phase = 0;                         // operand ring
-    int cs = 0; uint32_t cphase = 0;                           // code ring
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
-      const int n0 = (t % a.tiles_n) * N;
-      const int o = n0 + row;
-      const bool row_ok = active && o < a.d_out;
-      const __half* s_row = a.s16 + (size_t)o * a.ngroups;
-      const __half* b_row = a.b16 + (size_t)o * a.ngroups;
-      // s, b of the group of this thread's 32 codes (group size is a multiple of 32), fetched one k-step ahead
-      auto load_sb = [&](int kb, float& s_, float& b_) {
-        const int k = kb * INF_BK + q * 32;
-        s_ = 0.f; b_ = 0.f;                                    // rows / columns beyond the weight contribute nothing
-        if (row_ok && k < a.d_in) {
-          const int g = a.group_shift >= 0 ? (k >> a.group_shift) : (k / a.group);
-          s_ = __half2float(__ldg(s_row + g));
-          b_ = __half2float(__ldg(b_row + g));
-        }
       };
-      float s_next, b_next;
-      load_sb(0, s_next, b_next);
-      for (int kb = 0; kb < a.num_kb; ++kb) {
-        const float s2 = s_next * kScale, b2 = b_next - s_next * kScale;     // W_q = m * s2 + b2, m = 1 + u / 2^BITS
-        if (kb + 1 < a.num_kb) load_sb(kb + 1, s_next, b_next);
-        bounded_wait(&bars->full_c[cs], cphase, bars);         // the code words have landed
-        bounded_wait(&bars->empty_op[stage], phase ^ 1, bars); // the operand slot is free (its MMAs completed)
-        if (active) {
-          const uint8_t* crow = c_tile(cs) + row * (CW * 4) + q * (BITS * 4);
+      unsigned short s_next[2], b_next[2];
+      load_sb(ks, blk, s_next, b_next);
+      while (ks < a.num_kb) {
+        const int row = blk * 16 + r16;
+        const unsigned short s_cur[2] = {s_next[0], s_next[1]}, b_cur[2] = {b_next[0], b_next[1]};
+        int nblk = blk + step_blk, d = step_ks;
+        if (nblk >= NB) { nblk -= NB; ++d; }
+        load_sb(ks + d, nblk, s_next, b_next);
+        bounded_wait_a(full_c_a + (uint32_t)cs * 8u, cphase, bars);          // the code words have landed
+        bounded_wait_a(empty_op_a + (uint32_t)stage * 8u, phase ^ 1, bars);  // the operand slot is free (its MMAs completed)
+        const uint32_t c_row = c_base_a + (uint32_t)cs * a.c_bytes + (uint32_t)(row * (CW * 4));
+        const uint32_t w_row = smem_a + (uint32_t)stage * op_bytes + a.x_bytes + (uint32_t)(row * 128);
+        const uint32_t sw = (uint32_t)(row & 7);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int q = q0 ^ (h * 2);
+          const float s_ = __half2float(__ushort_as_half(s_cur[h]));
+          const float b_ = __half2float(__ushort_as_half(b_cur[h]));
           uint32_t w[BITS];
           if constexpr (BITS == 4) {
-            const uint4 v = *reinterpret_cast<const uint4*>(crow);
+            const uint4 v = ptx::lds128(c_row + (uint32_t)(q * 16));
             w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
           } else {
 #pragma unroll
-            for (int i = 0; i < BITS; ++i) w[i] = reinterpret_cast<const uint32_t*>(crow)[i];
+            for (int i = 0; i < BITS; ++i) w[i] = ptx::lds32(c_row + (uint32_t)(q * (BITS * 4) + i * 4));
           }
-          float m[32];
-          unpack_codes32<BITS>(w, m);
-          // W_q = u * s + b (Eq. 9 on the unsigned code) in fp32, rounded to bf16, into the K-major swizzled
-          // B operand: 64-k tile q >> 1, 16-byte chunks (q & 1) * 4 .. + 3 of row `row`
-          uint8_t* wrow = w_tile(stage) + (q >> 1) * (INF_W_BYTES / 2) + row * 128;
+          uint32_t wv[16];
+          dequant_codes32<BITS>(w, s_, b_, wv);
+          // into the K-major swizzled B operand: 64-k tile q >> 1, 16-byte chunks (q & 1) * 4 .. + 3 of row `row`
+          const uint32_t dst = w_row + (uint32_t)(q >> 1) * (a.w_bytes / 2);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 4; ++c)
+            ptx::sts128(dst + ((((uint32_t)((q & 1) * 4 + c)) ^ sw) << 4), wv[c * 4 + 0], wv[c * 4 + 1], wv[c * 4 + 2], wv[c * 4 + 3]);
+        }
+        ptx::mbar_arrive_a(empty_c_a + (uint32_t)cs * 8u);     // code words consumed
+        ptx::fence_proxy_async_smem();                         // the operand is read by the tensor cores
+        ptx::mbar_arrive_a(full_op_a + (uint32_t)stage * 8u);
+        blk = nblk;
+        if (ks + d < a.num_kb) advance(d);
+        else advance(a.num_kb - ks);                           // on to k-step 0 of the CTA's next tile
+        ks += d;
+      }
+      if (warp < 8) {
+        // ------------------------------ epilogue: lane = token ------------------------------
+        bounded_wait_relaxed(&bars->tmem_full[acc], acc_phase, bars, 512);
+        ptx::tc_fence_after_sync();
+        const int tok = m0 + quarter * 32 + lane;
+        const int nchunks = N >> 3;                            // 8 columns at a time
+        // which halves hold a sum: both, unless the tile is a single k-step (then only its issuer's)
+        const bool one_step = a.num_kb == 1;
+        const int only = one_step ? (int)(tiles_done & 1u) : 0;
+        for (int c = 0; c < nchunks; ++c) {
+          uint32_t raw[8], raw2[8];
+          const uint32_t col = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * INF_ACC_COLS + c * 8);
+          ptx::tmem_ld_32x8(col + (uint32_t)(only * INF_HALF_COLS), raw);
+          if (!one_step) ptx::tmem_ld_32x8(col + INF_HALF_COLS, raw2);
+          ptx::tmem_ld_wait();
+          if (c == nchunks - 1) {
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&bars->tmem_empty[acc]);
+          }
+          if (!one_step) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) raw[i] = __float_as_uint(__uint_as_float(raw[i]) + __uint_as_float(raw2[i]));
+          }
+          if (tok < a.tokens && n0 + c * 8 < a.d_out) {
             uint4 o4;
-            o4.x = pack_bf16x2(fmaf(m[c * 8 + 0], s2, b2), fmaf(m[c * 8 + 1], s2, b2));
-            o4.y = pack_bf16x2(fmaf(m[c * 8 + 2], s2, b2), fmaf(m[c * 8 + 3], s2, b2));
-            o4.z = pack_bf16x2(fmaf(m[c * 8 + 4], s2, b2), fmaf(m[c * 8 + 5], s2, b2));
-            o4.w = pack_bf16x2(fmaf(m[c * 8 + 6], s2, b2), fmaf(m[c * 8 + 7], s2, b2));
-            *reinterpret_cast<uint4*>(wrow + ((((q & 1) * 4 + c) ^ (row & 7)) << 4)) = o4;
+            o4.x = pack_bf16x2(__uint_as_float(raw[0]), __uint_as_float(raw[1]));
+            o4.y = pack_bf16x2(__uint_as_float(raw[2]), __uint_as_float(raw[3]));
+            o4.z = pack_bf16x2(__uint_as_float(raw[4]), __uint_as_float(raw[5]));
+            o4.w = pack_bf16x2(__uint_as_float(raw[6]), __uint_as_float(raw[7]));
+            *reinterpret_cast<uint4*>(a.Y + (size_t)tok * a.d_out + n0 + c * 8) = o4;
           }
         }
-        ptx::mbar_arrive(&bars->empty_c[cs]);                  // code words consumed
-        ptx::fence_proxy_async_smem();                         // the operand is read by the tensor cores
-        ptx::mbar_arrive(&bars->full_w[stage]);
-        if (++stage == INF_OP_STAGES) { stage = 0; phase ^= 1; }
-        if (++cs == INF_C_STAGES) { cs = 0; cphase ^= 1; }
+        ++tiles_done;
+        if (++acc == INF_ACC) { acc = 0; acc_phase ^= 1; }
       }
     }
   }
@@ -480,6 +586,7 @@ inline l4q_status launch_infer_bf16(const Params& p, const void* X, const uint32
   a.tokens = p.tokens; a.d_in = p.d_in; a.d_out = p.d_out; a.bits = p.bits; a.group = p.group; a.ngroups = p.ngroups;
   a.tiles_m = ceil_div(p.tokens, INF_M);
   a.tile_n = infer_pick_tile_n(p.d_out, a.tiles_m, sm_count());
+  a.nb = a.tile_n / 16;
   a.tiles_n = ceil_div(p.d_out, a.tile_n);
   a.num_kb = ceil_div(p.d_in, INF_BK);
   a.group_shift = -1;
@@ -491,7 +598,18 @@ inline l4q_status launch_infer_bf16(const Params& p, const void* X, const uint32
   a.x_rows = std::min(INF_M, (p.tokens + 7) / 8 * 8);
   if (!make_tmap_bf16(&tx, X, p.tokens, p.d_in, a.x_rows)) return cuda_fail();
   if (!make_tmap_words(&tc, codes, p.d_out, ((uint64_t)p.d_in * p.bits) >> 5, 4 * p.bits, a.tile_n)) return cuda_fail();
-  const size_t smem = infer_smem_bytes();
+  // shared-memory plan: the code ring, then as many operand stages as fit
+  a.x_bytes = (uint32_t)a.x_rows * 256u;                        // two boxes of x_rows x 128 bytes
+  a.w_bytes = (uint32_t)a.tile_n * 256u;
+  a.c_bytes = (uint32_t)(((size_t)a.tile_n * 4 * p.bits * 4 + 127) / 128 * 128);
+  // An MMA reads 128 rows of 128 bytes from each X box whatever x_rows is (the extra rows' results are never
+  // stored); the code ring and the slack behind the last stage keep those reads inside the allocation.
+  const size_t slack = a.x_rows < INF_M ? (size_t)INF_M * 128 : 0;
+  const size_t fixed = 1024 + (size_t)INF_C_STAGES * a.c_bytes + sizeof(InferBarriers) + slack;
+  a.op_stages = (int)std::min<size_t>(INF_MAX_OP_STAGES, (INF_SMEM_LIMIT - fixed) / (a.x_bytes + a.w_bytes));
+  if (a.op_stages < 2) return L4Q_ERR_UNSUPPORTED;
+  a.workers = std::min(INF_WORKERS, a.nb * a.op_stages);
+  const size_t smem = fixed + (size_t)a.op_stages * (a.x_bytes + a.w_bytes);
   const int grid = std::min(a.tiles_m * a.tiles_n, sm_count());
   auto launch = [&](auto kern) -> l4q_status {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
