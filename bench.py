@@ -542,6 +542,23 @@ def run_extras(args):
         wbytes = pk["codes"].numel() * 4 + pk["s16"].numel() * 4
         copies = int(L2_BYTES * 1.5 // wbytes) + 1
         ring = [{k: v.clone() for k, v in pk.items()} for _ in range(copies)]
+        # the unquantized layer for comparison: the same product with a dense bf16 weight through cuBLAS
+        # (torch.matmul), weights rotated the same way, CUDA events around every call
+        dense_copies = int(L2_BYTES * 1.5 // (d_in * d_out * 2)) + 1
+        dense = [d["W0"].clone() for _ in range(dense_copies)]
+
+        def dense_us(X, n_calls):
+            for k in range(args.warmup):
+                torch.matmul(X, dense[k % dense_copies].t())
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_calls)]
+            torch.cuda.synchronize()
+            for k, (e0, e1) in enumerate(evs):
+                e0.record()
+                torch.matmul(X, dense[k % dense_copies].t())
+                e1.record()
+            torch.cuda.synchronize()
+            return sum(e0.elapsed_time(e1) for e0, e1 in evs) / n_calls * 1e3
+
         for tokens in (1, 2, 16, 64):
             dsc = l4q.make_desc(cfg, tokens=tokens)
             X = torch.randn(tokens, d_in, device=dev).to(torch.bfloat16)
@@ -555,8 +572,9 @@ def run_extras(args):
             nbytes = wbytes + tokens * (d_in + d_out) * 2
             out[f"infer_{d_in}x{d_out}_t{tokens}"] = {"us": us, "bytes": nbytes, "gbs": nbytes / us / 1e3,
                                                        "frac_hbm": nbytes / us / 1e3 / pk_["hbm_gbs"],
-                                                       "dense_bf16_bytes": d_in * d_out * 2}
-        del ring
+                                                       "dense_bf16_bytes": d_in * d_out * 2,
+                                                       "dense_bf16_cublas_us": dense_us(X, reps * dense_copies)}
+        del ring, dense
 
     # ---- initialisation of s, b (App. B) and the error sums (Table 4): one pass over a bf16 weight ----
     cfg = synth.CONFIG3A

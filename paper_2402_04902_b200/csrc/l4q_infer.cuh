@@ -45,6 +45,7 @@ struct InferArgs {
   int x_rows;                              // token rows a TMA box of X brings in (8 .. 128)
   int tiles_m, tiles_n, num_kb;
   int op_stages;                           // depth of the operand ring
+  int one_group;                           // group size is a multiple of 128: a k-step lies in one group
   int workers;                             // dequantizer warps at work: min(INF_WORKERS, nb * op_stages)
   uint32_t x_bytes, w_bytes, c_bytes;      // per stage: X tile (two boxes of x_rows x 64), W tile (two of N x 64), codes
   const __half *s16, *b16;
@@ -63,32 +64,34 @@ struct __align__(8) InferBarriers {
 
 constexpr size_t INF_SMEM_LIMIT = 227 * 1024;
 
-// 32 unsigned codes of one weight row (starting at a multiple of 32 codes of the LSB-first bitstream), each
-// returned as the float m = 1 + u / 2^BITS: the code is moved into the top mantissa bits under the exponent
-// of 1.0 (one shift and one logic op, no integer-to-float conversion).  The caller folds the affine map back:
-// u * s + b = m * (2^BITS s) + (b - 2^BITS s), a single fma.
-template <int BITS>
-__device__ __forceinline__ float unpack_code(const uint32_t (&w)[BITS], int j) {      // j: compile-time after unrolling
-  constexpr int POS = 23 - BITS;                               // bit position of the code inside the mantissa
-  constexpr uint32_t MASK = ((1u << BITS) - 1u) << POS;
-  const int bit = j * BITS, wd = bit >> 5, off = bit & 31;
-  uint32_t v;
-  if (off + BITS > 32) v = __funnelshift_r(w[wd], w[wd + 1 < BITS ? wd + 1 : wd], off) << POS;   // code straddles two words
-  else v = (off <= POS) ? (w[wd] << (POS - off)) : (w[wd] >> (off - POS));
-  return __uint_as_float((v & MASK) | 0x3F800000u);
-}
-
-template <int BITS>
-__device__ __forceinline__ void unpack_codes32(const uint32_t (&w)[BITS], float (&m)[32]) {
-#pragma unroll
-  for (int j = 0; j < 32; ++j) m[j] = unpack_code<BITS>(w, j);
-}
-
 // (a & b) | c in one logic instruction, all three operands in registers.
 __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
   uint32_t d;
   asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
+}
+
+// 32 unsigned codes of one weight row (starting at a multiple of 32 codes of the LSB-first bitstream), each
+// returned as the float m = 1 + u / 2^BITS: the code is moved into the top mantissa bits under the exponent
+// of 1.0 (one shift and one logic op, no integer-to-float conversion).  The caller folds the affine map back:
+// u * s + b = m * (2^BITS s) + (b - 2^BITS s), a single fma.
+template <int BITS>
+__device__ __forceinline__ float unpack_code(const uint32_t (&w)[BITS], int j, uint32_t mask, uint32_t one) {   // j: compile-time after unrolling
+  constexpr int POS = 23 - BITS;                               // bit position of the code inside the mantissa
+  const int bit = j * BITS, wd = bit >> 5, off = bit & 31;
+  uint32_t v;
+  if (off + BITS > 32) v = __funnelshift_r(w[wd], w[wd + 1 < BITS ? wd + 1 : wd], off) << POS;   // code straddles two words
+  else v = (off <= POS) ? (w[wd] << (POS - off)) : (w[wd] >> (off - POS));
+  return __uint_as_float(and_or(v, mask, one));
+}
+
+// The mask of the code field and the exponent of 1.0 for unpack_code, in registers that the compiler cannot fold
+// back into immediates (with two immediates the and-or takes two instructions).
+template <int BITS>
+__device__ __forceinline__ void unpack_constants(uint32_t& mask, uint32_t& one) {
+  mask = ((1u << BITS) - 1u) << (23 - BITS);
+  one = 0x3F800000u;
+  asm volatile("" : "+r"(mask), "+r"(one));
 }
 
 // 32 codes of one weight row -> 16 words of bf16 pairs W_q = u * s + b (Eq. 9 on the unsigned code), formed in
@@ -280,6 +283,18 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
     const uint32_t c_base_a = smem_a + (uint32_t)S * op_bytes;
     const uint32_t full_c_a = ptx::smem_u32(&bars->full_c[0]), empty_c_a = ptx::smem_u32(&bars->empty_c[0]);
     const uint32_t full_op_a = ptx::smem_u32(&bars->full_op[0]), empty_op_a = ptx::smem_u32(&bars->empty_op[0]);
+    // byte offsets of this thread inside a block of 16 rows: its two runs of code words, and the eight 16-byte
+    // chunks it stores (the swizzle term row % 8 does not depend on the block)
+    const uint32_t c_off[2] = {(uint32_t)(r16 * (CW * 4) + q0 * (BITS * 4)), (uint32_t)(r16 * (CW * 4) + (q0 ^ 2) * (BITS * 4))};
+    uint32_t w_off[2][4];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int q = q0 ^ (h * 2);
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        w_off[h][c] = (uint32_t)(q >> 1) * (a.w_bytes / 2) + (uint32_t)(r16 * 128) +
+                      ((((uint32_t)((q & 1) * 4 + c)) ^ (uint32_t)(r16 & 7)) << 4);
+    }
     int stage = 0; uint32_t phase = 0;                         // operand ring, at k-step `ks` of the current tile
     int cs = 0; uint32_t cphase = 0;                           // code ring
     auto advance = [&](int d) {
@@ -300,57 +315,67 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
       while (works && blk >= NB) { blk -= NB; ++ks; }
       advance(min(ks, a.num_kb));                            // (a warp without a block in this tile just moves on)
       // s, b (fp16 bit patterns) of the groups of this thread's codes (group size is a multiple of 32), for quarter
-      // q0 and for quarter q0 ^ 2, fetched one block ahead and left untouched in registers until they are used
-      auto load_sb = [&](int ks_, int blk_, unsigned short (&sv)[2], unsigned short (&bv)[2]) {
+      // q0 and for quarter q0 ^ 2, fetched one block ahead and left untouched in registers until they are used.
+      // When the group size is a multiple of 128 both quarters lie in one group.
+      auto load_sb = [&](int ks_, int blk_, uint32_t (&sv)[2], uint32_t (&bv)[2]) {
         const int o = n0 + blk_ * 16 + r16;
-        sv[0] = sv[1] = bv[0] = bv[1] = 0;                     // rows / columns beyond the weight contribute nothing
+        sv[0] = sv[1] = bv[0] = bv[1] = 0u;                    // rows / columns beyond the weight contribute nothing
         if (ks_ < a.num_kb && o < a.d_out) {
           const unsigned short* s_row = reinterpret_cast<const unsigned short*>(a.s16) + (size_t)o * a.ngroups;
           const unsigned short* b_row = reinterpret_cast<const unsigned short*>(a.b16) + (size_t)o * a.ngroups;
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int k = ks_ * INF_BK + (q0 ^ (h * 2)) * 32;
+          if (a.one_group) {
+            const int k = ks_ * INF_BK;
             if (k < a.d_in) {
               const int g = a.group_shift >= 0 ? (k >> a.group_shift) : (k / a.group);
-              sv[h] = __ldg(s_row + g);
-              bv[h] = __ldg(b_row + g);
+              sv[0] = sv[1] = ptx::ldg_u16(s_row + g);
+              bv[0] = bv[1] = ptx::ldg_u16(b_row + g);
+            }
+          } else {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int k = ks_ * INF_BK + (q0 ^ (h * 2)) * 32;
+              if (k < a.d_in) {
+                const int g = a.group_shift >= 0 ? (k >> a.group_shift) : (k / a.group);
+                sv[h] = ptx::ldg_u16(s_row + g);
+                bv[h] = ptx::ldg_u16(b_row + g);
+              }
             }
           }
         }
       };
-      unsigned short s_next[2], b_next[2];
+      uint32_t s_next[2], b_next[2];
       load_sb(ks, blk, s_next, b_next);
       while (ks < a.num_kb) {
-        const int row = blk * 16 + r16;
-        const unsigned short s_cur[2] = {s_next[0], s_next[1]}, b_cur[2] = {b_next[0], b_next[1]};
+        const uint32_t s_cur[2] = {s_next[0], s_next[1]}, b_cur[2] = {b_next[0], b_next[1]};
         int nblk = blk + step_blk, d = step_ks;
         if (nblk >= NB) { nblk -= NB; ++d; }
         load_sb(ks + d, nblk, s_next, b_next);
         bounded_wait_a(full_c_a + (uint32_t)cs * 8u, cphase, bars);          // the code words have landed
         bounded_wait_a(empty_op_a + (uint32_t)stage * 8u, phase ^ 1, bars);  // the operand slot is free (its MMAs completed)
-        const uint32_t c_row = c_base_a + (uint32_t)cs * a.c_bytes + (uint32_t)(row * (CW * 4));
-        const uint32_t w_row = smem_a + (uint32_t)stage * op_bytes + a.x_bytes + (uint32_t)(row * 128);
-        const uint32_t sw = (uint32_t)(row & 7);
+        const uint32_t c_row = c_base_a + (uint32_t)cs * a.c_bytes + (uint32_t)(blk * (16 * CW * 4));
+        const uint32_t w_row = smem_a + (uint32_t)stage * op_bytes + a.x_bytes + (uint32_t)(blk * (16 * 128));
+        uint32_t w[2][BITS];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int q = q0 ^ (h * 2);
-          const float s_ = __half2float(__ushort_as_half(s_cur[h]));
-          const float b_ = __half2float(__ushort_as_half(b_cur[h]));
-          uint32_t w[BITS];
+        for (int h = 0; h < 2; ++h) {                          // (both loads first: they are independent of the stores below)
+          const uint32_t at = c_row + c_off[h];
           if constexpr (BITS == 4) {
-            const uint4 v = ptx::lds128(c_row + (uint32_t)(q * 16));
-            w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+            const uint4 v = ptx::lds128(at);
+            w[h][0] = v.x; w[h][1] = v.y; w[h][2] = v.z; w[h][3] = v.w;
           } else {
 #pragma unroll
-            for (int i = 0; i < BITS; ++i) w[i] = ptx::lds32(c_row + (uint32_t)(q * (BITS * 4) + i * 4));
+            for (int i = 0; i < BITS; ++i) w[h][i] = ptx::lds32(at + (uint32_t)(i * 4));
           }
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float s_ = __half2float(__ushort_as_half((unsigned short)s_cur[h]));
+          const float b_ = __half2float(__ushort_as_half((unsigned short)b_cur[h]));
           uint32_t wv[16];
-          dequant_codes32<BITS>(w, s_, b_, wv);
-          // into the K-major swizzled B operand: 64-k tile q >> 1, 16-byte chunks (q & 1) * 4 .. + 3 of row `row`
-          const uint32_t dst = w_row + (uint32_t)(q >> 1) * (a.w_bytes / 2);
+          dequant_codes32<BITS>(w[h], s_, b_, wv);
+          // into the K-major swizzled B operand: 64-k tile q >> 1, 16-byte chunks (q & 1) * 4 .. + 3 of the row
 #pragma unroll
           for (int c = 0; c < 4; ++c)
-            ptx::sts128(dst + ((((uint32_t)((q & 1) * 4 + c)) ^ sw) << 4), wv[c * 4 + 0], wv[c * 4 + 1], wv[c * 4 + 2], wv[c * 4 + 3]);
+            ptx::sts128(w_row + w_off[h][c], wv[c * 4 + 0], wv[c * 4 + 1], wv[c * 4 + 2], wv[c * 4 + 3]);
         }
         ptx::mbar_arrive_a(empty_c_a + (uint32_t)cs * 8u);     // code words consumed
         ptx::fence_proxy_async_smem();                         // the operand is read by the tensor cores
@@ -418,7 +443,7 @@ k_infer_bf16(const __grid_constant__ CUtensorMap tmap_x,      // X [tokens, d_in
 //   * a warp owns GEMV_ROWS weight rows at a time and walks along k; a lane takes 32 codes of each row
 //     (16 or 12 contiguous bytes: the warp reads 512 / 384 contiguous bytes per row) and the matching 32
 //     values of X, so the reads of X are shared by the rows;
-//   * codes become m = 1 + u / 2^bits (unpack_codes32); per piece  sum x W_q = (2^bits s) sum x m + (b - 2^bits s) sum x.
+//   * codes become m = 1 + u / 2^bits (unpack_code); per piece  sum x W_q = (2^bits s) sum x m + (b - 2^bits s) sum x.
 // ---------------------------------------------------------------------------
 constexpr int GEMV_ROWS = 2;
 constexpr int GEMV_THREADS = 256;
@@ -456,6 +481,8 @@ k_infer_gemv(const __nv_bfloat16* __restrict__ X, const uint32_t* __restrict__ c
   const int warps_total = gridDim.x * (GEMV_THREADS / 32);
   const int row_words = (d_in * BITS) >> 5;
   constexpr float kScale = (float)(1 << BITS);
+  uint32_t cmask, cone;
+  unpack_constants<BITS>(cmask, cone);
   for (int r0 = (blockIdx.x * (GEMV_THREADS / 32) + warp) * GEMV_ROWS; r0 < d_out; r0 += warps_total * GEMV_ROWS) {
     float acc[GEMV_ROWS][TOK];
 #pragma unroll
@@ -490,8 +517,8 @@ k_infer_gemv(const __nv_bfloat16* __restrict__ X, const uint32_t* __restrict__ c
           x4[t] = *reinterpret_cast<const float4*>(xs + (size_t)t * d_in + ((size_t)v * units + u) * 4);
 #pragma unroll
         for (int r = 0; r < GEMV_ROWS; ++r) {
-          const float m0 = unpack_code<BITS>(w[r], v * 4 + 0), m1 = unpack_code<BITS>(w[r], v * 4 + 1);
-          const float m2 = unpack_code<BITS>(w[r], v * 4 + 2), m3 = unpack_code<BITS>(w[r], v * 4 + 3);
+          const float m0 = unpack_code<BITS>(w[r], v * 4 + 0, cmask, cone), m1 = unpack_code<BITS>(w[r], v * 4 + 1, cmask, cone);
+          const float m2 = unpack_code<BITS>(w[r], v * 4 + 2, cmask, cone), m3 = unpack_code<BITS>(w[r], v * 4 + 3, cmask, cone);
 #pragma unroll
           for (int t = 0; t < TOK; ++t) {
             dot[r][t] = fmaf(x4[t].x, m0, dot[r][t]);
@@ -525,9 +552,14 @@ k_infer_gemv(const __nv_bfloat16* __restrict__ X, const uint32_t* __restrict__ c
 
 inline size_t gemv_smem_bytes(int tokens, int d_in) { return (size_t)tokens * (d_in + (d_in >> 5)) * sizeof(float); }
 
+inline int infer_pick_tile_n(int d_out, int tiles_m, int sms);
+
+// Measured (weights from HBM): at one token the matrix-vector kernel is the faster one on every layer shape; at two
+// tokens it still is where the tensor-core kernel's tiles are narrow (few weight rows per SM), and no longer where
+// they are 64 rows or taller; beyond two tokens the tensor-core kernel always is.
 inline bool gemv_supported(const Params& p) {
-  return p.tokens <= 2 && p.d_in % 32 == 0     // measured: beyond two tokens the tensor-core kernel is the faster one
-         && gemv_smem_bytes(p.tokens, p.d_in) <= 200 * 1024;
+  if (p.tokens > 2 || p.d_in % 32 != 0 || gemv_smem_bytes(p.tokens, p.d_in) > 200 * 1024) return false;
+  return p.tokens == 1 || infer_pick_tile_n(p.d_out, 1, sm_count()) < 64;
 }
 
 inline l4q_status launch_infer_gemv(const Params& p, const void* X, const uint32_t* codes, const __half* s16,
@@ -593,6 +625,7 @@ inline l4q_status launch_infer_bf16(const Params& p, const void* X, const uint32
   for (int sh = 5; sh < 31; ++sh)
     if ((1 << sh) == p.group) a.group_shift = sh;
   a.s16 = s16; a.b16 = b16;
+  a.one_group = (p.group % INF_BK == 0) ? 1 : 0;
   a.Y = reinterpret_cast<__nv_bfloat16*>(Y);
   CUtensorMap tx, tc;
   a.x_rows = std::min(INF_M, (p.tokens + 7) / 8 * 8);

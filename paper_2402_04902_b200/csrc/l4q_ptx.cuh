@@ -65,6 +65,13 @@ __device__ __forceinline__ void mbar_arrive_a(uint32_t bar_a) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_a) : "memory");
 }
 
+// 16-bit read-only global load, zero-extended into a 32-bit register
+__device__ __forceinline__ uint32_t ldg_u16(const unsigned short* p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.u16 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+
 // ---- shared memory through 32-bit shared-window addresses (smem_u32) --------
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;

@@ -62,6 +62,15 @@ def test_infer_llama7b_mlp_up_batch_16():
     _run(synth.CONFIG3A.with_(name="infer_cfg3a_b16", tokens=16), seed=0)
 
 
+def test_infer_llama7b_mlp_down_batch_64():
+    # 11008 -> 4096: 86 k-steps on narrow tiles (32 weight rows per SM)
+    _run(synth.CONFIG3B.with_(name="infer_cfg3b_b64", tokens=64), seed=0)
+
+
+def test_infer_llama7b_attn_proj_batch_16():
+    _run(synth.CONFIG2.with_(name="infer_cfg2_b16", tokens=16), seed=0)
+
+
 @pytest.mark.parametrize("d_in,d_out,tokens,bits", [(4096, 1000, 1, 4), (4096, 1000, 4, 4), (11008, 520, 1, 4),
                                                     (11008, 520, 2, 4), (14336, 264, 1, 4), (4096, 392, 2, 3),
                                                     (11008, 392, 1, 3), (11008, 392, 3, 4)])
