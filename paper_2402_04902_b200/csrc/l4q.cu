@@ -13,6 +13,7 @@
 #include "l4q_val.cuh"
 #include "l4q_gemm.cuh"
 #include "l4q_wtile.cuh"
+#include "l4q_init.cuh"
 #include "l4q_infer.cuh"
 #include "l4q_variants.cuh"
 #include "l4q_tilecopy.cuh"
@@ -570,6 +571,7 @@ l4q_status l4q_init_params(const l4q_desc* desc, const void* W, int method, floa
   const int blocks = (int)std::min<long long>((groups + 7) / 8, (long long)sm_count() * 16);
   const bool signed_grid = (desc->flags & L4Q_FLAG_SIGNED_GRID) != 0;
   KernelScope ks(L4Q_KERNEL_INIT, stream);
+  if (desc->io_dtype == L4Q_BF16 && init_tma_supported(p)) return launch_init_tma(p, method, signed_grid, W, s, b, stream);
   int lanes_log2 = -1;                                   // group = 8 * 2^k elements with k <= 5: the coalesced kernel
   for (int k = 0; k <= 5; ++k)
     if (p.group == (8 << k)) lanes_log2 = k;

@@ -27,6 +27,12 @@ CASES = [
     synth.LayerConfig("init_group256", tokens=8, d_in=768, d_out=40, rank=8, alpha=16.0, bits=3, group_size=256),
     synth.LayerConfig("init_many_pieces", tokens=8, d_in=4096, d_out=2048, rank=8, alpha=16.0, bits=4,
                       group_size=64),
+    # the TMA-fed kernel (bf16, groups of 32 / 64 / 128): a last column tile that is mostly beyond the weight and a
+    # ragged last row tile; and enough tiles per CTA for the ring of stages to go round twice
+    synth.LayerConfig("init_tma_ragged", tokens=8, d_in=1184, d_out=296, rank=8, alpha=16.0, bits=3, group_size=32,
+                      signed_grid=True),
+    synth.LayerConfig("init_tma_ring_wraps", tokens=8, d_in=8192, d_out=4096, rank=8, alpha=16.0, bits=4,
+                      group_size=128),
 ]
 
 
