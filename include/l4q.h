@@ -171,8 +171,8 @@ l4q_status l4q_lora_linear_bwd(const l4q_desc* desc, int kind, const void* X, co
  *     W_q[o, j] = u[o, j] * s_fp16[o, j / group_size] + b_fp16[o, j / group_size]     (Eq. 9, unsigned code u)
  * and never exists in memory as a whole (bits / 8 bytes per weight are read).
  * In: X [tokens, d_in] bf16; codes [d_out, d_in * bits / 32] uint32, s_fp16, b_fp16 [d_out, d_in / group_size]
- * exactly as written by l4q_pack_int.  Out: Y [tokens, d_out] bf16, overwritten.  W_q is formed in fp32 and
- * rounded to bf16 for the tensor cores, accumulation is fp32.
+ * exactly as written by l4q_pack_int.  Out: Y [tokens, d_out] bf16, overwritten.  W_q is formed in fp32 (within
+ * 2^-12 of a quantization step of u s + b) and rounded once to bf16 for the tensor cores; accumulation is fp32.
  * Meant for the few-token regime of App. F (a step of batch 1..64); larger token counts work (in tiles of 128
  * tokens, each of which reads the weight again).  io_dtype must be L4Q_BF16, bits 3 or 4, group_size a multiple
  * of 32 and d_in * bits / 8 a multiple of 16 (else L4Q_ERR_UNSUPPORTED); rank, alpha and flags are ignored.
